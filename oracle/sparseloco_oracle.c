@@ -1,0 +1,506 @@
+/*
+ * CPU oracle for the SparseLoCo outer step.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-definition implementation of what the outer step
+ * computes, written from the paper's statement of the method.  It shares no
+ * code with the CUDA library and is never called by it: only the tests, the
+ * smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What follows what:
+ *   pseudo-gradient  Delta_r = theta - theta_r         Sec. 3.1; Algorithm 1, pseudo-gradient line
+ *   error feedback   u = beta e + Delta                Eq. 2 line 1; Algorithm 1, compression line
+ *   chunked Top-k    64x64 blocks of 2-D tensors, runs of 4096 of 1-D tensors,
+ *                    Top-k by magnitude inside each chunk       Sec. 3.3 (chunk-wise Top-k paragraph)
+ *   quantiser Q      per tensor: centre by the mean, [-6 sigma, 6 sigma] in four
+ *                    uniform bins, each bin's centroid as look-up table    Sec. 4 (experimental setup)
+ *   index cost       12 bits per in-chunk index at C = 4096     App. "Compression of indices"
+ *   EF subtract      e = u - Delta_hat                  Eq. 2 line 2; Algorithm 1, error line
+ *   aggregate        Delta = (1/R) sum_r Delta_hat_r    Eq. 2 line 3; Algorithm 1, aggregation line
+ *   outer update     theta = theta - alpha Delta        Eq. 2 line 4; Algorithm 1, last line
+ *   EF freeze        e neither used nor accumulated     App. "Freezing Error Feedback"
+ *
+ * Readings taken where the paper is silent (each is also listed in the design
+ * notes of the repository):
+ *   - "magnitude" = the IEEE-754 bit pattern with the sign bit cleared, compared
+ *     as an unsigned integer; ties go to the lowest in-chunk index.
+ *   - in-chunk index of a 64x64 block is row-major inside the block; blocks are
+ *     visited block-row-major; a 2-D tensor whose sides are not both multiples
+ *     of the block side is treated as 1-D (row-major runs of 4096, short tail).
+ *   - selected entries of a chunk are listed by ascending in-chunk index.
+ *   - u = fmaf(beta, e, theta - theta_r): one fp32 subtraction, one fused
+ *     multiply-add, round-to-nearest, denormals kept.
+ *   - sigma is the population standard deviation (divide by n) of the fp32
+ *     centred values; sums are fp64, taken slot by slot inside a chunk and then
+ *     chunk by chunk.  Bin edges on centred values are -3 sigma, 0, +3 sigma
+ *     with the lower edge inclusive; values beyond +-6 sigma fall in the outer
+ *     bins.  Centroids are means of the raw (uncentred) values; an empty bin
+ *     stores +0.
+ *   - the average divides by R even when a worker's payload is absent, unless
+ *     divide_by_present is set.
+ *
+ * Every function here is pinned by tests/test_oracle_*.py against brute force,
+ * hand-worked cases, closed forms and invariants (none of them produced by this
+ * file or by the CUDA path).
+ *
+ * Arithmetic: fp32 where the method stores fp32 (u, e, centred values, sigma,
+ * thresholds, table), fp64 for every accumulation.  Build with
+ * -ffp-contract=off and without -ffast-math.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int64_t rows, cols; /* 1-D tensor: rows == 1 */
+    int64_t offset;     /* element offset into every flat buffer */
+} orc_tensor;
+
+typedef struct {
+    int32_t chunk_elems; /* C; tile_dim * tile_dim */
+    int32_t tile_dim;    /* side of a 2-D block */
+    int32_t k;
+    int32_t R, H;
+    float beta, outer_lr;
+    int32_t quant_bits;        /* 2, or 32 = values sent unquantised */
+    int32_t ef_enabled;        /* 0 during the error-feedback freeze */
+    int32_t divide_by_present; /* 0: divide by R; 1: by the number of payloads present */
+} orc_config;
+
+static int g_threads = 1;
+void orc_set_threads(int n) { g_threads = n < 1 ? 1 : n; }
+int orc_get_threads(void) { return g_threads; }
+
+/* ---------------------------------------------------------------- chunk geometry (Sec. 3.3) */
+
+static int is_tiled(const orc_config* c, const orc_tensor* t) {
+    return t->rows > 1 && t->rows % c->tile_dim == 0 && t->cols % c->tile_dim == 0;
+}
+
+int64_t orc_num_chunks(const orc_config* c, const orc_tensor* t) {
+    int64_t n = t->rows * t->cols;
+    if (is_tiled(c, t)) return (t->rows / c->tile_dim) * (t->cols / c->tile_dim);
+    return (n + c->chunk_elems - 1) / c->chunk_elems;
+}
+
+/* Length of chunk `ch` of tensor t. */
+int64_t orc_chunk_len(const orc_config* c, const orc_tensor* t, int64_t ch) {
+    if (is_tiled(c, t)) return c->chunk_elems;
+    int64_t n = t->rows * t->cols;
+    int64_t start = ch * c->chunk_elems;
+    int64_t rest = n - start;
+    return rest < c->chunk_elems ? rest : c->chunk_elems;
+}
+
+/* Element position (inside the tensor, row-major) of in-chunk index p of chunk ch. */
+int64_t orc_chunk_pos(const orc_config* c, const orc_tensor* t, int64_t ch, int64_t p) {
+    if (is_tiled(c, t)) {
+        int64_t tiles_per_row = t->cols / c->tile_dim;
+        int64_t tr = ch / tiles_per_row, tc = ch % tiles_per_row;
+        int64_t row = tr * c->tile_dim + p / c->tile_dim;
+        int64_t col = tc * c->tile_dim + p % c->tile_dim;
+        return row * t->cols + col;
+    }
+    return ch * c->chunk_elems + p;
+}
+
+int64_t orc_total_chunks(const orc_config* c, const orc_tensor* ts, int32_t nt) {
+    int64_t s = 0;
+    for (int32_t j = 0; j < nt; ++j) s += orc_num_chunks(c, &ts[j]);
+    return s;
+}
+
+/* Total number of selected entries of one worker: sum over chunks of min(k, chunk length). */
+int64_t orc_total_slots(const orc_config* c, const orc_tensor* ts, int32_t nt) {
+    int64_t s = 0;
+    for (int32_t j = 0; j < nt; ++j) {
+        int64_t nc = orc_num_chunks(c, &ts[j]);
+        for (int64_t ch = 0; ch < nc; ++ch) {
+            int64_t L = orc_chunk_len(c, &ts[j], ch);
+            s += L < c->k ? L : c->k;
+        }
+    }
+    return s;
+}
+
+/* ---------------------------------------------------------------- payload geometry (App. index cost) */
+
+/* Bytes of one chunk record: k 12-bit indices, then k 2-bit codes, rounded up to 16. */
+int64_t orc_record_stride(int32_t k) {
+    int64_t idx_bytes = (12 * (int64_t)k + 7) / 8;
+    int64_t code_bytes = (2 * (int64_t)k + 7) / 8;
+    return (idx_bytes + code_bytes + 15) / 16 * 16;
+}
+
+/* Bytes of one worker's payload: one 16-byte table per tensor, then every chunk record. */
+int64_t orc_payload_bytes(const orc_config* c, const orc_tensor* ts, int32_t nt) {
+    return 16 * (int64_t)nt + orc_record_stride(c->k) * orc_total_chunks(c, ts, nt);
+}
+
+/* ---------------------------------------------------------------- pseudo-gradient + error feedback */
+
+/* u[i] = beta * e[i] + (theta[i] - theta_r[i]); with the freeze on, u = theta - theta_r.
+ * Eq. 2 line 1 / Algorithm 1. */
+void orc_ef_accumulate(const float* theta, const float* theta_r, const float* e, int64_t n,
+                       float beta, int ef_enabled, float* u) {
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        float d = theta[i] - theta_r[i];
+        u[i] = ef_enabled ? fmaf(beta, e[i], d) : d;
+    }
+}
+
+/* ---------------------------------------------------------------- Top-k of one chunk */
+
+typedef struct {
+    uint32_t key; /* magnitude: bit pattern without the sign */
+    int32_t p;    /* in-chunk index */
+} keyed;
+
+static uint32_t mag_key(float x) {
+    uint32_t b;
+    memcpy(&b, &x, 4);
+    return b & 0x7FFFFFFFu;
+}
+
+static int cmp_mag_desc_index_asc(const void* a, const void* b) {
+    const keyed* x = (const keyed*)a;
+    const keyed* y = (const keyed*)b;
+    if (x->key != y->key) return x->key > y->key ? -1 : 1;
+    return x->p < y->p ? -1 : (x->p > y->p ? 1 : 0);
+}
+
+static int cmp_int32_asc(const void* a, const void* b) {
+    int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+/* The min(k, L) entries of u[0..L) of largest magnitude, ties to the lower index,
+ * returned as ascending in-chunk indices.  Full sort, by definition.  Returns the count. */
+int32_t orc_topk_chunk(const float* u, int32_t L, int32_t k, int32_t* idx_out) {
+    keyed* a = (keyed*)malloc(sizeof(keyed) * (size_t)(L > 0 ? L : 1));
+    for (int32_t p = 0; p < L; ++p) {
+        a[p].key = mag_key(u[p]);
+        a[p].p = p;
+    }
+    qsort(a, (size_t)L, sizeof(keyed), cmp_mag_desc_index_asc);
+    int32_t m = k < L ? k : L;
+    for (int32_t s = 0; s < m; ++s) idx_out[s] = a[s].p;
+    qsort(idx_out, (size_t)m, sizeof(int32_t), cmp_int32_asc);
+    free(a);
+    return m;
+}
+
+/* ---------------------------------------------------------------- quantiser Q of one tensor */
+
+/* v: the tensor's selected values, chunk after chunk, each chunk's `cnt[c]` values in slot order.
+ * Outputs: mu, sigma, lut[4], code per value.  Sec. 4: centre by the mean, [-6 sigma, 6 sigma]
+ * in four uniform bins (edges -3 sigma, 0, 3 sigma on centred values), centroid table. */
+void orc_quantize_tensor(const float* v, const int32_t* cnt, int64_t n_chunks, float* mu_out,
+                         float* sigma_out, float lut[4], uint8_t* code) {
+    int64_t n = 0;
+    for (int64_t c = 0; c < n_chunks; ++c) n += cnt[c];
+    lut[0] = lut[1] = lut[2] = lut[3] = 0.0f;
+    *mu_out = 0.0f;
+    *sigma_out = 0.0f;
+    if (n == 0) return;
+
+    double S = 0.0;
+    {
+        const float* q = v;
+        for (int64_t c = 0; c < n_chunks; ++c) {
+            double sc = 0.0;
+            for (int32_t s = 0; s < cnt[c]; ++s) sc += (double)q[s];
+            S += sc;
+            q += cnt[c];
+        }
+    }
+    float mu = (float)(S / (double)n);
+
+    double V = 0.0;
+    {
+        const float* q = v;
+        for (int64_t c = 0; c < n_chunks; ++c) {
+            double vc = 0.0;
+            for (int32_t s = 0; s < cnt[c]; ++s) {
+                float cen = q[s] - mu;
+                double d = (double)cen;
+                vc += d * d;
+            }
+            V += vc;
+            q += cnt[c];
+        }
+    }
+    float sigma = (float)sqrt(V / (double)n);
+    float t = 3.0f * sigma;
+
+    double Sb[4] = {0.0, 0.0, 0.0, 0.0};
+    int64_t nb[4] = {0, 0, 0, 0};
+    {
+        const float* q = v;
+        uint8_t* cq = code;
+        for (int64_t c = 0; c < n_chunks; ++c) {
+            double sb[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int32_t s = 0; s < cnt[c]; ++s) {
+                float cen = q[s] - mu;
+                int b = (cen >= -t) + (cen >= 0.0f) + (cen >= t);
+                cq[s] = (uint8_t)b;
+                sb[b] += (double)q[s];
+                nb[b] += 1;
+            }
+            for (int b = 0; b < 4; ++b) Sb[b] += sb[b];
+            q += cnt[c];
+            cq += cnt[c];
+        }
+    }
+    for (int b = 0; b < 4; ++b) lut[b] = nb[b] ? (float)(Sb[b] / (double)nb[b]) : 0.0f;
+    *mu_out = mu;
+    *sigma_out = sigma;
+}
+
+/* ---------------------------------------------------------------- packing (little-endian bit order) */
+
+static void put_bits(uint8_t* base, int64_t bit, int nbits, uint32_t val) {
+    for (int i = 0; i < nbits; ++i) {
+        if ((val >> i) & 1u) base[(bit + i) >> 3] |= (uint8_t)(1u << ((bit + i) & 7));
+    }
+}
+
+static uint32_t get_bits(const uint8_t* base, int64_t bit, int nbits) {
+    uint32_t v = 0;
+    for (int i = 0; i < nbits; ++i) {
+        v |= (uint32_t)((base[(bit + i) >> 3] >> ((bit + i) & 7)) & 1u) << i;
+    }
+    return v;
+}
+
+/* One chunk record: index block (12 bits per slot), then code block (2 bits per slot) starting
+ * at byte ceil(12k/8).  Slots >= m and all padding stay zero. */
+void orc_pack_record(const int32_t* idx, const uint8_t* code, int32_t m, int32_t k, uint8_t* rec) {
+    memset(rec, 0, (size_t)orc_record_stride(k));
+    int64_t code_base = ((12 * (int64_t)k + 7) / 8) * 8;
+    for (int32_t s = 0; s < m; ++s) {
+        put_bits(rec, 12 * (int64_t)s, 12, (uint32_t)idx[s]);
+        put_bits(rec, code_base + 2 * (int64_t)s, 2, code[s]);
+    }
+}
+
+void orc_unpack_record(const uint8_t* rec, int32_t m, int32_t k, int32_t* idx, uint8_t* code) {
+    int64_t code_base = ((12 * (int64_t)k + 7) / 8) * 8;
+    for (int32_t s = 0; s < m; ++s) {
+        idx[s] = (int32_t)get_bits(rec, 12 * (int64_t)s, 12);
+        code[s] = (uint8_t)get_bits(rec, code_base + 2 * (int64_t)s, 2);
+    }
+}
+
+/* ---------------------------------------------------------------- one worker's compression */
+
+/*
+ * Algorithm 1, compression + error feedback block, for one worker over all tensors.
+ *   theta, theta_r, e : flat fp32 buffers (tensor j at ts[j].offset); e is updated in place
+ *                       (left untouched when ef_enabled == 0).
+ *   payload           : orc_payload_bytes() bytes, or NULL (also unused when quant_bits == 32).
+ *   sel_idx, sel_val, sel_hat : optional (may be NULL) arrays of orc_total_slots() entries, in
+ *                       (tensor, chunk, slot) order: in-chunk index, raw value u, decoded value.
+ *   stats             : optional, 6 floats per tensor: mu, sigma, lut[0..3].
+ */
+void orc_compress(const orc_config* cfg, const orc_tensor* ts, int32_t nt, const float* theta,
+                  const float* theta_r, float* e, uint8_t* payload, int32_t* sel_idx,
+                  float* sel_val, float* sel_hat, float* stats) {
+    const int32_t k = cfg->k, C = cfg->chunk_elems;
+    const int64_t stride = orc_record_stride(k);
+    int64_t rec_off = 16 * (int64_t)nt; /* records follow the per-tensor tables */
+    int64_t slot_off = 0;
+    if (payload && cfg->quant_bits == 2) memset(payload, 0, (size_t)orc_payload_bytes(cfg, ts, nt));
+
+    for (int32_t j = 0; j < nt; ++j) {
+        const orc_tensor* t = &ts[j];
+        const int64_t n = t->rows * t->cols, nc = orc_num_chunks(cfg, t);
+        const float* th = theta + t->offset;
+        const float* tr = theta_r + t->offset;
+        float* ej = e + t->offset;
+
+        float* u = (float*)malloc(sizeof(float) * (size_t)n);
+        orc_ef_accumulate(th, tr, ej, n, cfg->beta, cfg->ef_enabled, u);
+
+        int32_t* cnt = (int32_t*)malloc(sizeof(int32_t) * (size_t)nc);
+        int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)(nc * k));
+        float* val = (float*)malloc(sizeof(float) * (size_t)(nc * k));
+
+        /* chunk-wise Top-k; chunks are independent */
+#pragma omp parallel for num_threads(g_threads) schedule(dynamic, 4)
+        for (int64_t ch = 0; ch < nc; ++ch) {
+            int32_t L = (int32_t)orc_chunk_len(cfg, t, ch);
+            float* cu = (float*)malloc(sizeof(float) * (size_t)C);
+            for (int32_t p = 0; p < L; ++p) cu[p] = u[orc_chunk_pos(cfg, t, ch, p)];
+            cnt[ch] = orc_topk_chunk(cu, L, k, idx + ch * k);
+            for (int32_t s = 0; s < cnt[ch]; ++s) val[ch * k + s] = cu[idx[ch * k + s]];
+            free(cu);
+        }
+
+        /* the tensor's selected values, chunk after chunk in slot order */
+        int64_t m_total = 0;
+        for (int64_t ch = 0; ch < nc; ++ch) m_total += cnt[ch];
+        float* v = (float*)malloc(sizeof(float) * (size_t)(m_total ? m_total : 1));
+        float* vhat = (float*)malloc(sizeof(float) * (size_t)(m_total ? m_total : 1));
+        uint8_t* code = (uint8_t*)malloc((size_t)(m_total ? m_total : 1));
+        {
+            int64_t w = 0;
+            for (int64_t ch = 0; ch < nc; ++ch)
+                for (int32_t s = 0; s < cnt[ch]; ++s) v[w++] = val[ch * k + s];
+        }
+
+        float mu = 0.0f, sigma = 0.0f, lut[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (cfg->quant_bits == 2) {
+            orc_quantize_tensor(v, cnt, nc, &mu, &sigma, lut, code);
+            for (int64_t w = 0; w < m_total; ++w) vhat[w] = lut[code[w]];
+        } else { /* 32: values travel unquantised */
+            for (int64_t w = 0; w < m_total; ++w) vhat[w] = v[w];
+        }
+        if (stats) {
+            stats[6 * j + 0] = mu;
+            stats[6 * j + 1] = sigma;
+            for (int b = 0; b < 4; ++b) stats[6 * j + 2 + b] = lut[b];
+        }
+
+        /* payload: table, then records */
+        if (payload && cfg->quant_bits == 2) {
+            memcpy(payload + 16 * (int64_t)j, lut, 16);
+            int64_t w = 0;
+            for (int64_t ch = 0; ch < nc; ++ch) {
+                orc_pack_record(idx + ch * k, code + w, cnt[ch], k, payload + rec_off + ch * stride);
+                w += cnt[ch];
+            }
+        }
+        rec_off += nc * stride;
+
+        /* error feedback: e = u - Delta_hat (Eq. 2 line 2) */
+        if (cfg->ef_enabled) {
+            for (int64_t i = 0; i < n; ++i) ej[i] = u[i];
+            int64_t w = 0;
+            for (int64_t ch = 0; ch < nc; ++ch)
+                for (int32_t s = 0; s < cnt[ch]; ++s, ++w) {
+                    int64_t pos = orc_chunk_pos(cfg, t, ch, idx[ch * k + s]);
+                    ej[pos] = u[pos] - vhat[w];
+                }
+        }
+
+        {
+            int64_t w = 0;
+            for (int64_t ch = 0; ch < nc; ++ch)
+                for (int32_t s = 0; s < cnt[ch]; ++s, ++w) {
+                    if (sel_idx) sel_idx[slot_off + w] = idx[ch * k + s];
+                    if (sel_val) sel_val[slot_off + w] = v[w];
+                    if (sel_hat) sel_hat[slot_off + w] = vhat[w];
+                }
+        }
+        slot_off += m_total;
+
+        free(u); free(cnt); free(idx); free(val); free(v); free(vhat); free(code);
+    }
+}
+
+/* ---------------------------------------------------------------- aggregate + outer update */
+
+/*
+ * Eq. 2 lines 3-4 from sparse lists.  For worker r (r < R), sel_idx[r] / sel_hat[r] hold its
+ * selected in-chunk indices and decoded values in (tensor, chunk, slot) order, or are NULL when
+ * that worker is absent.  theta[i] <- (float)(theta[i] - alpha * (sum_r hat_r[i]) / D) in fp64,
+ * r ascending; elements no worker selected are left bit-unchanged.
+ */
+void orc_aggregate_apply_sparse(const orc_config* cfg, const orc_tensor* ts, int32_t nt,
+                                const int32_t* const* sel_idx, const float* const* sel_hat,
+                                float* theta) {
+    const int32_t k = cfg->k, R = cfg->R;
+    int present = 0;
+    for (int32_t r = 0; r < R; ++r) present += sel_idx[r] != NULL;
+    const double D = cfg->divide_by_present ? (double)present : (double)R;
+    if (present == 0) return;
+
+    int64_t slot_off = 0;
+    for (int32_t j = 0; j < nt; ++j) {
+        const orc_tensor* t = &ts[j];
+        const int64_t n = t->rows * t->cols, nc = orc_num_chunks(cfg, t);
+        double* acc = (double*)calloc((size_t)n, sizeof(double));
+        uint8_t* hit = (uint8_t*)calloc((size_t)n, 1);
+        int64_t m_tensor = 0; /* slots of this tensor in every worker's list */
+        for (int64_t ch = 0; ch < nc; ++ch) {
+            int64_t L = orc_chunk_len(cfg, t, ch);
+            m_tensor += L < k ? L : k;
+        }
+        for (int32_t r = 0; r < R; ++r) {
+            if (!sel_idx[r]) continue;
+            int64_t w = slot_off;
+            for (int64_t ch = 0; ch < nc; ++ch) {
+                int64_t L = orc_chunk_len(cfg, t, ch);
+                int64_t m = L < k ? L : k;
+                for (int64_t s = 0; s < m; ++s, ++w) {
+                    int64_t pos = orc_chunk_pos(cfg, t, ch, sel_idx[r][w]);
+                    acc[pos] += (double)sel_hat[r][w];
+                    hit[pos] = 1;
+                }
+            }
+        }
+        float* th = theta + t->offset;
+        for (int64_t i = 0; i < n; ++i) {
+            if (hit[i]) th[i] = (float)((double)th[i] - (double)cfg->outer_lr * acc[i] / D);
+        }
+        slot_off += m_tensor;
+        free(acc); free(hit);
+    }
+}
+
+/* Decode one worker's payload (2-bit format) into sparse lists in (tensor, chunk, slot) order.
+ * Sec. 4: values are dequantised through the table before aggregation. */
+void orc_decode_payload(const orc_config* cfg, const orc_tensor* ts, int32_t nt,
+                        const uint8_t* payload, int32_t* sel_idx, float* sel_hat) {
+    const int32_t k = cfg->k;
+    const int64_t stride = orc_record_stride(k);
+    int64_t rec_off = 16 * (int64_t)nt, w = 0;
+    uint8_t* code = (uint8_t*)malloc((size_t)k);
+    for (int32_t j = 0; j < nt; ++j) {
+        float lut[4];
+        memcpy(lut, payload + 16 * (int64_t)j, 16);
+        int64_t nc = orc_num_chunks(cfg, &ts[j]);
+        for (int64_t ch = 0; ch < nc; ++ch) {
+            int64_t L = orc_chunk_len(cfg, &ts[j], ch);
+            int32_t m = (int32_t)(L < k ? L : k);
+            orc_unpack_record(payload + rec_off + ch * stride, m, k, sel_idx + w, code);
+            for (int32_t s = 0; s < m; ++s) sel_hat[w + s] = lut[code[s]];
+            w += m;
+        }
+        rec_off += nc * stride;
+    }
+    free(code);
+}
+
+/* Eq. 2 lines 3-4 from R packed payloads (NULL = absent worker). */
+void orc_aggregate_apply(const orc_config* cfg, const orc_tensor* ts, int32_t nt,
+                         const uint8_t* const* payloads, float* theta) {
+    const int32_t R = cfg->R;
+    const int64_t slots = orc_total_slots(cfg, ts, nt);
+    int32_t** idx = (int32_t**)calloc((size_t)R, sizeof(int32_t*));
+    float** hat = (float**)calloc((size_t)R, sizeof(float*));
+    for (int32_t r = 0; r < R; ++r) {
+        if (!payloads[r]) continue;
+        idx[r] = (int32_t*)malloc(sizeof(int32_t) * (size_t)(slots ? slots : 1));
+        hat[r] = (float*)malloc(sizeof(float) * (size_t)(slots ? slots : 1));
+        orc_decode_payload(cfg, ts, nt, payloads[r], idx[r], hat[r]);
+    }
+    orc_aggregate_apply_sparse(cfg, ts, nt, (const int32_t* const*)idx, (const float* const*)hat,
+                               theta);
+    for (int32_t r = 0; r < R; ++r) { free(idx[r]); free(hat[r]); }
+    free(idx); free(hat);
+}
+
+/* One full outer step (Algorithm 1, lines after the inner loop): compress every worker, then
+ * aggregate and update theta.  payloads[r] must each hold orc_payload_bytes() bytes. */
+void orc_outer_step(const orc_config* cfg, const orc_tensor* ts, int32_t nt, float* theta,
+                    const float* const* theta_r, float* const* e, uint8_t* const* payloads) {
+    for (int32_t r = 0; r < cfg->R; ++r)
+        orc_compress(cfg, ts, nt, theta, theta_r[r], e[r], payloads[r], NULL, NULL, NULL, NULL);
+    orc_aggregate_apply(cfg, ts, nt, (const uint8_t* const*)payloads, theta);
+}
