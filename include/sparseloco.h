@@ -1,0 +1,158 @@
+/*
+ * libsparseloco -- the SparseLoCo outer step on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every buffer argument is a DEVICE pointer unless it says "host".  The caller owns all
+ * device buffers it passes in (parameters, error buffers, payloads, workspace); the library owns
+ * only the context object and the small device-side chunk table built by sl_create().  All work is
+ * enqueued on the CUDA stream the caller passes (a cudaStream_t cast to void*; NULL = the default
+ * stream) and no entry point synchronises the host, except sl_create()/sl_destroy() and
+ * sl_outer_step_host().  There is no CPU implementation behind these calls.
+ *
+ * The method (paper: "SparseLoCo", Algorithm 1 and Eq. 2), per outer step, R workers:
+ *     Delta_r   = theta - theta_r                          pseudo-gradient       (Sec. 3.1, Alg. 1)
+ *     u_r       = beta * e_r + Delta_r                     error feedback        (Eq. 2 line 1)
+ *     Dhat_r    = Q(TopK(u_r))                             chunk-wise Top-k, 2-bit quantiser
+ *                                                          (Eq. 2 line 2; Sec. 3.3 chunking; Sec. 4 Q)
+ *     e_r       = u_r - Dhat_r                             error update          (Eq. 2 line 2)
+ *     theta     = theta - alpha * (1/R) sum_r Dhat_r       aggregate + outer SGD (Eq. 2 lines 3-4)
+ *
+ * Chunks (Sec. 3.3): a 2-D tensor whose sides are both multiples of 64 is cut into 64x64 blocks
+ * (block-row-major; in-chunk index = 64 * row_in_block + col_in_block); every other tensor is cut
+ * into row-major runs of 4096 elements with a short last run.  Top-k keeps, per chunk, the
+ * min(k, chunk length) entries of largest magnitude (IEEE bit pattern without the sign, compared
+ * as an integer; ties go to the lower in-chunk index), listed by ascending in-chunk index.
+ *
+ * Quantiser (Sec. 4): per (worker, tensor), over all selected values: mean mu, population sigma of
+ * the centred values, bins (-inf,-3s) [-3s,0) [0,3s) [3s,inf) on centred values, table entry =
+ * mean of the raw values in the bin (+0 when empty).  Sums are fp64, slot by slot inside a chunk,
+ * then chunk by chunk.
+ *
+ * Payload of one worker (little-endian; App. "Compression of indices": 12 bits per index):
+ *     bytes [16 j, 16 j + 16)          table of tensor j: 4 x fp32
+ *     then one record per chunk, in (tensor, chunk) order, each sl_record_stride(k) bytes:
+ *         bits  [12 s, 12 s + 12)                   in-chunk index of slot s
+ *         bytes from ceil(12 k / 8): bits [2 s, 2 s + 2)   code of slot s
+ *     slots >= min(k, chunk length) and all padding are zero.
+ */
+#ifndef SPARSELOCO_H
+#define SPARSELOCO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SL_OK = 0,
+    SL_ERR_INVALID_ARG = 1, /* NULL pointer, size or hyper-parameter out of range */
+    SL_ERR_ALIGNMENT = 2,   /* a device pointer or tensor offset is not 16-byte aligned */
+    SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, bits != 2, ...) */
+    SL_ERR_BAD_PAYLOAD = 4, /* reported through the device status word of sl_validate_payload */
+    SL_ERR_CUDA = 5,        /* a CUDA runtime call failed; see sl_last_cuda_error() */
+    SL_ERR_NOMEM = 6,       /* workspace missing or too small */
+    SL_ERR_TOO_LARGE = 7    /* problem exceeds a fixed built-in capacity */
+} sl_status;
+
+/* One parameter tensor: rows x cols fp32, row-major, at element offset `offset` of every flat
+ * buffer (theta, theta_r, e).  1-D tensors have rows == 1.  offset must be a multiple of 4. */
+typedef struct {
+    int64_t rows, cols;
+    int64_t offset;
+} sl_tensor_desc;
+
+/* Hyper-parameters, named as in Algorithm 1's "Require" line and Sec. 4. */
+typedef struct {
+    int32_t chunk_elems;       /* C: must be 4096 */
+    int32_t tile_dim;          /* must be 64 */
+    int32_t k;                 /* entries kept per chunk, 1..256 */
+    int32_t R;                 /* workers, 1..64 */
+    int32_t H;                 /* inner steps; carried for the caller, >= 1, unused by the math */
+    float beta;                /* error-feedback decay, 0 <= beta <= 1 */
+    float outer_lr;            /* alpha, finite */
+    int32_t quant_bits;        /* must be 2 */
+    int32_t ef_enabled;        /* 0 during the error-feedback freeze (App. "Freezing Error
+                                  Feedback"): u = Delta and e is neither read nor written */
+    int32_t divide_by_present; /* 0: average divides by R (Alg. 1); 1: by the payloads present */
+} sl_config;
+
+typedef struct sl_ctx sl_ctx;
+
+/* Build a context for a tensor table on the current CUDA device.  Allocates the device chunk
+ * table (32 bytes per chunk) -- the only allocation the library ever makes -- and synchronises.
+ * `tensors` is a host array.  Errors: INVALID_ARG, ALIGNMENT (offset % 4), UNSUPPORTED, CUDA. */
+sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t n_tensors,
+                    sl_ctx** out);
+sl_status sl_destroy(sl_ctx* ctx);
+
+/* Change beta / outer_lr / ef_enabled / divide_by_present / H between steps (k, R, chunking are
+ * fixed at creation).  Host-side only. */
+sl_status sl_set_hyper(sl_ctx* ctx, float beta, float outer_lr, int32_t ef_enabled,
+                       int32_t divide_by_present);
+
+/* Closed forms (host-side, no device work). */
+size_t sl_record_stride(int32_t k);                                   /* bytes of one chunk record */
+sl_status sl_payload_bytes(const sl_ctx* ctx, size_t* bytes_per_worker); /* 16 T + stride * chunks */
+sl_status sl_num_chunks(const sl_ctx* ctx, int64_t* chunks, int64_t* slots_per_worker);
+sl_status sl_flat_elems(const sl_ctx* ctx, int64_t* elems); /* max over tensors of offset + size */
+
+/* Scratch memory: selected (index, value) pairs and per-chunk partial sums for R workers.
+ * sl_workspace_bytes() gives the size sl_outer_step() needs (sl_compress() needs 1/R of it); the
+ * caller allocates it (256-byte aligned) and lends it with sl_set_workspace().  Contents need not
+ * be preserved between calls.  Calls that share a workspace must not overlap on the device. */
+sl_status sl_workspace_bytes(const sl_ctx* ctx, size_t* bytes);
+sl_status sl_set_workspace(sl_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* One worker's compression + error feedback (Alg. 1, green block; Eq. 2 lines 1-2).
+ *   theta_sync, theta_local : flat fp32, read only.
+ *   e       : flat fp32, updated in place to u - Dhat (untouched when ef_enabled == 0).
+ *   payload : sl_payload_bytes() bytes, fully overwritten.
+ * Errors: INVALID_ARG (NULL), ALIGNMENT, NOMEM (workspace), CUDA (launch failure). */
+sl_status sl_compress(sl_ctx* ctx, const float* theta_sync, const float* theta_local, float* e,
+                      uint8_t* payload, void* cuda_stream);
+
+/* Decode and average R payloads and apply the outer update (Alg. 1, orange block; Eq. 2 lines 3-4).
+ *   payloads : HOST array of R DEVICE pointers; NULL = that worker is absent.
+ *   theta_sync : updated in place: theta - alpha * (sum_r Dhat_r) / D, sum in fp32 with r
+ *   ascending, D = R or the number present.  Elements no worker selected are bit-unchanged.
+ * Payloads are trusted to be well formed (run sl_validate_payload on anything received from
+ * outside); an index beyond the chunk is ignored rather than written. */
+sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float* theta_sync,
+                             void* cuda_stream);
+
+/* The whole outer step for R resident workers: sl_compress for r = 0..R-1, then
+ * sl_aggregate_apply, with identical results, but free to share work between workers.
+ *   theta_local, e, payloads : HOST arrays of R DEVICE pointers.  theta_local entries may alias
+ *   each other; e and payload entries must not. */
+sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
+                        float* const* e, uint8_t* const* payloads, void* cuda_stream);
+
+/* Same step with the workers' parameters in HOST memory (pinned for full speed): theta_local_host
+ * is a host array of R host pointers; each is copied to the device staging buffer `dev_stage`
+ * (flat fp32, sl_flat_elems() elements, caller-owned) and compressed in turn; then the payloads are
+ * aggregated and, if theta_sync_host is not NULL, the updated theta_sync is copied back to it.
+ * Synchronises the stream before returning.  e, payloads and theta_sync stay resident on the
+ * device (Alg. 1 keeps e_r on its worker). */
+sl_status sl_outer_step_host(sl_ctx* ctx, float* theta_sync, const float* const* theta_local_host,
+                             float* dev_stage, float* const* e, uint8_t* const* payloads,
+                             float* theta_sync_host, void* cuda_stream);
+
+/* Check one payload before trusting it: every index < chunk length and strictly ascending over
+ * the used slots, unused slots and padding zero, table entries finite.  Writes SL_OK or
+ * SL_ERR_BAD_PAYLOAD to *dev_status (device int32); never traps. */
+sl_status sl_validate_payload(sl_ctx* ctx, const uint8_t* payload, int32_t* dev_status,
+                              void* cuda_stream);
+
+/* Per-(worker, tensor) quantiser statistics of the most recent compression, for logging:
+ * copies 8 floats per tensor (mu, sigma, 3 sigma, table[4], 0) for workspace worker slot
+ * `worker` into dev_out (device, 8 * n_tensors floats). */
+sl_status sl_read_stats(sl_ctx* ctx, int32_t worker, float* dev_out, void* cuda_stream);
+
+const char* sl_strerror(sl_status s);
+const char* sl_last_cuda_error(void); /* text of the last CUDA error seen by this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSELOCO_H */

@@ -1,0 +1,230 @@
+"""Thin ctypes binding over libsparseloco's C ABI (see include/sparseloco.h).
+
+Argument marshalling only: every step of the outer step runs in the CUDA kernels.  torch is
+used for device memory and streams.  Importing this module loads the shared library and raises
+if it is missing -- there is no CPU implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparseloco.so")
+
+EXPORTS = (
+    "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
+    "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
+    "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
+    "sl_last_cuda_error",
+)
+
+SL_OK = 0
+SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_BAD_PAYLOAD = 1, 2, 3, 4
+SL_ERR_CUDA, SL_ERR_NOMEM, SL_ERR_TOO_LARGE = 5, 6, 7
+
+
+class SlError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(msg)
+        self.status = status
+
+
+class _TensorDesc(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("offset", C.c_int64)]
+
+
+class _Config(C.Structure):
+    _fields_ = [("chunk_elems", C.c_int32), ("tile_dim", C.c_int32), ("k", C.c_int32),
+                ("R", C.c_int32), ("H", C.c_int32), ("beta", C.c_float), ("outer_lr", C.c_float),
+                ("quant_bits", C.c_int32), ("ef_enabled", C.c_int32),
+                ("divide_by_present", C.c_int32)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+            "(nvcc, sm_100a).  This package has no CPU fallback.")
+    L = C.CDLL(LIB_PATH)
+    P = C.c_void_p
+    L.sl_create.argtypes = [P, P, C.c_int32, C.POINTER(P)]
+    L.sl_destroy.argtypes = [P]
+    L.sl_set_hyper.argtypes = [P, C.c_float, C.c_float, C.c_int32, C.c_int32]
+    L.sl_record_stride.argtypes = [C.c_int32]
+    L.sl_record_stride.restype = C.c_size_t
+    L.sl_payload_bytes.argtypes = [P, C.POINTER(C.c_size_t)]
+    L.sl_num_chunks.argtypes = [P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    L.sl_flat_elems.argtypes = [P, C.POINTER(C.c_int64)]
+    L.sl_workspace_bytes.argtypes = [P, C.POINTER(C.c_size_t)]
+    L.sl_set_workspace.argtypes = [P, P, C.c_size_t]
+    L.sl_compress.argtypes = [P, P, P, P, P, P]
+    L.sl_aggregate_apply.argtypes = [P, P, P, P]
+    L.sl_outer_step.argtypes = [P, P, P, P, P, P]
+    L.sl_outer_step_host.argtypes = [P, P, P, P, P, P, P, P]
+    L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_read_stats.argtypes = [P, C.c_int32, P, P]
+    L.sl_strerror.argtypes = [C.c_int]
+    L.sl_strerror.restype = C.c_char_p
+    L.sl_last_cuda_error.restype = C.c_char_p
+    return L
+
+
+_L = _load()
+
+
+def _check(st: int) -> None:
+    if st != SL_OK:
+        msg = _L.sl_strerror(st).decode()
+        if st == SL_ERR_CUDA:
+            msg += ": " + _L.sl_last_cuda_error().decode()
+        raise SlError(st, f"libsparseloco: {msg} (status {st})")
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return t.data_ptr()
+
+
+def _ptr_array(ptrs: Sequence[Optional[int]]):
+    arr = (C.c_void_p * len(ptrs))()
+    for i, p in enumerate(ptrs):
+        arr[i] = p
+    return arr
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def record_stride(k: int) -> int:
+    return _L.sl_record_stride(k)
+
+
+class SparseLoCo:
+    """One context = one tensor table + hyper-parameters on the current CUDA device.
+
+    Method names mirror the C entry points: `compress`, `aggregate_apply`, `outer_step`,
+    `outer_step_host`, `validate_payload`.  All work is enqueued on torch's current stream.
+    """
+
+    def __init__(self, shapes: Sequence[Sequence[int]], offsets: Optional[Sequence[int]] = None, *,
+                 k: int, R: int, H: int = 1, beta: float = 0.95, outer_lr: float = 1.0,
+                 ef_enabled: bool = True, divide_by_present: bool = False, chunk_elems: int = 4096,
+                 tile_dim: int = 64, quant_bits: int = 2, alloc_workspace: bool = True):
+        n = len(shapes)
+        descs = (_TensorDesc * n)()
+        pos = 0
+        for j, sh in enumerate(shapes):
+            rows, cols = (1, sh[0]) if len(sh) == 1 else (sh[0], sh[1])
+            off = offsets[j] if offsets is not None else (pos + 3) // 4 * 4
+            descs[j] = _TensorDesc(rows, cols, off)
+            pos = off + rows * cols
+        cfg = _Config(chunk_elems, tile_dim, k, R, H, beta, outer_lr, quant_bits, int(ef_enabled),
+                      int(divide_by_present))
+        self._h = C.c_void_p()
+        self.k, self.R = k, R
+        self._beta, self._lr, self._ef, self._dbp = beta, outer_lr, int(ef_enabled), int(divide_by_present)
+        _check(_L.sl_create(C.byref(cfg), descs, n, C.byref(self._h)))
+        self.device = torch.device("cuda", torch.cuda.current_device())
+        self._ws = None
+        if alloc_workspace:
+            self._ws = torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
+            self.set_workspace(self._ws)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            _L.sl_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- closed forms
+    def payload_bytes(self) -> int:
+        v = C.c_size_t()
+        _check(_L.sl_payload_bytes(self._h, C.byref(v)))
+        return v.value
+
+    def num_chunks(self):
+        a, b = C.c_int64(), C.c_int64()
+        _check(_L.sl_num_chunks(self._h, C.byref(a), C.byref(b)))
+        return a.value, b.value
+
+    def flat_elems(self) -> int:
+        v = C.c_int64()
+        _check(_L.sl_flat_elems(self._h, C.byref(v)))
+        return v.value
+
+    def workspace_bytes(self) -> int:
+        v = C.c_size_t()
+        _check(_L.sl_workspace_bytes(self._h, C.byref(v)))
+        return v.value
+
+    def set_workspace(self, ws: Optional[torch.Tensor]) -> None:
+        self._ws = ws
+        if ws is None:
+            _check(_L.sl_set_workspace(self._h, None, 0))
+        else:
+            _check(_L.sl_set_workspace(self._h, _dev_ptr(ws), ws.numel() * ws.element_size()))
+
+    def set_hyper(self, beta=None, outer_lr=None, ef_enabled=None, divide_by_present=None) -> None:
+        if beta is not None:
+            self._beta = beta
+        if outer_lr is not None:
+            self._lr = outer_lr
+        if ef_enabled is not None:
+            self._ef = int(ef_enabled)
+        if divide_by_present is not None:
+            self._dbp = int(divide_by_present)
+        _check(_L.sl_set_hyper(self._h, self._beta, self._lr, self._ef, self._dbp))
+
+    # -- the path
+    def compress(self, theta_sync, theta_local, e, payload) -> None:
+        _check(_L.sl_compress(self._h, _dev_ptr(theta_sync, torch.float32), _dev_ptr(theta_local, torch.float32),
+                              _dev_ptr(e, torch.float32), _dev_ptr(payload, torch.uint8), _stream()))
+
+    def aggregate_apply(self, payloads: List[Optional[torch.Tensor]], theta_sync) -> None:
+        arr = _ptr_array([_dev_ptr(p, torch.uint8) for p in payloads])
+        _check(_L.sl_aggregate_apply(self._h, arr, _dev_ptr(theta_sync, torch.float32), _stream()))
+
+    def outer_step(self, theta_sync, theta_local: List[torch.Tensor], e: Optional[List[torch.Tensor]],
+                   payloads: List[torch.Tensor]) -> None:
+        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
+        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        pa = _ptr_array([_dev_ptr(t, torch.uint8) for t in payloads])
+        _check(_L.sl_outer_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, ea, pa, _stream()))
+
+    def outer_step_host(self, theta_sync, theta_local_host: List[torch.Tensor], dev_stage,
+                        e: Optional[List[torch.Tensor]], payloads: List[torch.Tensor],
+                        theta_sync_host: Optional[torch.Tensor] = None) -> None:
+        for t in theta_local_host:
+            assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
+        tl = _ptr_array([t.data_ptr() for t in theta_local_host])
+        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        pa = _ptr_array([_dev_ptr(t, torch.uint8) for t in payloads])
+        hp = None
+        if theta_sync_host is not None:
+            assert not theta_sync_host.is_cuda and theta_sync_host.is_contiguous()
+            hp = theta_sync_host.data_ptr()
+        _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
+                                     _dev_ptr(dev_stage, torch.float32), ea, pa, hp, _stream()))
+
+    def validate_payload(self, payload, status: torch.Tensor) -> None:
+        assert status.dtype == torch.int32
+        _check(_L.sl_validate_payload(self._h, _dev_ptr(payload, torch.uint8), _dev_ptr(status), _stream()))
+
+    def read_stats(self, worker: int, n_tensors: int) -> torch.Tensor:
+        out = torch.empty(n_tensors * 8, dtype=torch.float32, device=self.device)
+        _check(_L.sl_read_stats(self._h, worker, _dev_ptr(out), _stream()))
+        return out.view(n_tensors, 8)

@@ -1,0 +1,1075 @@
+// SparseLoCo outer step for sm_100a: kernels and the C ABI declared in include/sparseloco.h.
+//
+// Kernel sequence of one outer step (all on the caller's stream, no host synchronisation):
+//   ef_topk_kernel         pseudo-gradient + error feedback + chunk-wise Top-k     (Eq. 2 line 1, Sec. 3.3)
+//   chunk_sum_kernel       per-chunk fp64 sum of the selected values               (Sec. 4 quantiser: mean)
+//   tensor_reduce_kernel<0>  chunk-ordered fp64 sum per (worker, tensor) -> mu
+//   chunk_sum_kernel<1>    per-chunk fp64 sum of squared centred values            (sigma)
+//   tensor_reduce_kernel<1>  -> sigma, bin edge 3 sigma
+//   chunk_bins_kernel      per-chunk per-bin sums and counts                       (centroids)
+//   tensor_reduce_kernel<2>  -> 4-entry table, written to the payload header
+//   pack_fix_kernel        codes, 12-bit index + 2-bit code packing, e = u - Dhat   (Eq. 2 line 2)
+//   decode_avg_apply_kernel  decode R payloads, sum, theta -= alpha/D * sum         (Eq. 2 lines 3-4)
+//
+// Everything is HBM-bound streaming except the per-chunk selection, which works on registers and
+// shared memory.  No tensor cores: nothing here is a dense contraction.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "sparseloco.h"
+
+namespace {
+
+constexpr int kChunk = 4096;
+constexpr int kTile = 64;
+constexpr int kThreads = 256;          // threads per CTA of the chunk kernels
+constexpr int kPerThread = kChunk / kThreads;  // 16 elements = 4 x float4
+constexpr int kMaxR = 64;
+constexpr int kMaxK = 256;
+constexpr int kCandCap = 1024;         // candidate list capacity of the selection
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+thread_local char g_cuda_err[256] = "";
+
+// One chunk of one tensor: where its elements live in the flat buffers.
+struct ChunkDesc {
+    long long base;    // element offset of in-chunk index 0
+    int row_stride;    // elements between block rows (2-D blocks), 0 for flat runs
+    int len;           // elements in the chunk (4096, or the short tail of a flat tensor)
+    int tensor;        // owning tensor
+    int chunk_in_tensor;
+    long long rec_off; // byte offset of this chunk's record inside a payload
+};
+static_assert(sizeof(ChunkDesc) == 32, "ChunkDesc layout");
+
+struct TensorInfo {
+    long long first_chunk;
+    long long n_chunks;
+    long long n_slots;  // sum over chunks of min(k, len)
+};
+
+struct TStat {  // per (worker, tensor)
+    float mu, sigma, t3;
+    float lut[4];
+    float pad;
+};
+static_assert(sizeof(TStat) == 32, "TStat layout");
+
+struct WorkerPtrs {
+    const float* theta_local[kMaxR];
+    float* e[kMaxR];
+    uint8_t* payload[kMaxR];
+};
+
+struct PayloadPtrs {
+    const uint8_t* p[kMaxR];
+};
+
+struct Workspace {  // device arrays, dimensioned [workers][chunks]...
+    float* val;          // [W][G][kp]
+    uint16_t* idx;       // [W][G][kp]
+    double* psum;        // [W][G]
+    double* pbin;        // [W][G][4]
+    unsigned* pcnt;      // [W][G][4]
+    TStat* tstat;        // [W][T]
+};
+
+__host__ __device__ constexpr int record_index_bytes(int k) { return (12 * k + 7) / 8; }
+__host__ __device__ constexpr int record_stride(int k) {
+    return (record_index_bytes(k) + (2 * k + 7) / 8 + 15) / 16 * 16;
+}
+
+// Element offset (relative to ChunkDesc::base) of in-chunk index p.
+__device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
+    return row_stride ? (long long)(p >> 6) * row_stride + (p & 63) : (long long)p;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Selection: the keff largest of 4096 composites (magnitude, then lower index), exact.
+//
+// composite = key << 13 | (4095 - p) << 1 | sign, key = float bits without the sign.  All
+// composites of a chunk are distinct, so "the keff largest composites" is exactly the Top-k with
+// the lowest-index tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3.
+//
+// 1. every lane takes the maximum key of its 16 values; every warp takes the ceil(keff/8)-th
+//    largest of its 32 lane maxima; T = the minimum over the 8 warps.  At least keff values have
+//    key >= T, so nothing below T can be selected.
+// 2. values with key >= T (about 2 k of them on bell-shaped data) go to a shared candidate list.
+// 3. each candidate counts the candidates above it; rank < keff means selected.
+// 4. selected bits are set in a 4096-bit map; a prefix popcount over the map gives every selected
+//    entry its slot in ascending index order.
+// If the list overflows (heavy ties, constant chunks) an exact bitwise search over all 4096
+// composites finds the keff-th largest instead.
+// ------------------------------------------------------------------------------------------------
+
+struct SelectSmem {
+    unsigned long long cand[kCandCap];
+    unsigned bitmap[128];
+    unsigned prefix[128];
+    unsigned warp_t[8];
+    unsigned warp_cnt[2][8];
+    unsigned count;
+};
+
+__device__ __forceinline__ unsigned long long make_composite(unsigned bits, int p) {
+    unsigned key = bits & 0x7FFFFFFFu;
+    return ((unsigned long long)key << 13) | ((unsigned long long)(4095 - p) << 1) | (bits >> 31);
+}
+__device__ __forceinline__ int composite_index(unsigned long long c) { return 4095 - (int)((c >> 1) & 0xFFF); }
+__device__ __forceinline__ unsigned composite_bits(unsigned long long c) {
+    return (unsigned)(c >> 13) | ((unsigned)(c & 1ull) << 31);
+}
+
+__device__ __forceinline__ int owned_index(int tid, int q) { return 1024 * (q >> 2) + 4 * tid + (q & 3); }
+
+// Emits the selected (index, value) pairs of the chunk to out_idx / out_val in ascending index
+// order.  `ub` = the thread's 16 value bit patterns; entries with owned index >= len are padding.
+__device__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff, SelectSmem& sm,
+                            uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // -- 1. threshold
+    unsigned m = 0;
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) m = max(m, ub[q] & 0x7FFFFFFFu);
+    {
+        const int rounds = (keff + 7) >> 3;  // <= 32
+        unsigned cur = m, tw = 0;
+        bool alive = true;
+        for (int i = 0; i < rounds; ++i) {
+            tw = __reduce_max_sync(kFull, alive ? cur : 0u);
+            unsigned holders = __ballot_sync(kFull, alive && cur == tw);
+            if (holders == 0) break;  // only zeros remain: tw == 0
+            if (lane == __ffs(holders) - 1) alive = false;
+        }
+        if (lane == 0) sm.warp_t[warp] = tw;
+    }
+    if (tid < 128) sm.bitmap[tid] = 0;
+    if (tid == 0) sm.count = 0;
+    __syncthreads();
+    unsigned T = sm.warp_t[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) T = min(T, sm.warp_t[w]);
+
+    // -- 2. candidates
+#pragma unroll
+    for (int q = 0; q < kPerThread; ++q) {
+        const int p = owned_index(tid, q);
+        if ((ub[q] & 0x7FFFFFFFu) >= T && p < len) {
+            unsigned pos = atomicAdd(&sm.count, 1u);
+            if (pos < kCandCap) sm.cand[pos] = make_composite(ub[q], p);
+        }
+    }
+    __syncthreads();
+    unsigned M = sm.count;
+
+    if (M > kCandCap) {
+        // -- exact fallback: bitwise search for the keff-th largest composite over all elements
+        unsigned long long res = 0;
+        const bool any = __syncthreads_or(m != 0);
+        if (any) {
+            int buf = 0;
+            for (int bit = 43; bit >= 0; --bit) {
+                const unsigned long long trial = res | (1ull << bit);
+                unsigned c = 0;
+#pragma unroll
+                for (int q = 0; q < kPerThread; ++q) {
+                    const int p = owned_index(tid, q);
+                    c += (p < len && make_composite(ub[q], p) >= trial) ? 1u : 0u;
+                }
+                c = __reduce_add_sync(kFull, c);
+                if (lane == 0) sm.warp_cnt[buf][warp] = c;
+                __syncthreads();
+                unsigned tot = 0;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) tot += sm.warp_cnt[buf][w];
+                if (tot >= (unsigned)keff) res = trial;
+                buf ^= 1;
+            }
+        } else {
+            // all magnitudes are zero: the first keff indices win every tie
+            res = make_composite(0u, keff - 1) & ~1ull;
+        }
+        if (tid == 0) sm.count = 0;
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int p = owned_index(tid, q);
+            if (p < len) {
+                const unsigned long long c = make_composite(ub[q], p);
+                if (c >= res) {
+                    unsigned pos = atomicAdd(&sm.count, 1u);
+                    if (pos < kCandCap) sm.cand[pos] = c;
+                }
+            }
+        }
+        __syncthreads();
+        M = sm.count;  // == keff
+    }
+
+    // -- 3. rank among candidates (M <= kCandCap: up to 4 candidates per thread)
+    unsigned long long mine[kCandCap / kThreads];
+    unsigned sel_mask = 0;
+#pragma unroll
+    for (int s = 0; s < kCandCap / kThreads; ++s) {
+        const unsigned i = tid + s * kThreads;
+        if (i < M) {
+            const unsigned long long ci = sm.cand[i];
+            mine[s] = ci;
+            unsigned above = 0;
+            for (unsigned j = 0; j < M; ++j) above += (sm.cand[j] > ci) ? 1u : 0u;
+            if (above < (unsigned)keff) {
+                sel_mask |= 1u << s;
+                const int p = composite_index(ci);
+                atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
+            }
+        }
+    }
+    __syncthreads();
+
+    // -- 4. slots from a prefix popcount over the bitmap
+    if (warp == 0) {
+        unsigned w0 = sm.bitmap[4 * lane], w1 = sm.bitmap[4 * lane + 1], w2 = sm.bitmap[4 * lane + 2],
+                 w3 = sm.bitmap[4 * lane + 3];
+        unsigned c0 = __popc(w0), c1 = __popc(w1), c2 = __popc(w2), c3 = __popc(w3);
+        unsigned tot = c0 + c1 + c2 + c3, inc = tot;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned o = __shfl_up_sync(kFull, inc, d);
+            if (lane >= d) inc += o;
+        }
+        unsigned ex = inc - tot;
+        sm.prefix[4 * lane] = ex;
+        sm.prefix[4 * lane + 1] = ex + c0;
+        sm.prefix[4 * lane + 2] = ex + c0 + c1;
+        sm.prefix[4 * lane + 3] = ex + c0 + c1 + c2;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int s = 0; s < kCandCap / kThreads; ++s) {
+        if (sel_mask & (1u << s)) {
+            const int p = composite_index(mine[s]);
+            const unsigned slot = sm.prefix[p >> 5] + __popc(sm.bitmap[p >> 5] & ((1u << (p & 31)) - 1u));
+            if (slot < (unsigned)keff) {
+                out_idx[slot] = (uint16_t)p;
+                out_val[slot] = __uint_as_float(composite_bits(mine[s]));
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel 1: u = beta e + (theta - theta_r) written into e, chunk-wise Top-k of u into staging.
+// One CTA per (chunk, worker); workers of a chunk are adjacent in the grid so that the chunk of
+// theta_sync is fetched from HBM once and served to the other workers from L2.
+// ------------------------------------------------------------------------------------------------
+template <bool EF>
+__global__ void __launch_bounds__(kThreads)
+ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp,
+               float beta, const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
+    __shared__ SelectSmem sm;
+    const long long b = blockIdx.x;
+    const long long g = b / n_workers;
+    const int r = (int)(b - g * n_workers);
+    const ChunkDesc cd = chunks[g];
+    const int tid = threadIdx.x;
+    const float* __restrict__ ts = theta_sync + cd.base;
+    const float* __restrict__ tl = ptrs.theta_local[r] + cd.base;
+    float* __restrict__ er = EF ? ptrs.e[r] + cd.base : nullptr;
+
+    unsigned ub[kPerThread];
+    if (cd.len == kChunk) {
+        long long off[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = 1024 * i + 4 * tid;
+            off[i] = chunk_elem_offset(cd.row_stride, p);
+        }
+        float4 a[4], l[4], ev[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = __ldg(reinterpret_cast<const float4*>(ts + off[i]));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) l[i] = __ldcs(reinterpret_cast<const float4*>(tl + off[i]));
+        if (EF) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ev[i] = __ldcs(reinterpret_cast<const float4*>(er + off[i]));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 u;
+            u.x = __fsub_rn(a[i].x, l[i].x);
+            u.y = __fsub_rn(a[i].y, l[i].y);
+            u.z = __fsub_rn(a[i].z, l[i].z);
+            u.w = __fsub_rn(a[i].w, l[i].w);
+            if (EF) {
+                u.x = __fmaf_rn(beta, ev[i].x, u.x);
+                u.y = __fmaf_rn(beta, ev[i].y, u.y);
+                u.z = __fmaf_rn(beta, ev[i].z, u.z);
+                u.w = __fmaf_rn(beta, ev[i].w, u.w);
+                *reinterpret_cast<float4*>(er + off[i]) = u;
+            }
+            ub[4 * i + 0] = __float_as_uint(u.x);
+            ub[4 * i + 1] = __float_as_uint(u.y);
+            ub[4 * i + 2] = __float_as_uint(u.z);
+            ub[4 * i + 3] = __float_as_uint(u.w);
+        }
+    } else {  // short tail of a flat tensor: element-wise with bounds
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int p = owned_index(tid, q);
+            float u = 0.0f;
+            if (p < cd.len) {
+                u = __fsub_rn(ts[p], tl[p]);
+                if (EF) {
+                    u = __fmaf_rn(beta, er[p], u);
+                    er[p] = u;
+                }
+            }
+            ub[q] = __float_as_uint(u);
+        }
+    }
+
+    const int keff = min(k, cd.len);
+    const long long slot_base = ((long long)r * n_chunks + g) * kp;
+    select_topk(ub, cd.len, keff, sm, ws.idx + slot_base, ws.val + slot_base);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Quantiser statistics (Sec. 4).  The summation order is part of the definition of the payload
+// bits: fp64, slot by slot inside a chunk, then chunk by chunk inside the tensor.
+// ------------------------------------------------------------------------------------------------
+
+// mode 0: sum of values; mode 1: sum of squared fp32-centred values.  One thread per (worker, chunk).
+template <int MODE>
+__global__ void __launch_bounds__(128)
+chunk_sum_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
+                 int k, int kp, Workspace ws) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_chunks * n_workers) return;
+    const long long r = i / n_chunks, g = i - r * n_chunks;
+    const int len = chunks[g].len, keff = min(k, len);
+    const float* __restrict__ v = ws.val + i * kp;
+    float mu = 0.0f;
+    if (MODE == 1) mu = ws.tstat[r * n_tensors + chunks[g].tensor].mu;
+    double acc = 0.0;
+    for (int s0 = 0; s0 < keff; s0 += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(v + s0);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (s0 + j < keff) {
+                if (MODE == 0) {
+                    acc += (double)xs[j];
+                } else {
+                    const double d = (double)__fsub_rn(xs[j], mu);
+                    acc += d * d;  // d*d is exact in fp64, so fusing or not gives the same sum
+                }
+            }
+        }
+    }
+    ws.psum[i] = acc;
+}
+
+// Per-bin sums and counts of one chunk.  codes: (cen >= -t) + (cen >= 0) + (cen >= t).
+__device__ __forceinline__ int quant_code(float v, float mu, float t3) {
+    const float cen = __fsub_rn(v, mu);
+    return (cen >= -t3 ? 1 : 0) + (cen >= 0.0f ? 1 : 0) + (cen >= t3 ? 1 : 0);
+}
+
+__global__ void __launch_bounds__(128)
+chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
+                  int k, int kp, Workspace ws) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_chunks * n_workers) return;
+    const long long r = i / n_chunks, g = i - r * n_chunks;
+    const int len = chunks[g].len, keff = min(k, len);
+    const float* __restrict__ v = ws.val + i * kp;
+    const TStat st = ws.tstat[r * n_tensors + chunks[g].tensor];
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    unsigned n0 = 0, n1 = 0, n2 = 0, n3 = 0;
+    for (int sb = 0; sb < keff; sb += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(v + sb);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (sb + j < keff) {
+                const int c = quant_code(xs[j], st.mu, st.t3);
+                const double d = (double)xs[j];
+                // add only to the value's own bin (adding +0 elsewhere could flip a -0 sum)
+                if (c == 0) { s0 += d; ++n0; }
+                else if (c == 1) { s1 += d; ++n1; }
+                else if (c == 2) { s2 += d; ++n2; }
+                else { s3 += d; ++n3; }
+            }
+        }
+    }
+    double* pb = ws.pbin + i * 4;
+    pb[0] = s0; pb[1] = s1; pb[2] = s2; pb[3] = s3;
+    unsigned* pc = ws.pcnt + i * 4;
+    pc[0] = n0; pc[1] = n1; pc[2] = n2; pc[3] = n3;
+}
+
+// One warp per (worker, tensor): left-to-right fp64 sum of the tensor's chunk partials.
+// STAGE 0: psum -> mu.  STAGE 1: psum -> sigma, 3 sigma.  STAGE 2: pbin/pcnt -> table (+ payload header).
+template <int STAGE>
+__global__ void __launch_bounds__(128)
+tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, int n_workers, int n_tensors,
+                     Workspace ws, WorkerPtrs ptrs) {
+    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= (long long)n_workers * n_tensors) return;
+    const int r = (int)(w / n_tensors), t = (int)(w - (long long)r * n_tensors);
+    const TensorInfo ti = tinfo[t];
+    const long long first = (long long)r * n_chunks + ti.first_chunk;
+    TStat* st = ws.tstat + (long long)r * n_tensors + t;
+    const double n = (double)ti.n_slots;
+
+    if (STAGE < 2) {
+        double acc = 0.0;
+        for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32) {
+            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
+            const double x = lane < cnt ? ws.psum[first + c0 + lane] : 0.0;
+            for (int l = 0; l < cnt; ++l) acc += __shfl_sync(kFull, x, l);
+        }
+        if (lane == 0) {
+            if (STAGE == 0) {
+                st->mu = (float)(acc / n);
+            } else {
+                const float sigma = (float)sqrt(acc / n);
+                st->sigma = sigma;
+                st->t3 = __fmul_rn(3.0f, sigma);
+            }
+        }
+    } else {
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+        unsigned long long cn[4] = {0, 0, 0, 0};
+        for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32) {
+            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
+            double x0 = 0.0, x1 = 0.0, x2 = 0.0, x3 = 0.0;
+            if (lane < cnt) {
+                const double* pb = ws.pbin + (first + c0 + lane) * 4;
+                x0 = pb[0]; x1 = pb[1]; x2 = pb[2]; x3 = pb[3];
+                const unsigned* pc = ws.pcnt + (first + c0 + lane) * 4;
+                cn[0] += pc[0]; cn[1] += pc[1]; cn[2] += pc[2]; cn[3] += pc[3];
+            }
+            for (int l = 0; l < cnt; ++l) {
+                a0 += __shfl_sync(kFull, x0, l);
+                a1 += __shfl_sync(kFull, x1, l);
+                a2 += __shfl_sync(kFull, x2, l);
+                a3 += __shfl_sync(kFull, x3, l);
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) cn[b] += __shfl_xor_sync(kFull, cn[b], d);
+        }
+        if (lane == 0) {
+            float lut[4];
+            lut[0] = cn[0] ? (float)(a0 / (double)cn[0]) : 0.0f;
+            lut[1] = cn[1] ? (float)(a1 / (double)cn[1]) : 0.0f;
+            lut[2] = cn[2] ? (float)(a2 / (double)cn[2]) : 0.0f;
+            lut[3] = cn[3] ? (float)(a3 / (double)cn[3]) : 0.0f;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) st->lut[b] = lut[b];
+            st->pad = 0.0f;
+            float4* hdr = reinterpret_cast<float4*>(ptrs.payload[r] + 16ll * t);
+            *hdr = make_float4(lut[0], lut[1], lut[2], lut[3]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pack + error-feedback subtract.  One warp per (worker, chunk): codes from (mu, 3 sigma), 12-bit
+// indices and 2-bit codes OR-ed into a shared-memory record, record written as 16-byte vectors,
+// e[index] = value - table[code] at the selected positions (Eq. 2 line 2).
+// ------------------------------------------------------------------------------------------------
+template <bool EF>
+__global__ void __launch_bounds__(128)
+pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
+                int k, int kp, Workspace ws, WorkerPtrs ptrs) {
+    __shared__ __align__(16) unsigned rec[4][(record_stride(kMaxK) / 4) + 4];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long i = (long long)blockIdx.x * 4 + warp;
+    if (i >= n_chunks * n_workers) return;
+    const long long g = i / n_workers;
+    const int r = (int)(i - g * n_workers);
+    const ChunkDesc cd = chunks[g];
+    const int keff = min(k, cd.len);
+    const int stride = record_stride(k), words = stride / 4;
+    const int code_word0 = record_index_bytes(k);  // byte offset of the code block
+    const long long slot_base = ((long long)r * n_chunks + g) * kp;
+    const TStat st = ws.tstat[(long long)r * n_tensors + cd.tensor];
+
+    for (int w = lane; w < words; w += 32) rec[warp][w] = 0;
+    __syncwarp();
+    for (int s = lane; s < keff; s += 32) {
+        const unsigned p = ws.idx[slot_base + s];
+        const float v = ws.val[slot_base + s];
+        const int c = quant_code(v, st.mu, st.t3);
+        const int bit = 12 * s;
+        atomicOr(&rec[warp][bit >> 5], p << (bit & 31));
+        if ((bit & 31) > 20) atomicOr(&rec[warp][(bit >> 5) + 1], p >> (32 - (bit & 31)));
+        const int cbit = code_word0 * 8 + 2 * s;
+        atomicOr(&rec[warp][cbit >> 5], (unsigned)c << (cbit & 31));
+        if (EF && p < (unsigned)cd.len) {
+            float* er = ptrs.e[r] + cd.base + chunk_elem_offset(cd.row_stride, (int)p);
+            *er = __fsub_rn(v, st.lut[c]);
+        }
+    }
+    __syncwarp();
+    uint4* dst = reinterpret_cast<uint4*>(ptrs.payload[r] + cd.rec_off);
+    const uint4* src = reinterpret_cast<const uint4*>(rec[warp]);
+    for (int w = lane; w < stride / 16; w += 32) dst[w] = src[w];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Decode + average + outer update.  One CTA per chunk: all present workers' records are copied to
+// shared memory, warp 0 adds table[code] into a 4096-float shared tile worker by worker (fixed
+// order => reproducible bits), then every thread applies theta = fma(-alpha/D, sum, theta).
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned get12(const unsigned* rec, int s) {
+    const int bit = 12 * s;
+    return __funnelshift_r(rec[bit >> 5], rec[(bit >> 5) + 1], bit & 31) & 0xFFFu;
+}
+__device__ __forceinline__ unsigned get2(const unsigned* rec, int code_byte0, int s) {
+    const int bit = code_byte0 * 8 + 2 * s;
+    return (rec[bit >> 5] >> (bit & 31)) & 3u;
+}
+
+__global__ void __launch_bounds__(kThreads)
+decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale,
+                        PayloadPtrs pl, float* __restrict__ theta_sync) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    float* acc = reinterpret_cast<float*>(dyn);                       // 4096 floats
+    float* luts = acc + kChunk;                                       // n_workers x 4
+    unsigned* recs = reinterpret_cast<unsigned*>(luts + 4 * n_workers);  // n_workers x (stride + 16) bytes
+    const int stride = record_stride(k), rwords = stride / 4 + 4;
+    const int tid = threadIdx.x;
+    const ChunkDesc cd = chunks[blockIdx.x];
+    const int keff = min(k, cd.len);
+    float* __restrict__ th = theta_sync + cd.base;
+
+    // theta loads first (in flight while the records are staged)
+    float4 a[4];
+    long long off[4];
+    const bool full = cd.len == kChunk;
+    if (full) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            off[i] = chunk_elem_offset(cd.row_stride, 1024 * i + 4 * tid);
+            a[i] = *reinterpret_cast<const float4*>(th + off[i]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int vec_per_rec = stride / 16;
+    for (int v = tid; v < n_workers * vec_per_rec; v += kThreads) {
+        const int r = v / vec_per_rec, w = v - r * vec_per_rec;
+        if (pl.p[r]) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4*>(pl.p[r] + cd.rec_off) + w);
+            *reinterpret_cast<uint4*>(recs + r * rwords + 4 * w) = x;
+        }
+    }
+    for (int v = tid; v < n_workers; v += kThreads) {
+        if (pl.p[v]) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(pl.p[v] + 16ll * cd.tensor));
+            *reinterpret_cast<float4*>(luts + 4 * v) = x;
+        }
+        recs[v * rwords + stride / 4] = 0;  // word read past the index block by get12
+    }
+    __syncthreads();
+    if (tid < 32) {
+        const int code_byte0 = record_index_bytes(k);
+        for (int r = 0; r < n_workers; ++r) {
+            if (!pl.p[r]) continue;
+            const unsigned* rec = recs + r * rwords;
+            for (int s = tid; s < keff; s += 32) {
+                const unsigned p = get12(rec, s);
+                const unsigned c = get2(rec, code_byte0, s);
+                if (p < (unsigned)cd.len) acc[p] += luts[4 * r + c];
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    if (full) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 s = *reinterpret_cast<const float4*>(acc + 1024 * i + 4 * tid);
+            float4 o;
+            o.x = __fmaf_rn(scale, s.x, a[i].x);
+            o.y = __fmaf_rn(scale, s.y, a[i].y);
+            o.z = __fmaf_rn(scale, s.z, a[i].z);
+            o.w = __fmaf_rn(scale, s.w, a[i].w);
+            *reinterpret_cast<float4*>(th + off[i]) = o;
+        }
+    } else {
+        for (int p = tid; p < cd.len; p += kThreads) th[p] = __fmaf_rn(scale, acc[p], th[p]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Payload validation: never traps, reports through a device status word.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+validate_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_tensors, int k,
+                const uint8_t* __restrict__ payload, int* __restrict__ status) {
+    const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    bool bad = false;
+    if (g < n_tensors) {
+        const float* lut = reinterpret_cast<const float*>(payload + 16 * g);
+        for (int b = 0; b < 4; ++b) bad |= !isfinite(lut[b]);
+    }
+    if (g < n_chunks) {
+        const ChunkDesc cd = chunks[g];
+        const int keff = min(k, cd.len), stride = record_stride(k), ib = record_index_bytes(k);
+        const uint8_t* rec = payload + cd.rec_off;
+        int prev = -1;
+        for (int s = 0; s < k; ++s) {
+            const int bit = 12 * s, by = bit >> 3;
+            const unsigned two = rec[by] | ((unsigned)rec[by + 1] << 8);
+            const int p = (two >> (bit & 7)) & 0xFFF;
+            const int cbit = 2 * s;
+            const int c = (rec[ib + (cbit >> 3)] >> (cbit & 7)) & 3;
+            if (s < keff) {
+                bad |= p >= cd.len || p <= prev;
+                prev = p;
+            } else {
+                bad |= p != 0 || c != 0;
+            }
+        }
+        // padding: bits after the last index, bits after the last code
+        if ((12 * k) & 7) bad |= (rec[ib - 1] >> ((12 * k) & 7)) != 0;
+        const int code_bits = 2 * k, cb_full = code_bits >> 3;
+        if (code_bits & 7) bad |= (rec[ib + cb_full] >> (code_bits & 7)) != 0;
+        for (int by = ib + ((code_bits + 7) >> 3); by < stride; ++by) bad |= rec[by] != 0;
+    }
+    if (bad) atomicExch(status, (int)SL_ERR_BAD_PAYLOAD);
+}
+
+__global__ void set_status_kernel(int* status, int v) { *status = v; }
+
+__global__ void copy_stats_kernel(const TStat* __restrict__ src, int n, float* __restrict__ dst) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n * 8) dst[i] = reinterpret_cast<const float*>(src)[i];
+}
+
+}  // namespace
+
+// ================================================================================================
+// Host side
+// ================================================================================================
+
+struct sl_ctx {
+    sl_config cfg;
+    int device;
+    int n_tensors;
+    long long n_chunks;
+    long long n_slots;
+    long long flat_elems;
+    int kp;
+    std::vector<sl_tensor_desc> tensors;
+    ChunkDesc* d_chunks;
+    TensorInfo* d_tinfo;
+    void* ws_ptr;
+    size_t ws_bytes;
+    int last_workers;  // worker count the workspace was last laid out for
+};
+
+namespace {
+
+sl_status cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return SL_ERR_CUDA;
+}
+#define SL_CUDA(call)                                      \
+    do {                                                   \
+        cudaError_t e_ = (call);                           \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t workspace_bytes_for(const sl_ctx* c, int workers) {
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks;
+    return up256(WG * c->kp * sizeof(float)) + up256(WG * c->kp * sizeof(uint16_t)) +
+           up256(WG * sizeof(double)) + up256(WG * 4 * sizeof(double)) + up256(WG * 4 * sizeof(unsigned)) +
+           up256((size_t)workers * c->n_tensors * sizeof(TStat));
+}
+
+Workspace carve(const sl_ctx* c, int workers) {
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks;
+    char* p = static_cast<char*>(c->ws_ptr);
+    Workspace w;
+    w.val = reinterpret_cast<float*>(p);        p += up256(WG * c->kp * sizeof(float));
+    w.idx = reinterpret_cast<uint16_t*>(p);     p += up256(WG * c->kp * sizeof(uint16_t));
+    w.psum = reinterpret_cast<double*>(p);      p += up256(WG * sizeof(double));
+    w.pbin = reinterpret_cast<double*>(p);      p += up256(WG * 4 * sizeof(double));
+    w.pcnt = reinterpret_cast<unsigned*>(p);    p += up256(WG * 4 * sizeof(unsigned));
+    w.tstat = reinterpret_cast<TStat*>(p);
+    return w;
+}
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+unsigned blocks_for(long long items, int per_block) { return (unsigned)((items + per_block - 1) / per_block); }
+
+// Compression of `workers` workers whose pointers are in `ptrs` (kernels 1-8).
+sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const WorkerPtrs& ptrs,
+                          cudaStream_t st) {
+    if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, workers)) return SL_ERR_NOMEM;
+    const Workspace ws = carve(c, workers);
+    c->last_workers = workers;
+    const long long G = c->n_chunks, WG = G * workers;
+    const int k = c->cfg.k, kp = c->kp, T = c->n_tensors;
+    if (WG > 0x7FFFFFFFll) return SL_ERR_TOO_LARGE;
+    const bool ef = c->cfg.ef_enabled != 0;
+
+    if (ef)
+        ef_topk_kernel<true><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                theta_sync, ptrs, ws);
+    else
+        ef_topk_kernel<false><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                 theta_sync, ptrs, ws);
+    const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T * 32, 128);
+    chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    tensor_reduce_kernel<0><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    chunk_sum_kernel<1><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    tensor_reduce_kernel<1><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    chunk_bins_kernel<<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    if (ef)
+        pack_fix_kernel<true><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    else
+        pack_fix_kernel<false><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* theta_sync, cudaStream_t st) {
+    if (present == 0) return SL_OK;
+    const int R = c->cfg.R;
+    const double D = c->cfg.divide_by_present ? (double)present : (double)R;
+    const float scale = (float)(-(double)c->cfg.outer_lr / D);
+    const int stride = record_stride(c->cfg.k);
+    const size_t smem = (size_t)kChunk * 4 + (size_t)R * 16 + (size_t)R * (stride + 16);
+    if (smem > 48 * 1024) {
+        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem));
+    }
+    decode_avg_apply_kernel<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl,
+                                                                          theta_sync);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = prev == dev || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* sl_strerror(sl_status s) {
+    switch (s) {
+        case SL_OK: return "ok";
+        case SL_ERR_INVALID_ARG: return "invalid argument";
+        case SL_ERR_ALIGNMENT: return "pointer or offset not 16-byte aligned";
+        case SL_ERR_UNSUPPORTED: return "configuration not supported by this build";
+        case SL_ERR_BAD_PAYLOAD: return "malformed payload";
+        case SL_ERR_CUDA: return "CUDA error";
+        case SL_ERR_NOMEM: return "workspace missing or too small";
+        case SL_ERR_TOO_LARGE: return "problem exceeds a built-in capacity";
+    }
+    return "unknown status";
+}
+
+const char* sl_last_cuda_error(void) { return g_cuda_err; }
+
+size_t sl_record_stride(int32_t k) { return k < 1 ? 0 : (size_t)record_stride(k); }
+
+sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t n_tensors, sl_ctx** out) {
+    if (!cfg || !tensors || !out || n_tensors < 1) return SL_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->k < 1 || cfg->R < 1 || cfg->H < 1) return SL_ERR_INVALID_ARG;
+    if (!(cfg->beta >= 0.0f && cfg->beta <= 1.0f) || !isfinite(cfg->outer_lr)) return SL_ERR_INVALID_ARG;
+    if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile || cfg->quant_bits != 2) return SL_ERR_UNSUPPORTED;
+    if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
+
+    sl_ctx* c = new (std::nothrow) sl_ctx();
+    if (!c) return SL_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->n_tensors = n_tensors;
+    c->kp = (cfg->k + 3) / 4 * 4;
+    c->d_chunks = nullptr;
+    c->d_tinfo = nullptr;
+    c->ws_ptr = nullptr;
+    c->ws_bytes = 0;
+    c->last_workers = cfg->R;
+    c->tensors.assign(tensors, tensors + n_tensors);
+
+    const int stride = record_stride(cfg->k);
+    std::vector<ChunkDesc> chunks;
+    std::vector<TensorInfo> tinfo((size_t)n_tensors);
+    long long rec_off = 16ll * n_tensors, flat = 0, slots = 0;
+    for (int j = 0; j < n_tensors; ++j) {
+        const sl_tensor_desc& t = tensors[j];
+        if (t.rows < 1 || t.cols < 1 || t.offset < 0) { delete c; return SL_ERR_INVALID_ARG; }
+        if (t.offset % 4 != 0) { delete c; return SL_ERR_ALIGNMENT; }
+        const long long n = t.rows * t.cols;
+        if (t.offset + n > flat) flat = t.offset + n;
+        tinfo[j].first_chunk = (long long)chunks.size();
+        long long tslots = 0;
+        const bool tiled = t.rows > 1 && t.rows % kTile == 0 && t.cols % kTile == 0;
+        if (tiled) {
+            if (t.cols > 0x7FFFFFFFll) { delete c; return SL_ERR_TOO_LARGE; }
+            const long long tr = t.rows / kTile, tc = t.cols / kTile;
+            for (long long a = 0; a < tr; ++a)
+                for (long long b = 0; b < tc; ++b) {
+                    ChunkDesc d;
+                    d.base = t.offset + a * kTile * t.cols + b * kTile;
+                    d.row_stride = (int)t.cols;
+                    d.len = kChunk;
+                    d.tensor = j;
+                    d.chunk_in_tensor = (int)(a * tc + b);
+                    d.rec_off = rec_off;
+                    rec_off += stride;
+                    tslots += cfg->k < kChunk ? cfg->k : kChunk;
+                    chunks.push_back(d);
+                }
+        } else {
+            const long long nc = (n + kChunk - 1) / kChunk;
+            for (long long a = 0; a < nc; ++a) {
+                ChunkDesc d;
+                d.base = t.offset + a * kChunk;
+                d.row_stride = 0;
+                const long long rest = n - a * kChunk;
+                d.len = (int)(rest < kChunk ? rest : kChunk);
+                d.tensor = j;
+                d.chunk_in_tensor = (int)a;
+                d.rec_off = rec_off;
+                rec_off += stride;
+                tslots += cfg->k < d.len ? cfg->k : d.len;
+                chunks.push_back(d);
+            }
+        }
+        tinfo[j].n_chunks = (long long)chunks.size() - tinfo[j].first_chunk;
+        tinfo[j].n_slots = tslots;
+        slots += tslots;
+    }
+    c->n_chunks = (long long)chunks.size();
+    c->n_slots = slots;
+    c->flat_elems = flat;
+
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkDesc));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_tinfo, tinfo.size() * sizeof(TensorInfo));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkDesc), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->d_tinfo, tinfo.data(), tinfo.size() * sizeof(TensorInfo), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        sl_status s = cuda_fail(e, "sl_create");
+        if (c->d_chunks) cudaFree(c->d_chunks);
+        if (c->d_tinfo) cudaFree(c->d_tinfo);
+        delete c;
+        return s;
+    }
+    *out = c;
+    return SL_OK;
+}
+
+sl_status sl_destroy(sl_ctx* c) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    cudaFree(c->d_chunks);
+    cudaFree(c->d_tinfo);
+    delete c;
+    return SL_OK;
+}
+
+sl_status sl_set_hyper(sl_ctx* c, float beta, float outer_lr, int32_t ef_enabled, int32_t divide_by_present) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    if (!(beta >= 0.0f && beta <= 1.0f) || !isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
+    c->cfg.beta = beta;
+    c->cfg.outer_lr = outer_lr;
+    c->cfg.ef_enabled = ef_enabled != 0;
+    c->cfg.divide_by_present = divide_by_present != 0;
+    return SL_OK;
+}
+
+sl_status sl_payload_bytes(const sl_ctx* c, size_t* bytes) {
+    if (!c || !bytes) return SL_ERR_INVALID_ARG;
+    *bytes = 16 * (size_t)c->n_tensors + (size_t)record_stride(c->cfg.k) * (size_t)c->n_chunks;
+    return SL_OK;
+}
+
+sl_status sl_num_chunks(const sl_ctx* c, int64_t* chunks, int64_t* slots) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    if (chunks) *chunks = c->n_chunks;
+    if (slots) *slots = c->n_slots;
+    return SL_OK;
+}
+
+sl_status sl_flat_elems(const sl_ctx* c, int64_t* elems) {
+    if (!c || !elems) return SL_ERR_INVALID_ARG;
+    *elems = c->flat_elems;
+    return SL_OK;
+}
+
+sl_status sl_workspace_bytes(const sl_ctx* c, size_t* bytes) {
+    if (!c || !bytes) return SL_ERR_INVALID_ARG;
+    *bytes = workspace_bytes_for(c, c->cfg.R);
+    return SL_OK;
+}
+
+sl_status sl_set_workspace(sl_ctx* c, void* dev_ptr, size_t bytes) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return SL_ERR_ALIGNMENT;
+    c->ws_ptr = dev_ptr;
+    c->ws_bytes = dev_ptr ? bytes : 0;
+    return SL_OK;
+}
+
+sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
+                      void* stream) {
+    if (!c || !theta_sync || !theta_local || !payload) return SL_ERR_INVALID_ARG;
+    if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync) || misaligned(theta_local) || misaligned(e) || misaligned(payload))
+        return SL_ERR_ALIGNMENT;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    WorkerPtrs ptrs;
+    memset(&ptrs, 0, sizeof(ptrs));
+    ptrs.theta_local[0] = theta_local;
+    ptrs.e[0] = e;
+    ptrs.payload[0] = payload;
+    return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream));
+}
+
+sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
+    if (!c || !payloads || !theta_sync) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
+    PayloadPtrs pl;
+    memset(&pl, 0, sizeof(pl));
+    int present = 0;
+    for (int r = 0; r < c->cfg.R; ++r) {
+        if (misaligned(payloads[r])) return SL_ERR_ALIGNMENT;
+        pl.p[r] = payloads[r];
+        present += payloads[r] != nullptr;
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    return launch_apply(c, pl, present, theta_sync, static_cast<cudaStream_t>(stream));
+}
+
+sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+                        uint8_t* const* payloads, void* stream) {
+    if (!c || !theta_sync || !theta_local || !payloads) return SL_ERR_INVALID_ARG;
+    if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
+    const int R = c->cfg.R;
+    WorkerPtrs ptrs;
+    PayloadPtrs pl;
+    memset(&ptrs, 0, sizeof(ptrs));
+    memset(&pl, 0, sizeof(pl));
+    for (int r = 0; r < R; ++r) {
+        if (!theta_local[r] || !payloads[r] || (c->cfg.ef_enabled && !e[r])) return SL_ERR_INVALID_ARG;
+        if (misaligned(theta_local[r]) || misaligned(payloads[r]) || (e && misaligned(e[r]))) return SL_ERR_ALIGNMENT;
+        for (int q = 0; q < r; ++q) {
+            if (payloads[q] == payloads[r]) return SL_ERR_INVALID_ARG;
+            if (c->cfg.ef_enabled && e[q] == e[r]) return SL_ERR_INVALID_ARG;
+        }
+        ptrs.theta_local[r] = theta_local[r];
+        ptrs.e[r] = e ? e[r] : nullptr;
+        ptrs.payload[r] = payloads[r];
+        pl.p[r] = payloads[r];
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    sl_status s = launch_compress(c, R, theta_sync, ptrs, st);
+    if (s != SL_OK) return s;
+    return launch_apply(c, pl, R, theta_sync, st);
+}
+
+sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* theta_local_host, float* dev_stage,
+                             float* const* e, uint8_t* const* payloads, float* theta_sync_host, void* stream) {
+    if (!c || !theta_sync || !theta_local_host || !dev_stage || !payloads) return SL_ERR_INVALID_ARG;
+    if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync) || misaligned(dev_stage)) return SL_ERR_ALIGNMENT;
+    const int R = c->cfg.R;
+    for (int r = 0; r < R; ++r) {
+        if (!theta_local_host[r] || !payloads[r] || (c->cfg.ef_enabled && !e[r])) return SL_ERR_INVALID_ARG;
+        if (misaligned(payloads[r]) || (e && misaligned(e[r]))) return SL_ERR_ALIGNMENT;
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PayloadPtrs pl;
+    memset(&pl, 0, sizeof(pl));
+    const size_t bytes = (size_t)c->flat_elems * sizeof(float);
+    for (int r = 0; r < R; ++r) {
+        SL_CUDA(cudaMemcpyAsync(dev_stage, theta_local_host[r], bytes, cudaMemcpyHostToDevice, st));
+        WorkerPtrs ptrs;
+        memset(&ptrs, 0, sizeof(ptrs));
+        ptrs.theta_local[0] = dev_stage;
+        ptrs.e[0] = e ? e[r] : nullptr;
+        ptrs.payload[0] = payloads[r];
+        sl_status s = launch_compress(c, 1, theta_sync, ptrs, st);
+        if (s != SL_OK) return s;
+        pl.p[r] = payloads[r];
+    }
+    sl_status s = launch_apply(c, pl, R, theta_sync, st);
+    if (s != SL_OK) return s;
+    if (theta_sync_host)
+        SL_CUDA(cudaMemcpyAsync(theta_sync_host, theta_sync, bytes, cudaMemcpyDeviceToHost, st));
+    SL_CUDA(cudaStreamSynchronize(st));
+    return SL_OK;
+}
+
+sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {
+    if (!c || !payload || !dev_status) return SL_ERR_INVALID_ARG;
+    if (misaligned(payload)) return SL_ERR_ALIGNMENT;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    set_status_kernel<<<1, 1, 0, st>>>(dev_status, (int)SL_OK);
+    const long long items = c->n_chunks > c->n_tensors ? c->n_chunks : c->n_tensors;
+    validate_kernel<<<blocks_for(items, 128), 128, 0, st>>>(c->d_chunks, c->n_chunks, c->n_tensors, c->cfg.k, payload,
+                                                            dev_status);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+sl_status sl_read_stats(sl_ctx* c, int32_t worker, float* dev_out, void* stream) {
+    if (!c || !dev_out || worker < 0 || worker >= c->last_workers) return SL_ERR_INVALID_ARG;
+    if (!c->ws_ptr) return SL_ERR_NOMEM;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    const Workspace ws = carve(c, c->last_workers);
+    copy_stats_kernel<<<blocks_for((long long)c->n_tensors * 8, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        ws.tstat + (long long)worker * c->n_tensors, c->n_tensors, dev_out);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+}  // extern "C"

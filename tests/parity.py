@@ -1,0 +1,132 @@
+"""Helpers for the GPU-vs-oracle parity tests (not a test module).
+
+The CUDA path runs on the whole workload; the oracle is run tensor by tensor on copies taken
+before the step (every stage of the method is per tensor, so a tensor can be checked alone).
+Bars: payload bytes (indices, codes, tables) and error buffers bit-exact; theta_sync within
+1e-6 x RMS(tensor) of the oracle's fp64 evaluation.
+"""
+from __future__ import annotations
+
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import oracle as O
+from paper_2508_15706_b200 import inputs as I
+
+THETA_TOL_REL_RMS = 1e-6
+
+
+def oracle_threads() -> int:
+    n = os.cpu_count() or 1
+    O.set_threads(n)
+    return n
+
+
+class DeviceCase:
+    """Device-resident buffers of one workload: theta_sync, D distinct theta_local buffers
+    (worker r reads buffer r % D), R error buffers, R payloads."""
+
+    def __init__(self, wl: I.Workload, k: Optional[int] = None, distinct_local: Optional[int] = None,
+                 e_scale: float = 0.0, device=None):
+        from paper_2508_15706_b200.binding import SparseLoCo
+        self.wl = wl
+        self.k = wl.k if k is None else k
+        self.dev = device or torch.device("cuda", torch.cuda.current_device())
+        self.offs = I.offsets(wl.tensors)
+        self.shapes = [(t.rows, t.cols) for t in wl.tensors]
+        self.D = wl.R if distinct_local is None else distinct_local
+        self.sl = SparseLoCo(self.shapes, self.offs, k=self.k, R=wl.R, H=wl.H, beta=wl.beta,
+                             outer_lr=wl.outer_lr)
+        self.theta = I.theta_sync(wl, self.dev)
+        self.local = [torch.empty_like(self.theta) for _ in range(self.D)]
+        self.e = [I.initial_error(wl, r, self.dev, scale=e_scale) for r in range(wl.R)]
+        self.payloads = [torch.zeros(self.sl.payload_bytes(), dtype=torch.uint8, device=self.dev)
+                         for _ in range(wl.R)]
+        self.cfg = O.Config(k=self.k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr)
+        # payload geometry, from the oracle's definitions
+        self.rec_off, self.n_chunks = [], []
+        stride = O.record_stride(self.k)
+        pos = 16 * len(self.shapes)
+        for j, sh in enumerate(self.shapes):
+            nc = O.num_chunks(self.cfg, O.Table([sh]), 0)
+            self.rec_off.append(pos)
+            self.n_chunks.append(nc)
+            pos += nc * stride
+        self.payload_bytes = pos
+        self.stride = stride
+
+    def fill_local(self, step: int) -> None:
+        for d in range(self.D):
+            I.theta_local(self.wl, self.theta, d, step, out=self.local[d])
+
+    def local_of(self, r: int) -> torch.Tensor:
+        return self.local[r % self.D]
+
+    def snapshot(self, tensor_ids: Sequence[int]) -> Dict[int, dict]:
+        """CPU copies of theta_sync / theta_local / e slices of the given tensors (pre-step)."""
+        snap = {}
+        for j in tensor_ids:
+            t, off = self.wl.tensors[j], self.offs[j]
+            sl = slice(off, off + t.numel)
+            snap[j] = {
+                "theta": self.theta[sl].cpu().numpy().copy(),
+                "local": [self.local_of(r)[sl].cpu().numpy().copy() for r in range(self.wl.R)],
+                "e": [self.e[r][sl].cpu().numpy().copy() for r in range(self.wl.R)],
+            }
+        return snap
+
+    def step(self) -> None:
+        self.sl.outer_step(self.theta, [self.local_of(r) for r in range(self.wl.R)], self.e, self.payloads)
+
+    def tensor_payload(self, r: int, j: int) -> np.ndarray:
+        p = self.payloads[r]
+        hdr = p[16 * j:16 * j + 16].cpu().numpy()
+        recs = p[self.rec_off[j]:self.rec_off[j] + self.n_chunks[j] * self.stride].cpu().numpy()
+        return np.concatenate([hdr, recs])
+
+    def check(self, snap: Dict[int, dict], ef_enabled: bool = True, present: Optional[List[bool]] = None) -> dict:
+        """Run the oracle on the snapshot tensors and compare with the device state after step()."""
+        torch.cuda.synchronize()
+        R = self.wl.R
+        worst = 0.0
+        report = {"tensors": 0, "payload_bytes": 0, "theta_max_err_over_rms": 0.0}
+        cfg = O.Config(k=self.k, R=R, H=self.wl.H, beta=self.wl.beta, outer_lr=self.wl.outer_lr,
+                       ef_enabled=int(ef_enabled))
+        for j, s in snap.items():
+            t, off = self.wl.tensors[j], self.offs[j]
+            tab = O.Table([(t.rows, t.cols)])
+            th = s["theta"].copy()
+            pays = []
+            for r in range(R):
+                e_o = s["e"][r].copy()
+                out = O.compress(cfg, tab, s["theta"], s["local"][r], e_o)
+                got = self.tensor_payload(r, j)
+                if not np.array_equal(got, out.payload):
+                    bad = np.nonzero(got != out.payload)[0]
+                    raise AssertionError(
+                        f"payload mismatch: tensor {j} ({t.name}) worker {r}: {bad.size} bytes differ, first at "
+                        f"{bad[0]} (record {(bad[0] - 16) // self.stride if bad[0] >= 16 else 'header'})")
+                e_g = self.e[r][off:off + t.numel].cpu().numpy()
+                if not np.array_equal(e_g.view(np.uint32), e_o.view(np.uint32)):
+                    bad = np.nonzero(e_g.view(np.uint32) != e_o.view(np.uint32))[0]
+                    raise AssertionError(f"error buffer mismatch: tensor {j} ({t.name}) worker {r}: "
+                                         f"{bad.size} elements, first {bad[0]}: {e_g[bad[0]]} vs {e_o[bad[0]]}")
+                pays.append(out.payload if (present is None or present[r]) else None)
+                report["payload_bytes"] += out.payload.size
+            O.aggregate_apply(cfg, tab, pays, th)
+            th_g = self.theta[off:off + t.numel].cpu().numpy()
+            rms = float(np.sqrt(np.mean(th.astype(np.float64) ** 2)))
+            err = float(np.max(np.abs(th_g.astype(np.float64) - th.astype(np.float64))))
+            assert err <= THETA_TOL_REL_RMS * rms, f"theta mismatch: tensor {j} ({t.name}): {err} vs rms {rms}"
+            worst = max(worst, err / rms if rms > 0 else 0.0)
+            report["tensors"] += 1
+        report["theta_max_err_over_rms"] = worst
+        return report
+
+
+def sample_tensor_ids(wl: I.Workload, want_names: Sequence[str]) -> List[int]:
+    names = [t.name for t in wl.tensors]
+    return [names.index(n) for n in want_names if n in names]

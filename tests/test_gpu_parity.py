@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+Bit-exact payloads (indices, codes, tables) and error buffers; theta_sync within 1e-6 x RMS."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2508_15706_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(*a, **kw):
+    from parity import DeviceCase, oracle_threads
+    oracle_threads()
+    return DeviceCase(*a, **kw)
+
+
+SMALL = [I.TensorSpec("a", 128, 192, 0), I.TensorSpec("flat", 1, 5000, 0), I.TensorSpec("router", 8, 1024, 1),
+         I.TensorSpec("norm", 1, 768, 1), I.TensorSpec("tiny", 1, 40, 2), I.TensorSpec("odd2d", 70, 64, 2),
+         I.TensorSpec("mid", 1, 4096 + 2051, 3), I.TensorSpec("b", 64, 64, 3)]
+
+
+def test_config1_single_tensor_with_ties():
+    wl = I.workload("c1_single_1024")
+    c = _case(wl)
+    for step in range(2):
+        c.fill_local(step)
+        snap = c.snapshot([0])
+        c.step()
+        rep = c.check(snap)
+        assert rep["tensors"] == 1
+    assert c.sl.payload_bytes() == 28688
+
+
+@pytest.mark.parametrize("k", [1, 41, 64, 82, 123, 256])
+def test_small_shapes_k_sweep(k):
+    wl = I.Workload("small", SMALL, R=3, k=k, recipe="student_t4", seed=20 + k, outer_lr=0.7)
+    c = _case(wl, e_scale=0.5)
+    for step in range(2):
+        c.fill_local(step)
+        snap = c.snapshot(range(len(SMALL)))
+        c.step()
+        c.check(snap)
+
+
+def test_zero_and_heavy_ties():
+    wl = I.Workload("ties", SMALL, R=2, k=64, recipe="normal", seed=31)
+    c = _case(wl)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    n = c.theta.numel()
+    # worker 0: theta_local == theta_sync and e == 0  -> all-zero chunks
+    c.local[0].copy_(c.theta)
+    # worker 1: drift takes five magnitudes only (both signs) -> every chunk is one big tie group
+    vals = torch.tensor([0.0, 2.0 ** -9, -2.0 ** -9, 2.0 ** -7, -2.0 ** -7], dtype=torch.float32)
+    pick = vals[torch.randint(0, 5, (n,), generator=g)].to(c.dev)
+    c.theta.copy_(torch.round(c.theta * 1024) / 1024)  # exact differences
+    c.local[0].copy_(c.theta)
+    c.local[1].copy_(c.theta - pick)
+    snap = c.snapshot(range(len(SMALL)))
+    c.step()
+    c.check(snap)
+    # second step: zero drift with non-zero error buffers
+    c.local[1].copy_(c.theta)
+    c.local[0].copy_(c.theta)
+    snap = c.snapshot(range(len(SMALL)))
+    c.step()
+    c.check(snap)
+
+
+def test_extreme_values():
+    """Denormals are ordinary values: nothing is flushed to zero on either side."""
+    wl = I.Workload("extreme", [I.TensorSpec("a", 64, 128, 0), I.TensorSpec("v", 1, 4096, 0)], R=1, k=64,
+                    recipe="normal", seed=33, beta=1.0)
+    c = _case(wl)
+    c.fill_local(0)
+    n = c.theta.numel()
+    g = torch.Generator(device="cpu").manual_seed(6)
+    pos = torch.randperm(n, generator=g)[:600].to(c.dev)
+    c.theta[pos[:200]] = 0.0
+    c.local[0][pos[:100]] = 1e-41
+    c.local[0][pos[100:200]] = -3e-42
+    c.e[0][pos[200:400]] = 2e-44
+    c.local[0][pos[400:600]] = c.theta[pos[400:600]]
+    snap = c.snapshot([0, 1])
+    c.step()
+    c.check(snap)
+
+
+def test_error_feedback_freeze():
+    wl = I.Workload("freeze", SMALL, R=2, k=64, recipe="normal", seed=41)
+    c = _case(wl, e_scale=0.5)
+    c.sl.set_hyper(ef_enabled=False)
+    c.fill_local(0)
+    e_before = [x.clone() for x in c.e]
+    snap = c.snapshot(range(len(SMALL)))
+    c.step()
+    c.check(snap, ef_enabled=False)
+    for a, b in zip(c.e, e_before):
+        assert torch.equal(a, b)
+
+
+def test_compress_then_aggregate_equals_outer_step_and_absent_workers():
+    import oracle as O
+    wl = I.Workload("split", SMALL, R=3, k=64, recipe="normal", seed=51, outer_lr=0.8)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    a.fill_local(0)
+    b.fill_local(0)
+    a.step()
+    for r in range(3):
+        b.sl.compress(b.theta, b.local[r], b.e[r], b.payloads[r])
+    theta_before = b.theta.clone()
+    b.sl.aggregate_apply(b.payloads, b.theta)
+    torch.cuda.synchronize()
+    assert torch.equal(a.theta, b.theta)
+    for r in range(3):
+        assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+    # one worker absent: oracle with the same payloads, divisor R then divisor 2
+    pays = [p.cpu().numpy() for p in b.payloads]
+    tab = O.Table(b.shapes, b.offs)
+    for dbp in (0, 1):
+        th = theta_before.clone()
+        b.sl.set_hyper(divide_by_present=bool(dbp))
+        b.sl.aggregate_apply([b.payloads[0], None, b.payloads[2]], th)
+        th_o = theta_before.cpu().numpy().copy()
+        O.aggregate_apply(O.Config(k=64, R=3, outer_lr=0.8, divide_by_present=dbp), tab, [pays[0], None, pays[2]], th_o)
+        rms = float(np.sqrt(np.mean(th_o.astype(np.float64) ** 2)))
+        assert np.max(np.abs(th.cpu().numpy().astype(np.float64) - th_o)) <= 1e-6 * rms
+    # nobody present: theta untouched
+    th = theta_before.clone()
+    b.sl.aggregate_apply([None, None, None], th)
+    torch.cuda.synchronize()
+    assert torch.equal(th, theta_before)
+
+
+def test_runs_are_bit_reproducible():
+    wl = I.Workload("repro", SMALL, R=4, k=64, recipe="student_t4", seed=61)
+    outs = []
+    for _ in range(2):
+        c = _case(wl, e_scale=0.5)
+        c.fill_local(0)
+        c.step()
+        torch.cuda.synchronize()
+        outs.append((c.theta.clone(), [x.clone() for x in c.e], [p.clone() for p in c.payloads]))
+    assert torch.equal(outs[0][0], outs[1][0])
+    for x, y in zip(outs[0][1] + outs[0][2], outs[1][1] + outs[1][2]):
+        assert torch.equal(x, y)
+
+
+def test_validate_payload_flags_corruption():
+    wl = I.Workload("val", SMALL, R=1, k=41, recipe="normal", seed=71)
+    c = _case(wl)
+    c.fill_local(0)
+    c.step()
+    status = torch.full((1,), -1, dtype=torch.int32, device=c.dev)
+    c.sl.validate_payload(c.payloads[0], status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    stride = c.stride
+    first = c.rec_off[0]
+    corruptions = []
+    p = c.payloads[0].clone()
+    p[first] = 0xFF; p[first + 1] = 0xFF  # index 0xFFF first, then a smaller one: not ascending
+    corruptions.append(p)
+    p = c.payloads[0].clone()
+    p[first + stride - 1] = 1  # padding must be zero
+    corruptions.append(p)
+    p = c.payloads[0].clone()
+    p[0:4] = torch.tensor(np.frombuffer(np.float32(np.inf).tobytes(), np.uint8).copy())  # table not finite
+    corruptions.append(p)
+    p = c.payloads[0].clone()
+    tiny_rec = c.rec_off[4]  # the 40-element tensor: slots >= 40 must be zero
+    p[tiny_rec + (12 * 40) // 8 + 1] = 0x10
+    corruptions.append(p)
+    for bad in corruptions:
+        c.sl.validate_payload(bad, status)
+        torch.cuda.synchronize()
+        assert status.item() == 4
+    # a corrupted payload must not fault the apply kernel either (indices beyond the chunk are dropped)
+    th = c.theta.clone()
+    c.sl.aggregate_apply([corruptions[0]], th)
+    torch.cuda.synchronize()
+
+
+def test_argument_errors():
+    from paper_2508_15706_b200 import binding as B
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo([(64, 64)], k=64, R=1, chunk_elems=1024, tile_dim=32)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo([(64, 64)], k=0, R=1)
+    assert ei.value.status == B.SL_ERR_INVALID_ARG
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo([(64, 64)], k=300, R=1)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo([(64, 64), (1, 10)], offsets=[0, 4098], k=8, R=1)
+    assert ei.value.status == B.SL_ERR_ALIGNMENT
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo([(64, 64)], k=8, R=1, beta=1.5)
+    assert ei.value.status == B.SL_ERR_INVALID_ARG
+    sl = B.SparseLoCo([(64, 64)], k=8, R=2, alloc_workspace=False)
+    dev = torch.device("cuda")
+    th = torch.zeros(4096, device=dev)
+    pay = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(2)]
+    e = [torch.zeros(4096, device=dev) for _ in range(2)]
+    with pytest.raises(B.SlError) as ei:  # no workspace lent
+        sl.outer_step(th, [th, th], e, pay)
+    assert ei.value.status == B.SL_ERR_NOMEM
+    ws = torch.empty(sl.workspace_bytes(), dtype=torch.uint8, device=dev)
+    sl.set_workspace(ws)
+    with pytest.raises(B.SlError) as ei:  # aliased error buffers
+        sl.outer_step(th, [th, th], [e[0], e[0]], pay)
+    assert ei.value.status == B.SL_ERR_INVALID_ARG
+    with pytest.raises(B.SlError) as ei:  # misaligned pointer
+        sl.outer_step(th, [th, th], e, [pay[0], pay[1][1:]])
+    assert ei.value.status == B.SL_ERR_ALIGNMENT
+    sl.outer_step(th, [th, th], e, pay)
+    torch.cuda.synchronize()
