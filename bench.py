@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the SparseLoCo outer step (metric: outer-step params/s and achieved HBM GB/s).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one whole outer step -- pseudo-gradient, error feedback, chunk-wise Top-k, 2-bit
+quantise + pack, error subtract, decode/average of the R payloads, outer update -- for all R
+resident workers of the workload, through the C ABI (sl_outer_step).  Prints ONE JSON line.
+
+The path has no exchange between GPUs (R workers are R buffer sets on one GPU), so with N > 1 every
+rank runs an independent replica of the workload ("replicas only"): value = N x params / max time.
+
+--impl reference times the CPU oracle (test infrastructure, a deliberately plain program) on a
+bounded sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparseloco_outer_step_params_per_s"
+UNIT = "params/s"
+DEFAULT_WORKLOAD = "c5_dense_d2048"
+
+# DRAM bytes per ef_topk launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
+# on a smaller case of the same kernel, as bytes per (parameter x worker); see profiles/.
+NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = None
+
+
+def record_stride(k: int) -> int:
+    return ((12 * k + 7) // 8 + (2 * k + 7) // 8 + 15) // 16 * 16
+
+
+def algorithmic_bytes_per_param(R: int, k: int) -> float:
+    """Bytes the method must move per parameter per outer step (fp32 state): per worker theta_r
+    read + e read + e write; theta_sync read once by the compression and read + written by the
+    update; every payload written once and read once."""
+    return R * 12 + 4 + 8 + R * 2 * record_stride(k) / 4096.0
+
+
+def ef_topk_bytes_per_param(R: int) -> float:
+    return R * 12 + 4
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        sm, smax, power, reasons = [], [], [], set()
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def pick_distinct_locals(torch, wl, k: int, flat: int, payload_bytes: int, workspace_bytes: int) -> int:
+    """How many distinct theta_local buffers fit (worker r reads buffer r % D)."""
+    free, _total = torch.cuda.mem_get_info()
+    fixed = (1 + wl.R) * 4 * flat + wl.R * payload_bytes + workspace_bytes + (6 << 30)
+    for D in [wl.R] + [d for d in (32, 16, 8, 4, 2, 1) if d < wl.R]:
+        if fixed + D * 4 * flat <= free:
+            return D
+    raise RuntimeError(f"workload {wl.name} does not fit: need {fixed + 4 * flat} bytes, {free} free")
+
+
+def run_ours(args) -> dict:
+    import torch
+    import torch.distributed as dist
+    from paper_2508_15706_b200 import inputs as I
+    from paper_2508_15706_b200.binding import SparseLoCo
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the outer step has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = I.workload(args.workload)
+    if args.R:
+        import dataclasses
+        wl = dataclasses.replace(wl, R=args.R)
+    k = args.k or wl.k
+    shapes = [(t.rows, t.cols) for t in wl.tensors]
+    offs = I.offsets(wl.tensors)
+    flat = I.flat_numel(wl.tensors)
+    N = wl.numel
+
+    sl = SparseLoCo(shapes, offs, k=k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr, alloc_workspace=False)
+    D = pick_distinct_locals(torch, wl, k, flat, sl.payload_bytes(), sl.workspace_bytes())
+    ws = torch.empty(sl.workspace_bytes(), dtype=torch.uint8, device=dev)
+    sl.set_workspace(ws)
+    theta = I.theta_sync(wl, dev)
+    local = []
+    for d in range(D):
+        local.append(I.theta_local(wl, theta, d, 0))
+    e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(wl.R)]
+    payloads = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(wl.R)]
+    locals_r = [local[r % D] for r in range(wl.R)]
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        sl.outer_step(theta, locals_r, e, payloads)
+    torch.cuda.synchronize()
+    sl.profile_enable(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        sl.outer_step(theta, locals_r, e, payloads)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t0, t1)
+    prof = sl.profile_read()
+    sl.profile_enable(False)
+    if world > 1:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_max = float(tmax.item())
+    else:
+        ms_max = ms
+    ms_per_step = ms_max / args.steps
+    value = world * N * args.steps / (ms_max * 1e-3)
+
+    # roofline of the dominant kernel, timed live with CUDA events inside the timed region
+    top = max(prof.items(), key=lambda kv: kv[1][0])
+    ef_ms, ef_n = prof["ef_topk"]
+    ef_avg_ms = ef_ms / max(ef_n, 1)
+    ef_bytes = ef_topk_bytes_per_param(wl.R) * N
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_src = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
+    achieved = ef_bytes / (ef_avg_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER is not None:
+        traffic = NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER * N * wl.R
+    step_bytes = algorithmic_bytes_per_param(wl.R, k) * N
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    kernel_ms = {name: round(v[0] / max(v[1], 1), 4) for name, v in prof.items()}
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "params": N, "tensors": len(wl.tensors), "R": wl.R, "k": k, "H": wl.H,
+                   "chunk": 4096, "beta": wl.beta, "outer_lr": wl.outer_lr,
+                   "distinct_theta_local_buffers": D,
+                   "l2": "inputs larger than L2 (every buffer is %.1f GB; state evolves every step)" % (4 * flat / 1e9),
+                   "multi_gpu": "replicas only (no data-path collective)"},
+        "clocks": clocks,
+        "gpu_launches": 9 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "ef_topk", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": ef_bytes, "avg_launch_ms": ef_avg_ms,
+                     "dominant_by_time": top[0]},
+        "step_roofline": {"algorithmic_bytes_per_param": algorithmic_bytes_per_param(wl.R, k),
+                          "achieved_gbs": step_gbs, "frac_of_measured_peak": step_gbs / peak,
+                          "frac_of_nominal_8000": step_gbs / 8000.0},
+        "kernel_ms_per_launch": kernel_ms,
+    }
+
+    if rank == 0 and world == 1 and not args.no_e2e:
+        del local, locals_r
+        torch.cuda.empty_cache()
+        result["e2e"] = run_e2e(torch, I, sl, wl, theta, e, payloads, flat, N, args)
+    elif not args.no_e2e:
+        result["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(wl, k, budget_s=args.cpu_budget)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return result if rank == 0 else None
+
+
+def run_e2e(torch, I, sl, wl, theta, e, payloads, flat, N, args) -> dict:
+    """The same step through the host-buffer entry point: every worker's parameters start in pinned
+    host memory and cross to the device inside the timed region; the updated theta_sync is read back."""
+    dev = theta.device
+    n_host = min(2, wl.R)  # distinct pinned host buffers; worker r reads buffer r % n_host
+    host = []
+    for d in range(n_host):
+        h = torch.empty(flat, dtype=torch.float32, pin_memory=True)
+        tmp = I.theta_local(wl, theta, d, 1)
+        h.copy_(tmp)
+        del tmp
+        host.append(h)
+    theta_host = torch.empty(flat, dtype=torch.float32, pin_memory=True)
+    flat4 = (flat + 3) // 4 * 4
+    stage = torch.empty(2 * flat4, dtype=torch.float32, device=dev)
+    hosts_r = [host[r % n_host] for r in range(wl.R)]
+    torch.cuda.synchronize()
+    steps = max(1, min(args.e2e_steps, args.steps))
+    sl.outer_step_host(theta, hosts_r, stage, e, payloads, theta_host)  # warm-up
+    t0 = time.time()
+    for _ in range(steps):
+        sl.outer_step_host(theta, hosts_r, stage, e, payloads, theta_host)
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    return {"value": N * steps / dt, "unit": UNIT, "steps": steps, "ms_per_step": dt / steps * 1e3,
+            "h2d_bytes_per_step": wl.R * 4 * flat, "d2h_bytes_per_step": 4 * flat,
+            "entry_point": "sl_outer_step_host", "distinct_host_buffers": n_host,
+            "checksum": float(theta_host[:1024].double().sum())}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places bench.py touches oracle/)
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample(wl, k, budget_s: float):
+    """A bounded sample of the workload for the oracle: tensors of the first layer, as many as fit
+    the time budget (calibrated on one small tensor), all R workers, one whole outer step."""
+    import numpy as np
+    import oracle as O
+    from paper_2508_15706_b200 import inputs as I
+    cores = os.cpu_count() or 1
+    O.set_threads(cores)
+    cand = [j for j, t in enumerate(wl.tensors) if t.layer == 0 and t.rows > 1] or list(range(len(wl.tensors)))
+
+    def make(ids, step):
+        tensors = [wl.tensors[j] for j in ids]
+        sub = I.Workload(wl.name + "_sample", tensors, R=wl.R, k=k, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr,
+                         recipe="normal" if wl.recipe == "moe_zero" else wl.recipe, seed=wl.seed)
+        if wl.recipe == "outlier_ties":
+            sub = wl
+        theta = I.theta_sync(sub, "cpu")
+        local = [I.theta_local(sub, theta, r, step).numpy() for r in range(wl.R)]
+        e = [I.initial_error(sub, r, "cpu", scale=0.5).numpy() for r in range(wl.R)]
+        tab = O.Table([(t.rows, t.cols) for t in sub.tensors], I.offsets(sub.tensors))
+        cfg = O.Config(k=k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr)
+        return cfg, tab, theta.numpy(), local, e, sum(t.numel for t in sub.tensors)
+
+    # calibrate on the smallest candidate
+    j0 = min(cand, key=lambda j: wl.tensors[j].numel)
+    cfg, tab, th, lo, e, n0 = make([j0], 0)
+    t0 = time.time()
+    O.outer_step(cfg, tab, th, lo, e)
+    rate = n0 / max(time.time() - t0, 1e-6)
+    ids, tot = [], 0
+    for j in cand:
+        if ids and (tot + wl.tensors[j].numel) / rate > budget_s:
+            break
+        ids.append(j)
+        tot += wl.tensors[j].numel
+    return make, ids, cores
+
+
+def cpu_baseline(wl, k, budget_s: float) -> dict:
+    import oracle as O
+    make, ids, cores = oracle_sample(wl, k, budget_s)
+    cfg, tab, th, lo, e, n = make(ids, 0)
+    t0 = time.time()
+    O.outer_step(cfg, tab, th, lo, e)
+    dt = time.time() - t0
+    names = ",".join(wl.tensors[j].name for j in ids)
+    return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
+            "sample": f"one outer step, all R={wl.R} workers, tensors [{names}] = {n} params of {wl.numel}"}
+
+
+def run_reference(args) -> dict:
+    from paper_2508_15706_b200 import inputs as I
+    import oracle as O
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    wl = I.workload(args.workload)
+    k = args.k or wl.k
+    total = args.steps + args.warmup
+    make, ids, cores = oracle_sample(wl, k, budget_s=max(1.0, args.reference_budget / max(total, 1)))
+    cfg, tab, th, lo, e, n = make(ids, 0)
+    for _ in range(args.warmup):
+        O.outer_step(cfg, tab, th, lo, e)
+    t0 = time.time()
+    for _ in range(args.steps):
+        O.outer_step(cfg, tab, th, lo, e)
+    dt = time.time() - t0
+    value = n * args.steps / dt
+    names = ",".join(wl.tensors[j].name for j in ids)
+    sample = f"each step = one outer step, all R={wl.R} workers, tensors [{names}] = {n} params of {wl.numel}"
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "params": wl.numel, "R": wl.R, "k": k, "H": wl.H, "chunk": 4096},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--k", type=int, default=0)
+    ap.add_argument("--R", type=int, default=0, help="override the workload's worker count (profiling)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    out = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if out is not None:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

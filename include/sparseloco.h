@@ -128,15 +128,18 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
 
-/* Same step with the workers' parameters in HOST memory (pinned for full speed): theta_local_host
- * is a host array of R host pointers; each is copied to the device staging buffer `dev_stage`
- * (flat fp32, sl_flat_elems() elements, caller-owned) and compressed in turn; then the payloads are
+/* Same step with the workers' parameters in HOST memory (pinned for full speed), the shape a
+ * deployment has when the inner loop's result arrives over the host (Alg. 1: every worker's
+ * Dhat_r is gathered before the update).  theta_local_host is a host array of R host pointers;
+ * worker r is copied to the caller-owned device staging area `dev_stage` (stage_elems floats:
+ * at least sl_flat_elems() rounded up to 4; with twice that, the copy of worker r + 1 overlaps
+ * the compression of worker r on an internal copy stream) and compressed; then the payloads are
  * aggregated and, if theta_sync_host is not NULL, the updated theta_sync is copied back to it.
  * Synchronises the stream before returning.  e, payloads and theta_sync stay resident on the
- * device (Alg. 1 keeps e_r on its worker). */
+ * device (Alg. 1 keeps e_r on its worker).  Errors as sl_outer_step, plus NOMEM (stage too small). */
 sl_status sl_outer_step_host(sl_ctx* ctx, float* theta_sync, const float* const* theta_local_host,
-                             float* dev_stage, float* const* e, uint8_t* const* payloads,
-                             float* theta_sync_host, void* cuda_stream);
+                             float* dev_stage, size_t stage_elems, float* const* e,
+                             uint8_t* const* payloads, float* theta_sync_host, void* cuda_stream);
 
 /* Check one payload before trusting it: every index < chunk length and strictly ascending over
  * the used slots, unused slots and padding zero, table entries finite.  Writes SL_OK or
@@ -148,6 +151,16 @@ sl_status sl_validate_payload(sl_ctx* ctx, const uint8_t* payload, int32_t* dev_
  * copies 8 floats per tensor (mu, sigma, 3 sigma, table[4], 0) for workspace worker slot
  * `worker` into dev_out (device, 8 * n_tensors floats). */
 sl_status sl_read_stats(sl_ctx* ctx, int32_t worker, float* dev_out, void* cuda_stream);
+
+/* Optional per-kernel timing for benchmarks (no counterpart in the paper, which reports no
+ * kernel times).  While enabled, every outer step / compression records CUDA events between its
+ * kernels on the caller's stream (up to 256 sequences between reads).  sl_profile_read()
+ * waits for the recorded events, writes per-kernel total milliseconds and launch counts into
+ * two host arrays of SL_PROFILE_SLOTS entries, and clears the record. */
+#define SL_PROFILE_SLOTS 9
+sl_status sl_profile_enable(sl_ctx* ctx, int32_t enable);
+sl_status sl_profile_read(sl_ctx* ctx, float* ms_total, int64_t* launches);
+const char* sl_profile_name(int32_t slot);
 
 const char* sl_strerror(sl_status s);
 const char* sl_last_cuda_error(void); /* text of the last CUDA error seen by this thread */

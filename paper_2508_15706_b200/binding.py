@@ -19,8 +19,9 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error",
+    "sl_last_cuda_error", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
+PROFILE_SLOTS = 9
 
 SL_OK = 0
 SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_BAD_PAYLOAD = 1, 2, 3, 4
@@ -64,7 +65,11 @@ def _load():
     L.sl_compress.argtypes = [P, P, P, P, P, P]
     L.sl_aggregate_apply.argtypes = [P, P, P, P]
     L.sl_outer_step.argtypes = [P, P, P, P, P, P]
-    L.sl_outer_step_host.argtypes = [P, P, P, P, P, P, P, P]
+    L.sl_outer_step_host.argtypes = [P, P, P, P, C.c_size_t, P, P, P, P]
+    L.sl_profile_enable.argtypes = [P, C.c_int32]
+    L.sl_profile_read.argtypes = [P, P, P]
+    L.sl_profile_name.argtypes = [C.c_int32]
+    L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
     L.sl_read_stats.argtypes = [P, C.c_int32, P, P]
     L.sl_strerror.argtypes = [C.c_int]
@@ -218,7 +223,18 @@ class SparseLoCo:
             assert not theta_sync_host.is_cuda and theta_sync_host.is_contiguous()
             hp = theta_sync_host.data_ptr()
         _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
-                                     _dev_ptr(dev_stage, torch.float32), ea, pa, hp, _stream()))
+                                     _dev_ptr(dev_stage, torch.float32), dev_stage.numel(), ea, pa, hp,
+                                     _stream()))
+
+    def profile_enable(self, on: bool = True) -> None:
+        _check(_L.sl_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        """{kernel name: (total ms, launches)} since the last read; waits for the recorded events."""
+        ms = (C.c_float * PROFILE_SLOTS)()
+        n = (C.c_int64 * PROFILE_SLOTS)()
+        _check(_L.sl_profile_read(self._h, ms, n))
+        return {_L.sl_profile_name(i).decode(): (ms[i], n[i]) for i in range(PROFILE_SLOTS)}
 
     def validate_payload(self, payload, status: torch.Tensor) -> None:
         assert status.dtype == torch.int32

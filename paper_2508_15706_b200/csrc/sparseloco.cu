@@ -34,6 +34,8 @@ constexpr int kMaxR = 64;
 constexpr int kMaxK = 256;
 constexpr int kCandCap = 1024;         // candidate list capacity of the selection
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kProfSlots = 9;     // kernels of one outer step
+constexpr int kProfMaxSeq = 256;  // recorded sequences kept between two reads
 
 thread_local char g_cuda_err[256] = "";
 
@@ -682,6 +684,14 @@ struct sl_ctx {
     void* ws_ptr;
     size_t ws_bytes;
     int last_workers;  // worker count the workspace was last laid out for
+    // optional per-kernel timing (sl_profile_*)
+    bool prof_on;
+    int prof_steps;                        // compress/apply sequences recorded since the last read
+    std::vector<cudaEvent_t> prof_events;  // [kProfMaxSeq][kProfSlots + 1]
+    // copy stream + events of sl_outer_step_host (created on first use)
+    cudaStream_t copy_stream;
+    cudaEvent_t ev_copied[2], ev_consumed[2];
+    bool host_path_ready;
 };
 
 namespace {
@@ -722,6 +732,12 @@ inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) &
 
 unsigned blocks_for(long long items, int per_block) { return (unsigned)((items + per_block - 1) / per_block); }
 
+// Event after profile slot `slot` (slot -1 = start of the sequence) of the sequence being recorded.
+inline void prof_mark(sl_ctx* c, int slot, cudaStream_t st) {
+    if (!c->prof_on || c->prof_steps >= kProfMaxSeq) return;
+    cudaEventRecord(c->prof_events[(size_t)c->prof_steps * (kProfSlots + 1) + (slot + 1)], st);
+}
+
 // Compression of `workers` workers whose pointers are in `ptrs` (kernels 1-8).
 sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const WorkerPtrs& ptrs,
                           cudaStream_t st) {
@@ -733,23 +749,32 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     if (WG > 0x7FFFFFFFll) return SL_ERR_TOO_LARGE;
     const bool ef = c->cfg.ef_enabled != 0;
 
+    prof_mark(c, -1, st);
     if (ef)
         ef_topk_kernel<true><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
                                                                 theta_sync, ptrs, ws);
     else
         ef_topk_kernel<false><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
                                                                  theta_sync, ptrs, ws);
+    prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T * 32, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    prof_mark(c, 1, st);
     tensor_reduce_kernel<0><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    prof_mark(c, 2, st);
     chunk_sum_kernel<1><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    prof_mark(c, 3, st);
     tensor_reduce_kernel<1><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    prof_mark(c, 4, st);
     chunk_bins_kernel<<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
+    prof_mark(c, 5, st);
     tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    prof_mark(c, 6, st);
     if (ef)
         pack_fix_kernel<true><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     else
         pack_fix_kernel<false><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    prof_mark(c, 7, st);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -767,6 +792,8 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     }
     decode_avg_apply_kernel<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl,
                                                                           theta_sync);
+    prof_mark(c, 8, st);
+    if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -824,6 +851,10 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->ws_ptr = nullptr;
     c->ws_bytes = 0;
     c->last_workers = cfg->R;
+    c->prof_on = false;
+    c->prof_steps = 0;
+    c->copy_stream = nullptr;
+    c->host_path_ready = false;
     c->tensors.assign(tensors, tensors + n_tensors);
 
     const int stride = record_stride(cfg->k);
@@ -902,6 +933,14 @@ sl_status sl_destroy(sl_ctx* c) {
     DeviceGuard g(c->device);
     cudaFree(c->d_chunks);
     cudaFree(c->d_tinfo);
+    for (auto& ev : c->prof_events) cudaEventDestroy(ev);
+    if (c->host_path_ready) {
+        cudaStreamDestroy(c->copy_stream);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(c->ev_copied[i]);
+            cudaEventDestroy(c->ev_consumed[i]);
+        }
+    }
     delete c;
     return SL_OK;
 }
@@ -1012,11 +1051,15 @@ sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
 }
 
 sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* theta_local_host, float* dev_stage,
-                             float* const* e, uint8_t* const* payloads, float* theta_sync_host, void* stream) {
+                             size_t stage_elems, float* const* e, uint8_t* const* payloads, float* theta_sync_host,
+                             void* stream) {
     if (!c || !theta_sync || !theta_local_host || !dev_stage || !payloads) return SL_ERR_INVALID_ARG;
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(dev_stage)) return SL_ERR_ALIGNMENT;
     const int R = c->cfg.R;
+    const size_t flat = (size_t)((c->flat_elems + 3) / 4 * 4);
+    if (stage_elems < flat) return SL_ERR_NOMEM;
+    const int nbuf = stage_elems >= 2 * flat ? 2 : 1;
     for (int r = 0; r < R; ++r) {
         if (!theta_local_host[r] || !payloads[r] || (c->cfg.ef_enabled && !e[r])) return SL_ERR_INVALID_ARG;
         if (misaligned(payloads[r]) || (e && misaligned(e[r]))) return SL_ERR_ALIGNMENT;
@@ -1024,18 +1067,36 @@ sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* t
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!c->host_path_ready) {
+        SL_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            SL_CUDA(cudaEventCreateWithFlags(&c->ev_copied[i], cudaEventDisableTiming));
+            SL_CUDA(cudaEventCreateWithFlags(&c->ev_consumed[i], cudaEventDisableTiming));
+        }
+        c->host_path_ready = true;
+    }
     PayloadPtrs pl;
     memset(&pl, 0, sizeof(pl));
     const size_t bytes = (size_t)c->flat_elems * sizeof(float);
+    // Worker r's parameters travel on the copy stream into staging buffer r % nbuf while worker
+    // r - 1 is being compressed on the caller's stream.
+    SL_CUDA(cudaEventRecord(c->ev_consumed[0], st));  // orders the first copies after prior work on `st`
+    SL_CUDA(cudaEventRecord(c->ev_consumed[1], st));
     for (int r = 0; r < R; ++r) {
-        SL_CUDA(cudaMemcpyAsync(dev_stage, theta_local_host[r], bytes, cudaMemcpyHostToDevice, st));
+        const int bsel = r % nbuf;
+        float* stage = dev_stage + (size_t)bsel * flat;
+        SL_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_consumed[bsel], 0));
+        SL_CUDA(cudaMemcpyAsync(stage, theta_local_host[r], bytes, cudaMemcpyHostToDevice, c->copy_stream));
+        SL_CUDA(cudaEventRecord(c->ev_copied[bsel], c->copy_stream));
+        SL_CUDA(cudaStreamWaitEvent(st, c->ev_copied[bsel], 0));
         WorkerPtrs ptrs;
         memset(&ptrs, 0, sizeof(ptrs));
-        ptrs.theta_local[0] = dev_stage;
+        ptrs.theta_local[0] = stage;
         ptrs.e[0] = e ? e[r] : nullptr;
         ptrs.payload[0] = payloads[r];
         sl_status s = launch_compress(c, 1, theta_sync, ptrs, st);
         if (s != SL_OK) return s;
+        SL_CUDA(cudaEventRecord(c->ev_consumed[bsel], st));
         pl.p[r] = payloads[r];
     }
     sl_status s = launch_apply(c, pl, R, theta_sync, st);
@@ -1044,6 +1105,44 @@ sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* t
         SL_CUDA(cudaMemcpyAsync(theta_sync_host, theta_sync, bytes, cudaMemcpyDeviceToHost, st));
     SL_CUDA(cudaStreamSynchronize(st));
     return SL_OK;
+}
+
+sl_status sl_profile_enable(sl_ctx* c, int32_t enable) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    if (enable && c->prof_events.empty()) {
+        c->prof_events.resize((size_t)kProfMaxSeq * (kProfSlots + 1));
+        for (auto& ev : c->prof_events) SL_CUDA(cudaEventCreate(&ev));
+    }
+    c->prof_on = enable != 0;
+    c->prof_steps = 0;
+    return SL_OK;
+}
+
+sl_status sl_profile_read(sl_ctx* c, float* ms_total, int64_t* launches) {
+    if (!c || !ms_total || !launches) return SL_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    for (int i = 0; i < kProfSlots; ++i) { ms_total[i] = 0.0f; launches[i] = 0; }
+    for (int q = 0; q < c->prof_steps; ++q) {
+        cudaEvent_t* ev = &c->prof_events[(size_t)q * (kProfSlots + 1)];
+        SL_CUDA(cudaEventSynchronize(ev[kProfSlots]));
+        for (int i = 0; i < kProfSlots; ++i) {
+            float ms = 0.0f;
+            SL_CUDA(cudaEventElapsedTime(&ms, ev[i], ev[i + 1]));
+            ms_total[i] += ms;
+            launches[i] += 1;
+        }
+    }
+    c->prof_steps = 0;
+    return SL_OK;
+}
+
+const char* sl_profile_name(int32_t slot) {
+    static const char* names[kProfSlots] = {"ef_topk", "chunk_sum", "tensor_mean", "chunk_var", "tensor_sigma",
+                                            "chunk_bins", "tensor_lut", "pack_fix", "decode_avg_apply"};
+    return slot >= 0 && slot < kProfSlots ? names[slot] : "";
 }
 
 sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {
