@@ -93,17 +93,22 @@ __device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Selection: the keff largest of 4096 composites (magnitude, then lower index), exact.
+// Selection: the keff largest of 4096 (magnitude, then lower index), exact.
 //
-// composite = key << 13 | (4095 - p) << 1 | sign, key = float bits without the sign.  All
-// composites of a chunk are distinct, so "the keff largest composites" is exactly the Top-k with
-// the lowest-index tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3.
+// key = float bits without the sign (31 bits); the order is (key descending, index ascending), so
+// every element has a distinct rank and "the keff first" is exactly Top-k with the lowest-index
+// tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3.
 //
 // 1. every lane takes the maximum key of its 16 values; every warp takes the ceil(keff/8)-th
 //    largest of its 32 lane maxima; T = the minimum over the 8 warps.  At least keff values have
 //    key >= T, so nothing below T can be selected.
-// 2. values with key >= T (about 2 k of them on bell-shaped data) go to a shared candidate list.
-// 3. each candidate counts the candidates above it; rank < keff means selected.
+// 2. values with key >= T (about 2 k of them on bell-shaped data) are compacted into a shared
+//    candidate list (ballot + one atomic per warp and round).
+// 3. fast path (<= 256 candidates): every candidate counts the candidate keys strictly above its
+//    own (32-bit arithmetic, four keys per shared load, the pair loop split over all threads).
+//    Candidates with fewer than keff keys above them are tentatively selected; if exactly keff
+//    are, no tie straddles the cut and that is the answer.  Otherwise (or with more candidates)
+//    the general path ranks 64-bit composites (key, 4095 - index), which are all distinct.
 // 4. selected bits are set in a 4096-bit map; a prefix popcount over the map gives every selected
 //    entry its slot in ascending index order.
 // If the list overflows (heavy ties, constant chunks) an exact bitwise search over all 4096
@@ -111,7 +116,9 @@ __device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
 // ------------------------------------------------------------------------------------------------
 
 struct SelectSmem {
-    unsigned long long cand[kCandCap];
+    __align__(16) unsigned ckey[kCandCap + 4];  // candidate keys; zero beyond the last candidate
+    unsigned cinfo[kCandCap];                    // in-chunk index | sign << 12
+    unsigned gt[256];                            // keys strictly above candidate i (fast path)
     unsigned bitmap[128];
     unsigned prefix[128];
     unsigned warp_t[8];
@@ -119,22 +126,93 @@ struct SelectSmem {
     unsigned count;
 };
 
-__device__ __forceinline__ unsigned long long make_composite(unsigned bits, int p) {
-    unsigned key = bits & 0x7FFFFFFFu;
-    return ((unsigned long long)key << 13) | ((unsigned long long)(4095 - p) << 1) | (bits >> 31);
-}
-__device__ __forceinline__ int composite_index(unsigned long long c) { return 4095 - (int)((c >> 1) & 0xFFF); }
-__device__ __forceinline__ unsigned composite_bits(unsigned long long c) {
-    return (unsigned)(c >> 13) | ((unsigned)(c & 1ull) << 31);
+__device__ __forceinline__ unsigned long long make_composite(unsigned key, int p) {
+    return ((unsigned long long)key << 12) | (unsigned long long)(4095 - p);
 }
 
 __device__ __forceinline__ int owned_index(int tid, int q) { return 1024 * (q >> 2) + 4 * tid + (q & 3); }
 
-// Emits the selected (index, value) pairs of the chunk to out_idx / out_val in ascending index
-// order.  `ub` = the thread's 16 value bit patterns; entries with owned index >= len are padding.
-__device__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff, SelectSmem& sm,
-                            uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+// Exact fallback when the candidate list overflows: bitwise search for the keff-th largest
+// composite over all elements, then rebuild the candidate list with exactly the keff winners.
+// Returns the new candidate count (== keff).  Rare path, kept out of line.
+__device__ __noinline__ unsigned select_overflow(const unsigned* ub, bool nonzero, int len, int keff, SelectSmem& sm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long res = 0;
+    const bool any = __syncthreads_or(nonzero);
+    if (any) {
+        int buf = 0;
+        for (int bit = 42; bit >= 0; --bit) {
+            const unsigned long long trial = res | (1ull << bit);
+            unsigned c = 0;
+            for (int q = 0; q < kPerThread; ++q) {
+                const int p = owned_index(tid, q);
+                c += (p < len && make_composite(ub[q] & 0x7FFFFFFFu, p) >= trial) ? 1u : 0u;
+            }
+            c = __reduce_add_sync(kFull, c);
+            if (lane == 0) sm.warp_cnt[buf][warp] = c;
+            __syncthreads();
+            unsigned tot = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) tot += sm.warp_cnt[buf][w];
+            if (tot >= (unsigned)keff) res = trial;
+            buf ^= 1;
+        }
+    } else {
+        // all magnitudes are zero: the first keff indices win every tie
+        res = make_composite(0u, keff - 1);
+    }
+    *reinterpret_cast<uint4*>(&sm.ckey[4 * tid]) = make_uint4(0u, 0u, 0u, 0u);
+    if (tid == 0) sm.count = 0;
+    __syncthreads();
+    for (int q = 0; q < kPerThread; ++q) {
+        const int p = owned_index(tid, q);
+        const unsigned key = ub[q] & 0x7FFFFFFFu;
+        if (p < len && make_composite(key, p) >= res) {
+            const unsigned pos = atomicAdd(&sm.count, 1u);
+            if (pos < kCandCap) {
+                sm.ckey[pos] = key;
+                sm.cinfo[pos] = (unsigned)p | ((ub[q] >> 31) << 12);
+            }
+        }
+    }
+    __syncthreads();
+    return sm.count;
+}
+
+// General ranking: distinct 64-bit composites, any candidate count up to the list capacity.
+// Returns the mask of selected candidates tid + 256 s.  Rare path, kept out of line.
+__device__ __noinline__ unsigned select_rank_general(unsigned M, int keff, const SelectSmem& sm) {
+    const int tid = threadIdx.x;
+    unsigned sel_mask = 0;
+    for (int s = 0; s < kCandCap / kThreads; ++s) {
+        const unsigned i = tid + s * kThreads;
+        if (i < M) {
+            const unsigned long long ci = make_composite(sm.ckey[i], (int)(sm.cinfo[i] & 0xFFFu));
+            unsigned above = 0;
+            for (unsigned j = 0; j < M; ++j)
+                above += (make_composite(sm.ckey[j], (int)(sm.cinfo[j] & 0xFFFu)) > ci) ? 1u : 0u;
+            if (above < (unsigned)keff) sel_mask |= 1u << s;
+        }
+    }
+    return sel_mask;
+}
+
+// Emits the selected (index, value) pairs of the chunk to out_idx / out_val in ascending index
+// order.  `ub` = the thread's 16 value bit patterns; entries with owned index >= len are padding
+// (they must hold 0).  FULL: len == 4096 known at compile time.
+template <bool FULL>
+__device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff, SelectSmem& sm,
+                                            uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // zero the lists this CTA relies on being zero
+    *reinterpret_cast<uint4*>(&sm.ckey[4 * tid]) = make_uint4(0u, 0u, 0u, 0u);
+    sm.gt[tid] = 0;
+    if (tid < 128) sm.bitmap[tid] = 0;
+    if (tid == 0) {
+        sm.count = 0;
+        *reinterpret_cast<uint4*>(&sm.ckey[kCandCap]) = make_uint4(0u, 0u, 0u, 0u);
+    }
 
     // -- 1. threshold
     unsigned m = 0;
@@ -143,124 +221,112 @@ __device__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff,
     {
         const int rounds = (keff + 7) >> 3;  // <= 32
         unsigned cur = m, tw = 0;
-        bool alive = true;
         for (int i = 0; i < rounds; ++i) {
-            tw = __reduce_max_sync(kFull, alive ? cur : 0u);
-            unsigned holders = __ballot_sync(kFull, alive && cur == tw);
-            if (holders == 0) break;  // only zeros remain: tw == 0
-            if (lane == __ffs(holders) - 1) alive = false;
+            tw = __reduce_max_sync(kFull, cur);
+            const unsigned holders = __ballot_sync(kFull, cur == tw);
+            if (tw == 0) break;                          // only zeros remain
+            if (lane == __ffs(holders) - 1) cur = 0;     // retire one holder of the maximum
         }
         if (lane == 0) sm.warp_t[warp] = tw;
     }
-    if (tid < 128) sm.bitmap[tid] = 0;
-    if (tid == 0) sm.count = 0;
     __syncthreads();
     unsigned T = sm.warp_t[0];
 #pragma unroll
     for (int w = 1; w < 8; ++w) T = min(T, sm.warp_t[w]);
 
-    // -- 2. candidates
+    // -- 2. candidates (warp-aggregated compaction)
 #pragma unroll
     for (int q = 0; q < kPerThread; ++q) {
         const int p = owned_index(tid, q);
-        if ((ub[q] & 0x7FFFFFFFu) >= T && p < len) {
-            unsigned pos = atomicAdd(&sm.count, 1u);
-            if (pos < kCandCap) sm.cand[pos] = make_composite(ub[q], p);
+        const unsigned key = ub[q] & 0x7FFFFFFFu;
+        const bool hit = key >= T && (FULL || p < len);
+        const unsigned b = __ballot_sync(kFull, hit);
+        if (b) {
+            unsigned base = 0;
+            if (lane == 0) base = atomicAdd(&sm.count, (unsigned)__popc(b));
+            base = __shfl_sync(kFull, base, 0);
+            const unsigned pos = base + __popc(b & ((1u << lane) - 1u));
+            if (hit && pos < kCandCap) {
+                sm.ckey[pos] = key;
+                sm.cinfo[pos] = (unsigned)p | ((ub[q] >> 31) << 12);
+            }
         }
     }
     __syncthreads();
     unsigned M = sm.count;
 
     if (M > kCandCap) {
-        // -- exact fallback: bitwise search for the keff-th largest composite over all elements
-        unsigned long long res = 0;
-        const bool any = __syncthreads_or(m != 0);
-        if (any) {
-            int buf = 0;
-            for (int bit = 43; bit >= 0; --bit) {
-                const unsigned long long trial = res | (1ull << bit);
-                unsigned c = 0;
+        unsigned tmp[kPerThread];
 #pragma unroll
-                for (int q = 0; q < kPerThread; ++q) {
-                    const int p = owned_index(tid, q);
-                    c += (p < len && make_composite(ub[q], p) >= trial) ? 1u : 0u;
-                }
-                c = __reduce_add_sync(kFull, c);
-                if (lane == 0) sm.warp_cnt[buf][warp] = c;
-                __syncthreads();
-                unsigned tot = 0;
-#pragma unroll
-                for (int w = 0; w < 8; ++w) tot += sm.warp_cnt[buf][w];
-                if (tot >= (unsigned)keff) res = trial;
-                buf ^= 1;
-            }
-        } else {
-            // all magnitudes are zero: the first keff indices win every tie
-            res = make_composite(0u, keff - 1) & ~1ull;
-        }
-        if (tid == 0) sm.count = 0;
-        __syncthreads();
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            const int p = owned_index(tid, q);
-            if (p < len) {
-                const unsigned long long c = make_composite(ub[q], p);
-                if (c >= res) {
-                    unsigned pos = atomicAdd(&sm.count, 1u);
-                    if (pos < kCandCap) sm.cand[pos] = c;
-                }
-            }
-        }
-        __syncthreads();
-        M = sm.count;  // == keff
+        for (int q = 0; q < kPerThread; ++q) tmp[q] = ub[q];
+        M = select_overflow(tmp, m != 0, len, keff, sm);
     }
 
-    // -- 3. rank among candidates (M <= kCandCap: up to 4 candidates per thread)
-    unsigned long long mine[kCandCap / kThreads];
-    unsigned sel_mask = 0;
+    // -- 3. which candidates are selected
+    unsigned sel_mask = 0;  // bit s: candidate tid + 256 s is selected
+    bool settled = false;
+    if (M <= 256) {
+        const unsigned Mp = (M + 31u) & ~31u;
+        const unsigned nseg = Mp ? 256u / Mp : 1u;              // >= 1
+        const unsigned seglen = ((M + nseg - 1) / nseg + 3u) & ~3u;
+        const unsigned seg = tid / Mp, i = tid - seg * Mp;
+        if (seg < nseg && i < M) {
+            const unsigned ki = sm.ckey[i];
+            const unsigned j0 = seg * seglen, j1 = min(j0 + seglen, (M + 3u) & ~3u);
+            unsigned cnt = 0;
+            for (unsigned j = j0; j < j1; j += 4) {
+                const uint4 kk = *reinterpret_cast<const uint4*>(&sm.ckey[j]);
+                // keys are < 2^31, so (ki - kj) has its top bit set exactly when kj > ki
+                cnt += (ki - kk.x) >> 31;
+                cnt += (ki - kk.y) >> 31;
+                cnt += (ki - kk.z) >> 31;
+                cnt += (ki - kk.w) >> 31;
+            }
+            if (nseg > 1) atomicAdd(&sm.gt[i], cnt);
+            else sm.gt[i] = cnt;
+        }
+        __syncthreads();
+        const bool tentative = (unsigned)tid < M && sm.gt[tid] < (unsigned)keff;
+        const int S = __syncthreads_count(tentative);
+        if (S == keff) {
+            settled = true;
+            sel_mask = tentative ? 1u : 0u;
+        }
+    }
+    if (!settled) sel_mask = select_rank_general(M, keff, sm);
 #pragma unroll
     for (int s = 0; s < kCandCap / kThreads; ++s) {
-        const unsigned i = tid + s * kThreads;
-        if (i < M) {
-            const unsigned long long ci = sm.cand[i];
-            mine[s] = ci;
-            unsigned above = 0;
-            for (unsigned j = 0; j < M; ++j) above += (sm.cand[j] > ci) ? 1u : 0u;
-            if (above < (unsigned)keff) {
-                sel_mask |= 1u << s;
-                const int p = composite_index(ci);
-                atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
-            }
+        if (sel_mask & (1u << s)) {
+            const unsigned p = sm.cinfo[tid + s * kThreads] & 0xFFFu;
+            atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
         }
     }
     __syncthreads();
 
     // -- 4. slots from a prefix popcount over the bitmap
     if (warp == 0) {
-        unsigned w0 = sm.bitmap[4 * lane], w1 = sm.bitmap[4 * lane + 1], w2 = sm.bitmap[4 * lane + 2],
-                 w3 = sm.bitmap[4 * lane + 3];
-        unsigned c0 = __popc(w0), c1 = __popc(w1), c2 = __popc(w2), c3 = __popc(w3);
-        unsigned tot = c0 + c1 + c2 + c3, inc = tot;
+        const uint4 w = *reinterpret_cast<const uint4*>(&sm.bitmap[4 * lane]);
+        const unsigned c0 = __popc(w.x), c1 = __popc(w.y), c2 = __popc(w.z), c3 = __popc(w.w);
+        const unsigned tot = c0 + c1 + c2 + c3;
+        unsigned inc = tot;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            unsigned o = __shfl_up_sync(kFull, inc, d);
+            const unsigned o = __shfl_up_sync(kFull, inc, d);
             if (lane >= d) inc += o;
         }
-        unsigned ex = inc - tot;
-        sm.prefix[4 * lane] = ex;
-        sm.prefix[4 * lane + 1] = ex + c0;
-        sm.prefix[4 * lane + 2] = ex + c0 + c1;
-        sm.prefix[4 * lane + 3] = ex + c0 + c1 + c2;
+        const unsigned ex = inc - tot;
+        *reinterpret_cast<uint4*>(&sm.prefix[4 * lane]) = make_uint4(ex, ex + c0, ex + c0 + c1, ex + c0 + c1 + c2);
     }
     __syncthreads();
 #pragma unroll
     for (int s = 0; s < kCandCap / kThreads; ++s) {
         if (sel_mask & (1u << s)) {
-            const int p = composite_index(mine[s]);
+            const unsigned info = sm.cinfo[tid + s * kThreads], key = sm.ckey[tid + s * kThreads];
+            const unsigned p = info & 0xFFFu;
             const unsigned slot = sm.prefix[p >> 5] + __popc(sm.bitmap[p >> 5] & ((1u << (p & 31)) - 1u));
             if (slot < (unsigned)keff) {
                 out_idx[slot] = (uint16_t)p;
-                out_val[slot] = __uint_as_float(composite_bits(mine[s]));
+                out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
             }
         }
     }
@@ -272,7 +338,7 @@ __device__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff,
 // theta_sync is fetched from HBM once and served to the other workers from L2.
 // ------------------------------------------------------------------------------------------------
 template <bool EF>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp,
                float beta, const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
     __shared__ SelectSmem sm;
@@ -287,39 +353,41 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
 
     unsigned ub[kPerThread];
     if (cd.len == kChunk) {
-        long long off[4];
+        // two halves of 2 x float4 per array: fewer registers held by loads in flight
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int p = 1024 * i + 4 * tid;
-            off[i] = chunk_elem_offset(cd.row_stride, p);
-        }
-        float4 a[4], l[4], ev[4];
+        for (int h = 0; h < 2; ++h) {
+            long long off[2];
+            float4 a[2], l[2], ev[2];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a[i] = __ldg(reinterpret_cast<const float4*>(ts + off[i]));
+            for (int i = 0; i < 2; ++i) off[i] = chunk_elem_offset(cd.row_stride, 1024 * (2 * h + i) + 4 * tid);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) l[i] = __ldcs(reinterpret_cast<const float4*>(tl + off[i]));
-        if (EF) {
+            for (int i = 0; i < 2; ++i) a[i] = __ldg(reinterpret_cast<const float4*>(ts + off[i]));
 #pragma unroll
-            for (int i = 0; i < 4; ++i) ev[i] = __ldcs(reinterpret_cast<const float4*>(er + off[i]));
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float4 u;
-            u.x = __fsub_rn(a[i].x, l[i].x);
-            u.y = __fsub_rn(a[i].y, l[i].y);
-            u.z = __fsub_rn(a[i].z, l[i].z);
-            u.w = __fsub_rn(a[i].w, l[i].w);
+            for (int i = 0; i < 2; ++i) l[i] = __ldcs(reinterpret_cast<const float4*>(tl + off[i]));
             if (EF) {
-                u.x = __fmaf_rn(beta, ev[i].x, u.x);
-                u.y = __fmaf_rn(beta, ev[i].y, u.y);
-                u.z = __fmaf_rn(beta, ev[i].z, u.z);
-                u.w = __fmaf_rn(beta, ev[i].w, u.w);
-                *reinterpret_cast<float4*>(er + off[i]) = u;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) ev[i] = __ldcs(reinterpret_cast<const float4*>(er + off[i]));
             }
-            ub[4 * i + 0] = __float_as_uint(u.x);
-            ub[4 * i + 1] = __float_as_uint(u.y);
-            ub[4 * i + 2] = __float_as_uint(u.z);
-            ub[4 * i + 3] = __float_as_uint(u.w);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                float4 u;
+                u.x = __fsub_rn(a[i].x, l[i].x);
+                u.y = __fsub_rn(a[i].y, l[i].y);
+                u.z = __fsub_rn(a[i].z, l[i].z);
+                u.w = __fsub_rn(a[i].w, l[i].w);
+                if (EF) {
+                    u.x = __fmaf_rn(beta, ev[i].x, u.x);
+                    u.y = __fmaf_rn(beta, ev[i].y, u.y);
+                    u.z = __fmaf_rn(beta, ev[i].z, u.z);
+                    u.w = __fmaf_rn(beta, ev[i].w, u.w);
+                    *reinterpret_cast<float4*>(er + off[i]) = u;
+                }
+                const int q0 = 4 * (2 * h + i);
+                ub[q0 + 0] = __float_as_uint(u.x);
+                ub[q0 + 1] = __float_as_uint(u.y);
+                ub[q0 + 2] = __float_as_uint(u.z);
+                ub[q0 + 3] = __float_as_uint(u.w);
+            }
         }
     } else {  // short tail of a flat tensor: element-wise with bounds
 #pragma unroll
@@ -339,7 +407,10 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
 
     const int keff = min(k, cd.len);
     const long long slot_base = ((long long)r * n_chunks + g) * kp;
-    select_topk(ub, cd.len, keff, sm, ws.idx + slot_base, ws.val + slot_base);
+    if (cd.len == kChunk)
+        select_topk<true>(ub, kChunk, keff, sm, ws.idx + slot_base, ws.val + slot_base);
+    else
+        select_topk<false>(ub, cd.len, keff, sm, ws.idx + slot_base, ws.val + slot_base);
 }
 
 // ------------------------------------------------------------------------------------------------
