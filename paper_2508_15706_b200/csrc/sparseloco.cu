@@ -118,7 +118,6 @@ __device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
 struct SelectSmem {
     __align__(16) unsigned ckey[kCandCap + 4];  // candidate keys; zero beyond the last candidate
     unsigned cinfo[kCandCap];                    // in-chunk index | sign << 12
-    unsigned gt[256];                            // keys strictly above candidate i (fast path)
     unsigned bitmap[128];
     unsigned prefix[128];
     unsigned warp_t[8];
@@ -197,6 +196,32 @@ __device__ __noinline__ unsigned select_rank_general(unsigned M, int keff, const
     return sel_mask;
 }
 
+// Writes one selected candidate to its slot.  `pack` = this lane's packed bitmap prefix
+// (exclusive count before its 4 words | popcounts of its first three words); every lane of the
+// warp must call this together (shuffle inside).
+__device__ __forceinline__ void emit_candidate(bool active, unsigned cand, unsigned pack, int keff, const SelectSmem& sm,
+                                               uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    unsigned info = 0, key = 0;
+    if (active) {
+        info = sm.cinfo[cand];
+        key = sm.ckey[cand];
+    }
+    const unsigned p = info & 0xFFFu, w = p >> 5;
+    const unsigned pk = __shfl_sync(kFull, pack, w >> 2);
+    if (active) {
+        const unsigned sub = w & 3u;
+        unsigned before = pk & 0x1FFFu;
+        if (sub > 0) before += (pk >> 13) & 0x3Fu;
+        if (sub > 1) before += (pk >> 19) & 0x3Fu;
+        if (sub > 2) before += (pk >> 25) & 0x3Fu;
+        const unsigned slot = before + __popc(sm.bitmap[w] & ((1u << (p & 31)) - 1u));
+        if (slot < (unsigned)keff) {
+            out_idx[slot] = (uint16_t)p;
+            out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
+        }
+    }
+}
+
 // Emits the selected (index, value) pairs of the chunk to out_idx / out_val in ascending index
 // order.  `ub` = the thread's 16 value bit patterns; entries with owned index >= len are padding
 // (they must hold 0).  FULL: len == 4096 known at compile time.
@@ -207,7 +232,6 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
 
     // zero the lists this CTA relies on being zero
     *reinterpret_cast<uint4*>(&sm.ckey[4 * tid]) = make_uint4(0u, 0u, 0u, 0u);
-    sm.gt[tid] = 0;
     if (tid < 128) sm.bitmap[tid] = 0;
     if (tid == 0) {
         sm.count = 0;
@@ -234,21 +258,33 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
 #pragma unroll
     for (int w = 1; w < 8; ++w) T = min(T, sm.warp_t[w]);
 
-    // -- 2. candidates (warp-aggregated compaction)
+    // -- 2. candidates: per-thread hit mask, warp scan, one atomic per warp, then the writes
+    {
+        unsigned hits = 0;
 #pragma unroll
-    for (int q = 0; q < kPerThread; ++q) {
-        const int p = owned_index(tid, q);
-        const unsigned key = ub[q] & 0x7FFFFFFFu;
-        const bool hit = key >= T && (FULL || p < len);
-        const unsigned b = __ballot_sync(kFull, hit);
-        if (b) {
-            unsigned base = 0;
-            if (lane == 0) base = atomicAdd(&sm.count, (unsigned)__popc(b));
-            base = __shfl_sync(kFull, base, 0);
-            const unsigned pos = base + __popc(b & ((1u << lane) - 1u));
-            if (hit && pos < kCandCap) {
-                sm.ckey[pos] = key;
-                sm.cinfo[pos] = (unsigned)p | ((ub[q] >> 31) << 12);
+        for (int q = 0; q < kPerThread; ++q) {
+            const bool hit = (ub[q] & 0x7FFFFFFFu) >= T && (FULL || owned_index(tid, q) < len);
+            hits |= hit ? (1u << q) : 0u;
+        }
+        const unsigned mine = __popc(hits);
+        unsigned inc = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned o = __shfl_up_sync(kFull, inc, d);
+            if (lane >= d) inc += o;
+        }
+        unsigned base = 0;
+        if (lane == 31 && inc) base = atomicAdd(&sm.count, inc);
+        base = __shfl_sync(kFull, base, 31);
+        unsigned pos = base + inc - mine;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            if (hits & (1u << q)) {
+                if (pos < kCandCap) {
+                    sm.ckey[pos] = ub[q] & 0x7FFFFFFFu;
+                    sm.cinfo[pos] = (unsigned)owned_index(tid, q) | ((ub[q] >> 31) << 12);
+                }
+                ++pos;
             }
         }
     }
@@ -263,17 +299,19 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
     }
 
     // -- 3. which candidates are selected
-    unsigned sel_mask = 0;  // bit s: candidate tid + 256 s is selected
     bool settled = false;
+    unsigned my_cand = 0;
+    bool owner = false;
     if (M <= 256) {
-        const unsigned Mp = (M + 31u) & ~31u;
-        const unsigned nseg = Mp ? 256u / Mp : 1u;              // >= 1
+        // candidate i = tid / nseg is counted by nseg adjacent lanes, each over one segment of the list
+        unsigned nseg = 1;
+        while (nseg < 8 && M * (nseg * 2) <= 256u) nseg *= 2;
+        const unsigned i = tid / nseg, seg = tid & (nseg - 1);
         const unsigned seglen = ((M + nseg - 1) / nseg + 3u) & ~3u;
-        const unsigned seg = tid / Mp, i = tid - seg * Mp;
-        if (seg < nseg && i < M) {
+        unsigned cnt = 0;
+        if (i < M) {
             const unsigned ki = sm.ckey[i];
             const unsigned j0 = seg * seglen, j1 = min(j0 + seglen, (M + 3u) & ~3u);
-            unsigned cnt = 0;
             for (unsigned j = j0; j < j1; j += 4) {
                 const uint4 kk = *reinterpret_cast<const uint4*>(&sm.ckey[j]);
                 // keys are < 2^31, so (ki - kj) has its top bit set exactly when kj > ki
@@ -282,29 +320,37 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
                 cnt += (ki - kk.z) >> 31;
                 cnt += (ki - kk.w) >> 31;
             }
-            if (nseg > 1) atomicAdd(&sm.gt[i], cnt);
-            else sm.gt[i] = cnt;
         }
-        __syncthreads();
-        const bool tentative = (unsigned)tid < M && sm.gt[tid] < (unsigned)keff;
-        const int S = __syncthreads_count(tentative);
-        if (S == keff) {
-            settled = true;
-            sel_mask = tentative ? 1u : 0u;
-        }
-    }
-    if (!settled) sel_mask = select_rank_general(M, keff, sm);
-#pragma unroll
-    for (int s = 0; s < kCandCap / kThreads; ++s) {
-        if (sel_mask & (1u << s)) {
-            const unsigned p = sm.cinfo[tid + s * kThreads] & 0xFFFu;
+        for (unsigned d = 1; d < nseg; d <<= 1) cnt += __shfl_xor_sync(kFull, cnt, d);
+        owner = i < M && seg == 0 && cnt < (unsigned)keff;
+        my_cand = i;
+        if (owner) {  // speculative: right unless a tie group straddles the cut
+            const unsigned p = sm.cinfo[i] & 0xFFFu;
             atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
         }
+        const int S = __syncthreads_count(owner);
+        settled = S == keff;
+        if (!settled) {
+            if (tid < 128) sm.bitmap[tid] = 0;
+            __syncthreads();
+        }
     }
-    __syncthreads();
+    unsigned sel_mask = 0;  // general path: bit s = candidate tid + 256 s is selected
+    if (!settled) {
+        sel_mask = select_rank_general(M, keff, sm);
+#pragma unroll
+        for (int s = 0; s < kCandCap / kThreads; ++s) {
+            if (sel_mask & (1u << s)) {
+                const unsigned p = sm.cinfo[tid + s * kThreads] & 0xFFFu;
+                atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
+            }
+        }
+        __syncthreads();
+    }
 
-    // -- 4. slots from a prefix popcount over the bitmap
-    if (warp == 0) {
+    // -- 4. slots from a prefix popcount over the bitmap (every warp computes its own copy)
+    unsigned pack;
+    {
         const uint4 w = *reinterpret_cast<const uint4*>(&sm.bitmap[4 * lane]);
         const unsigned c0 = __popc(w.x), c1 = __popc(w.y), c2 = __popc(w.z), c3 = __popc(w.w);
         const unsigned tot = c0 + c1 + c2 + c3;
@@ -314,21 +360,14 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
             const unsigned o = __shfl_up_sync(kFull, inc, d);
             if (lane >= d) inc += o;
         }
-        const unsigned ex = inc - tot;
-        *reinterpret_cast<uint4*>(&sm.prefix[4 * lane]) = make_uint4(ex, ex + c0, ex + c0 + c1, ex + c0 + c1 + c2);
+        pack = (inc - tot) | (c0 << 13) | (c1 << 19) | (c2 << 25);
     }
-    __syncthreads();
-#pragma unroll
-    for (int s = 0; s < kCandCap / kThreads; ++s) {
-        if (sel_mask & (1u << s)) {
-            const unsigned info = sm.cinfo[tid + s * kThreads], key = sm.ckey[tid + s * kThreads];
-            const unsigned p = info & 0xFFFu;
-            const unsigned slot = sm.prefix[p >> 5] + __popc(sm.bitmap[p >> 5] & ((1u << (p & 31)) - 1u));
-            if (slot < (unsigned)keff) {
-                out_idx[slot] = (uint16_t)p;
-                out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
-            }
-        }
+    if (settled) {
+        emit_candidate(owner, my_cand, pack, keff, sm, out_idx, out_val);
+    } else {
+#pragma unroll 1
+        for (int s = 0; s < kCandCap / kThreads; ++s)
+            emit_candidate((sel_mask >> s) & 1u, tid + s * kThreads, pack, keff, sm, out_idx, out_val);
     }
 }
 
