@@ -32,7 +32,6 @@ constexpr int kThreads = 256;          // threads per CTA of the chunk kernels
 constexpr int kPerThread = kChunk / kThreads;  // 16 elements = 4 x float4
 constexpr int kMaxR = 64;
 constexpr int kMaxK = 256;
-constexpr int kCandCap = 1024;         // candidate list capacity of the selection
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kProfSlots = 9;     // kernels of one outer step
 constexpr int kProfMaxSeq = 256;  // recorded sequences kept between two reads
@@ -93,36 +92,50 @@ __device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Asynchronous 16-byte copies global -> shared (one per thread and vector), grouped per unit.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's committed groups are still in flight
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
 // Selection: the keff largest of 4096 (magnitude, then lower index), exact.
 //
 // key = float bits without the sign (31 bits); the order is (key descending, index ascending), so
 // every element has a distinct rank and "the keff first" is exactly Top-k with the lowest-index
-// tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3.
+// tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3; its 16 values are
+// in registers and, for indexing by a run-time position, in its own slots of a shared tile.
 //
 // 1. every lane takes the maximum key of its 16 values; every warp takes the ceil(keff/8)-th
-//    largest of its 32 lane maxima; T = the minimum over the 8 warps.  At least keff values have
-//    key >= T, so nothing below T can be selected.
-// 2. values with key >= T (about 2 k of them on bell-shaped data) are compacted into a shared
-//    candidate list (ballot + one atomic per warp and round).
-// 3. fast path (<= 256 candidates): every candidate counts the candidate keys strictly above its
-//    own (32-bit arithmetic, four keys per shared load, the pair loop split over all threads).
-//    Candidates with fewer than keff keys above them are tentatively selected; if exactly keff
-//    are, no tie straddles the cut and that is the answer.  Otherwise (or with more candidates)
-//    the general path ranks 64-bit composites (key, 4095 - index), which are all distinct.
-// 4. selected bits are set in a 4096-bit map; a prefix popcount over the map gives every selected
-//    entry its slot in ascending index order.
-// If the list overflows (heavy ties, constant chunks) an exact bitwise search over all 4096
-// composites finds the keff-th largest instead.
+//    largest of its 32 lane maxima (low 5 bits replaced by the lane number, so that the maxima
+//    are distinct and one reduction per round suffices); T = the minimum over the 8 warps,
+//    rounded down to a multiple of 32.  At least keff values have key >= T.
+// 2. the 8 warp values cluster around the keff-th largest key, so three splitters between their
+//    minimum and maximum cut the candidates (key >= T, about 2 keff of them) into four classes.
+//    Every candidate is appended to its class list; the class counts say which class holds the
+//    cut: classes above it are selected whole, and only that class (some tens of entries) is
+//    ranked, by all-pairs counting on (key, index).
+// 3. selected entries set their bit in a 4096-bit map; a prefix popcount over the map gives every
+//    selected entry its slot in ascending index order, and its owner writes (index, value).
+// If T is 0 or a class list overflows (constant chunks, heavy ties, large k) an exact bitwise
+// search over all 4096 (key, index) composites finds the keff-th largest instead.
 // ------------------------------------------------------------------------------------------------
+constexpr int kClassCap = 256;  // entries per class list (= threads: one thread per entry suffices)
 
 struct SelectSmem {
-    __align__(16) unsigned ckey[kCandCap + 4];  // candidate keys; zero beyond the last candidate
-    unsigned cinfo[kCandCap];                    // in-chunk index | sign << 12
-    unsigned bitmap[128];
-    unsigned prefix[128];
+    uint2 list[4][kClassCap];  // (key, in-chunk index | sign << 12) per class
+    unsigned bitmap[2][128];   // selected positions, double-buffered by unit parity
     unsigned warp_t[8];
+    unsigned cnt[4];
     unsigned warp_cnt[2][8];
-    unsigned count;
+    unsigned n_exact;          // entries the exact search appended to list[0]
 };
 
 __device__ __forceinline__ unsigned long long make_composite(unsigned key, int p) {
@@ -131,12 +144,16 @@ __device__ __forceinline__ unsigned long long make_composite(unsigned key, int p
 
 __device__ __forceinline__ int owned_index(int tid, int q) { return 1024 * (q >> 2) + 4 * tid + (q & 3); }
 
-// Exact fallback when the candidate list overflows: bitwise search for the keff-th largest
-// composite over all elements, then rebuild the candidate list with exactly the keff winners.
-// Returns the new candidate count (== keff).  Rare path, kept out of line.
-__device__ __noinline__ unsigned select_overflow(const unsigned* ub, bool nonzero, int len, int keff, SelectSmem& sm) {
+__device__ __forceinline__ void set_bit(unsigned* bitmap, unsigned p) { atomicOr(&bitmap[p >> 5], 1u << (p & 31)); }
+
+// Exact fallback: bitwise search for the keff-th largest composite over all elements; the keff
+// elements at or above it are appended to list[0] (count in n_exact) and marked in the map.
+// Contains CTA barriers.  Rare path, kept out of line.
+__device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzero, int len, int keff,
+                                                 SelectSmem& sm, unsigned* bitmap) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long res = 0;
+    if (tid == 0) sm.n_exact = 0;
     const bool any = __syncthreads_or(nonzero);
     if (any) {
         int buf = 0;
@@ -160,83 +177,32 @@ __device__ __noinline__ unsigned select_overflow(const unsigned* ub, bool nonzer
         // all magnitudes are zero: the first keff indices win every tie
         res = make_composite(0u, keff - 1);
     }
-    *reinterpret_cast<uint4*>(&sm.ckey[4 * tid]) = make_uint4(0u, 0u, 0u, 0u);
-    if (tid == 0) sm.count = 0;
-    __syncthreads();
     for (int q = 0; q < kPerThread; ++q) {
         const int p = owned_index(tid, q);
         const unsigned key = ub[q] & 0x7FFFFFFFu;
         if (p < len && make_composite(key, p) >= res) {
-            const unsigned pos = atomicAdd(&sm.count, 1u);
-            if (pos < kCandCap) {
-                sm.ckey[pos] = key;
-                sm.cinfo[pos] = (unsigned)p | ((ub[q] >> 31) << 12);
-            }
-        }
-    }
-    __syncthreads();
-    return sm.count;
-}
-
-// General ranking: distinct 64-bit composites, any candidate count up to the list capacity.
-// Returns the mask of selected candidates tid + 256 s.  Rare path, kept out of line.
-__device__ __noinline__ unsigned select_rank_general(unsigned M, int keff, const SelectSmem& sm) {
-    const int tid = threadIdx.x;
-    unsigned sel_mask = 0;
-    for (int s = 0; s < kCandCap / kThreads; ++s) {
-        const unsigned i = tid + s * kThreads;
-        if (i < M) {
-            const unsigned long long ci = make_composite(sm.ckey[i], (int)(sm.cinfo[i] & 0xFFFu));
-            unsigned above = 0;
-            for (unsigned j = 0; j < M; ++j)
-                above += (make_composite(sm.ckey[j], (int)(sm.cinfo[j] & 0xFFFu)) > ci) ? 1u : 0u;
-            if (above < (unsigned)keff) sel_mask |= 1u << s;
-        }
-    }
-    return sel_mask;
-}
-
-// Writes one selected candidate to its slot.  `pack` = this lane's packed bitmap prefix
-// (exclusive count before its 4 words | popcounts of its first three words); every lane of the
-// warp must call this together (shuffle inside).
-__device__ __forceinline__ void emit_candidate(bool active, unsigned cand, unsigned pack, int keff, const SelectSmem& sm,
-                                               uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
-    unsigned info = 0, key = 0;
-    if (active) {
-        info = sm.cinfo[cand];
-        key = sm.ckey[cand];
-    }
-    const unsigned p = info & 0xFFFu, w = p >> 5;
-    const unsigned pk = __shfl_sync(kFull, pack, w >> 2);
-    if (active) {
-        const unsigned sub = w & 3u;
-        unsigned before = pk & 0x1FFFu;
-        if (sub > 0) before += (pk >> 13) & 0x3Fu;
-        if (sub > 1) before += (pk >> 19) & 0x3Fu;
-        if (sub > 2) before += (pk >> 25) & 0x3Fu;
-        const unsigned slot = before + __popc(sm.bitmap[w] & ((1u << (p & 31)) - 1u));
-        if (slot < (unsigned)keff) {
-            out_idx[slot] = (uint16_t)p;
-            out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
+            const unsigned pos = atomicAdd(&sm.n_exact, 1u);
+            if (pos < kClassCap) sm.list[0][pos] = make_uint2(key, (unsigned)p | ((ub[q] >> 31) << 12));
+            set_bit(bitmap, (unsigned)p);
         }
     }
 }
 
-// Emits the selected (index, value) pairs of the chunk to out_idx / out_val in ascending index
-// order.  `ub` = the thread's 16 value bit patterns; entries with owned index >= len are padding
-// (they must hold 0).  FULL: len == 4096 known at compile time.
-template <bool FULL>
-__device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], int len, int keff, SelectSmem& sm,
-                                            uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+// A thread's selected entries: up to four (one of the cut class, one per class above the cut).
+struct Picked {
+    uint2 e0, e1, e2, e3;  // (key, in-chunk index | sign << 12): cut class, classes 3, 2, 1
+    unsigned mask;         // bit i: entry i is selected
+};
+
+// First half of the selection: threshold and class lists.  `ub` = the thread's 16 value bit patterns
+// (0 at in-chunk indices >= the chunk length); `tile` = the shared tile holding the same values (only
+// the thread's own slots are read).  Contains one CTA barrier: every thread of the CTA must call
+// it, and must synchronise again before select_rank().  Returns true when the threshold is 0, in
+// which case nothing was listed and the exact search has to run instead.
+__device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], const unsigned* __restrict__ tile,
+                                            int keff, SelectSmem& sm, Picked& out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    // zero the lists this CTA relies on being zero
-    *reinterpret_cast<uint4*>(&sm.ckey[4 * tid]) = make_uint4(0u, 0u, 0u, 0u);
-    if (tid < 128) sm.bitmap[tid] = 0;
-    if (tid == 0) {
-        sm.count = 0;
-        *reinterpret_cast<uint4*>(&sm.ckey[kCandCap]) = make_uint4(0u, 0u, 0u, 0u);
-    }
+    out.mask = 0;
 
     // -- 1. threshold
     unsigned m = 0;
@@ -244,114 +210,105 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
     for (int q = 0; q < kPerThread; ++q) m = max(m, ub[q] & 0x7FFFFFFFu);
     {
         const int rounds = (keff + 7) >> 3;  // <= 32
-        unsigned cur = m, tw = 0;
+        unsigned cur = (m & ~31u) | (unsigned)lane, tw = 0;
         for (int i = 0; i < rounds; ++i) {
             tw = __reduce_max_sync(kFull, cur);
-            const unsigned holders = __ballot_sync(kFull, cur == tw);
-            if (tw == 0) break;                          // only zeros remain
-            if (lane == __ffs(holders) - 1) cur = 0;     // retire one holder of the maximum
+            cur = cur == tw ? 0u : cur;  // retire the holder (tagged values are distinct, or all 0)
         }
-        if (lane == 0) sm.warp_t[warp] = tw;
+        if (lane == 0) sm.warp_t[warp] = tw & ~31u;
+        if (tid < 4) sm.cnt[tid] = 0;
     }
     __syncthreads();
-    unsigned T = sm.warp_t[0];
-#pragma unroll
-    for (int w = 1; w < 8; ++w) T = min(T, sm.warp_t[w]);
-
-    // -- 2. candidates: per-thread hit mask, warp scan, one atomic per warp, then the writes
+    unsigned T, s1, s2, s3;
     {
+        const uint4 a = *reinterpret_cast<const uint4*>(&sm.warp_t[0]);
+        const uint4 b = *reinterpret_cast<const uint4*>(&sm.warp_t[4]);
+        const unsigned lo = min(min(min(a.x, a.y), min(a.z, a.w)), min(min(b.x, b.y), min(b.z, b.w)));
+        const unsigned hi = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w)));
+        const unsigned mean = (a.x >> 3) + (a.y >> 3) + (a.z >> 3) + (a.w >> 3) + (b.x >> 3) + (b.y >> 3) +
+                              (b.z >> 3) + (b.w >> 3);
+        T = lo;
+        s2 = max(mean, lo);
+        s1 = (lo >> 1) + (s2 >> 1);
+        s3 = (s2 >> 1) + (hi >> 1);
+    }
+
+    bool exact = T == 0;  // uniform over the CTA
+    if (!exact) {
+        // -- 2. candidates into class lists.  (T - 1 - key) has its top bit set exactly when key >= T.
         unsigned hits = 0;
+        const unsigned tm1 = T - 1u;
 #pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            const bool hit = (ub[q] & 0x7FFFFFFFu) >= T && (FULL || owned_index(tid, q) < len);
-            hits |= hit ? (1u << q) : 0u;
-        }
-        const unsigned mine = __popc(hits);
-        unsigned inc = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned o = __shfl_up_sync(kFull, inc, d);
-            if (lane >= d) inc += o;
-        }
-        unsigned base = 0;
-        if (lane == 31 && inc) base = atomicAdd(&sm.count, inc);
-        base = __shfl_sync(kFull, base, 31);
-        unsigned pos = base + inc - mine;
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            if (hits & (1u << q)) {
-                if (pos < kCandCap) {
-                    sm.ckey[pos] = ub[q] & 0x7FFFFFFFu;
-                    sm.cinfo[pos] = (unsigned)owned_index(tid, q) | ((ub[q] >> 31) << 12);
-                }
-                ++pos;
-            }
+        for (int q = 0; q < kPerThread; ++q) hits = __funnelshift_l(tm1 - (ub[q] & 0x7FFFFFFFu), hits, 1);  // bit 15 - q
+        while (hits) {
+            const int b = 31 - __clz(hits);
+            hits &= ~(1u << b);
+            const int p = owned_index(tid, 15 - b);
+            const unsigned bits = tile[p];
+            const unsigned kq = bits & 0x7FFFFFFFu;
+            const unsigned cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
+            const unsigned pos = atomicAdd(&sm.cnt[cls], 1u);
+            if (pos < kClassCap) sm.list[cls][pos] = make_uint2(kq, (unsigned)p | ((bits >> 31) << 12));
         }
     }
-    __syncthreads();
-    unsigned M = sm.count;
+    return exact;
+}
 
-    if (M > kCandCap) {
-        unsigned tmp[kPerThread];
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) tmp[q] = ub[q];
-        M = select_overflow(tmp, m != 0, len, keff, sm);
+// Second half of the selection, after the barrier that completes the class lists.
+__device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* bitmap, Picked& out) {
+    const int tid = threadIdx.x;
+    const uint4 cn = *reinterpret_cast<const uint4*>(&sm.cnt[0]);
+    // the class holding the cut: the highest class c with count(classes >= c) >= keff
+    unsigned above = 0, cstar = 3, L = cn.w;
+    if (cn.w < (unsigned)keff) {
+        above = cn.w; cstar = 2; L = cn.z;
+        if (above + cn.z < (unsigned)keff) {
+            above += cn.z; cstar = 1; L = cn.y;
+            if (above + cn.y < (unsigned)keff) { above += cn.y; cstar = 0; L = cn.x; }
+        }
     }
+    if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)kClassCap) return true;  // overflow: exact search
+    const unsigned want = (unsigned)keff - above;  // 1 <= want <= L
+    // classes above the cut: selected whole, one entry per thread
+    if (cstar < 3 && tid < (int)cn.w) { out.e1 = sm.list[3][tid]; out.mask |= 2u; set_bit(bitmap, out.e1.y & 0xFFFu); }
+    if (cstar < 2 && tid < (int)cn.z) { out.e2 = sm.list[2][tid]; out.mask |= 4u; set_bit(bitmap, out.e2.y & 0xFFFu); }
+    if (cstar < 1 && tid < (int)cn.y) { out.e3 = sm.list[1][tid]; out.mask |= 8u; set_bit(bitmap, out.e3.y & 0xFFFu); }
+    // the cut class: entry i = tid / nseg is ranked by nseg adjacent lanes, each over one segment
+    const uint2* __restrict__ lst = sm.list[cstar];
+    unsigned nseg = 1;
+    while (nseg < 8 && L * (nseg * 2) <= 64u) nseg *= 2;
+    const unsigned i = tid / nseg, seg = tid & (nseg - 1);
+    const unsigned seglen = (L + nseg - 1) / nseg;
+    unsigned beat = 0;
+    uint2 me = make_uint2(0u, 0u);
+    if (i < L) {
+        me = lst[i];
+        const unsigned mp = me.y & 0xFFFu;
+        const unsigned j0 = seg * seglen, j1 = min(j0 + seglen, L);
+        for (unsigned j = j0; j < j1; ++j) {
+            const uint2 o = lst[j];
+            beat += (o.x > me.x || (o.x == me.x && (o.y & 0xFFFu) < mp)) ? 1u : 0u;
+        }
+    }
+    for (unsigned d = 1; d < nseg; d <<= 1) beat += __shfl_xor_sync(kFull, beat, d);
+    if (i < L && seg == 0 && beat < want) {
+        out.e0 = me;
+        out.mask |= 1u;
+        set_bit(bitmap, me.y & 0xFFFu);
+    }
+    return false;
+}
 
-    // -- 3. which candidates are selected
-    bool settled = false;
-    unsigned my_cand = 0;
-    bool owner = false;
-    if (M <= 256) {
-        // candidate i = tid / nseg is counted by nseg adjacent lanes, each over one segment of the list
-        unsigned nseg = 1;
-        while (nseg < 8 && M * (nseg * 2) <= 256u) nseg *= 2;
-        const unsigned i = tid / nseg, seg = tid & (nseg - 1);
-        const unsigned seglen = ((M + nseg - 1) / nseg + 3u) & ~3u;
-        unsigned cnt = 0;
-        if (i < M) {
-            const unsigned ki = sm.ckey[i];
-            const unsigned j0 = seg * seglen, j1 = min(j0 + seglen, (M + 3u) & ~3u);
-            for (unsigned j = j0; j < j1; j += 4) {
-                const uint4 kk = *reinterpret_cast<const uint4*>(&sm.ckey[j]);
-                // keys are < 2^31, so (ki - kj) has its top bit set exactly when kj > ki
-                cnt += (ki - kk.x) >> 31;
-                cnt += (ki - kk.y) >> 31;
-                cnt += (ki - kk.z) >> 31;
-                cnt += (ki - kk.w) >> 31;
-            }
-        }
-        for (unsigned d = 1; d < nseg; d <<= 1) cnt += __shfl_xor_sync(kFull, cnt, d);
-        owner = i < M && seg == 0 && cnt < (unsigned)keff;
-        my_cand = i;
-        if (owner) {  // speculative: right unless a tie group straddles the cut
-            const unsigned p = sm.cinfo[i] & 0xFFFu;
-            atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
-        }
-        const int S = __syncthreads_count(owner);
-        settled = S == keff;
-        if (!settled) {
-            if (tid < 128) sm.bitmap[tid] = 0;
-            __syncthreads();
-        }
-    }
-    unsigned sel_mask = 0;  // general path: bit s = candidate tid + 256 s is selected
-    if (!settled) {
-        sel_mask = select_rank_general(M, keff, sm);
-#pragma unroll
-        for (int s = 0; s < kCandCap / kThreads; ++s) {
-            if (sel_mask & (1u << s)) {
-                const unsigned p = sm.cinfo[tid + s * kThreads] & 0xFFFu;
-                atomicOr(&sm.bitmap[p >> 5], 1u << (p & 31));
-            }
-        }
-        __syncthreads();
-    }
-
-    // -- 4. slots from a prefix popcount over the bitmap (every warp computes its own copy)
+// Writes the thread's selected entries to their slots (ascending in-chunk index).  Every lane of a
+// warp must call this together.  Reads the completed map.
+__device__ __forceinline__ void emit_picked(const Picked& pk, const unsigned* __restrict__ bitmap, int keff,
+                                            uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    const int lane = threadIdx.x & 31;
+    if (!__any_sync(kFull, pk.mask != 0)) return;
+    // this lane's packed prefix: exclusive count before its 4 words | popcounts of its first three words
     unsigned pack;
     {
-        const uint4 w = *reinterpret_cast<const uint4*>(&sm.bitmap[4 * lane]);
+        const uint4 w = *reinterpret_cast<const uint4*>(&bitmap[4 * lane]);
         const unsigned c0 = __popc(w.x), c1 = __popc(w.y), c2 = __popc(w.z), c3 = __popc(w.w);
         const unsigned tot = c0 + c1 + c2 + c3;
         unsigned inc = tot;
@@ -362,94 +319,226 @@ __device__ __forceinline__ void select_topk(const unsigned (&ub)[kPerThread], in
         }
         pack = (inc - tot) | (c0 << 13) | (c1 << 19) | (c2 << 25);
     }
-    if (settled) {
-        emit_candidate(owner, my_cand, pack, keff, sm, out_idx, out_val);
-    } else {
-#pragma unroll 1
-        for (int s = 0; s < kCandCap / kThreads; ++s)
-            emit_candidate((sel_mask >> s) & 1u, tid + s * kThreads, pack, keff, sm, out_idx, out_val);
-    }
+    auto write_one = [&](bool active, uint2 ent) {
+        if (!__any_sync(kFull, active)) return;
+        const unsigned info = active ? ent.y : 0u, key = ent.x;
+        const unsigned p = info & 0xFFFu, w = p >> 5;
+        const unsigned pq = __shfl_sync(kFull, pack, w >> 2);
+        if (active) {
+            const unsigned sub = w & 3u;
+            unsigned before = pq & 0x1FFFu;
+            if (sub > 0) before += (pq >> 13) & 0x3Fu;
+            if (sub > 1) before += (pq >> 19) & 0x3Fu;
+            if (sub > 2) before += (pq >> 25) & 0x3Fu;
+            const unsigned slot = before + __popc(bitmap[w] & ((1u << (p & 31)) - 1u));
+            if (slot < (unsigned)keff) {
+                out_idx[slot] = (uint16_t)p;
+                out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
+            }
+        }
+    };
+    write_one(pk.mask & 1u, pk.e0);
+    write_one(pk.mask & 2u, pk.e1);
+    write_one(pk.mask & 4u, pk.e2);
+    write_one(pk.mask & 8u, pk.e3);
 }
 
 // ------------------------------------------------------------------------------------------------
 // Kernel 1: u = beta e + (theta - theta_r) written into e, chunk-wise Top-k of u into staging.
-// One CTA per (chunk, worker); workers of a chunk are adjacent in the grid so that the chunk of
-// theta_sync is fetched from HBM once and served to the other workers from L2.
+//
+// Persistent CTAs (three per SM).  CTA b takes chunks b, b + grid, ... and, for each, the R workers
+// in turn ("units"), so the chunk of theta_sync is fetched once per chunk and kept in registers.
+// theta_r and e of a unit travel global -> shared as asynchronous 16-byte copies issued two units
+// ahead (two stages); every thread copies exactly the vectors it will consume itself, so no barrier
+// guards the stages.  u is formed in registers, stored to e with 128-bit stores and kept in the
+// thread's own slots of the e stage for the selection.  Short tail chunks take plain loads.
 // ------------------------------------------------------------------------------------------------
-template <bool EF>
-__global__ void __launch_bounds__(kThreads, 4)
-ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp,
-               float beta, const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
-    __shared__ SelectSmem sm;
-    const long long b = blockIdx.x;
-    const long long g = b / n_workers;
-    const int r = (int)(b - g * n_workers);
-    const ChunkDesc cd = chunks[g];
-    const int tid = threadIdx.x;
-    const float* __restrict__ ts = theta_sync + cd.base;
-    const float* __restrict__ tl = ptrs.theta_local[r] + cd.base;
-    float* __restrict__ er = EF ? ptrs.e[r] + cd.base : nullptr;
+struct PipeSmem {
+    float theta_l[2][kChunk];
+    float e[2][kChunk];  // e on arrival, u after the update
+    SelectSmem sel;
+};
 
-    unsigned ub[kPerThread];
-    if (cd.len == kChunk) {
-        // two halves of 2 x float4 per array: fewer registers held by loads in flight
+template <bool EF>
+__global__ void __launch_bounds__(kThreads, 3)
+ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
+               const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    PipeSmem& sm = *reinterpret_cast<PipeSmem*>(dyn_smem);
+    const int tid = threadIdx.x;
+    const long long grid = gridDim.x, first = blockIdx.x;
+    const long long my_chunks = (n_chunks - first + grid - 1) / grid;  // >= 1: the grid never exceeds n_chunks
+    const long long n_units = my_chunks * n_workers;
+
+    if (tid < 128) {
+        sm.sel.bitmap[0][tid] = 0;
+        sm.sel.bitmap[1][tid] = 0;
+    }
+    __syncthreads();
+
+    // element offset (from ChunkDesc::base) of this thread's i-th vector
+    auto vec_off = [&](int row_stride, int i) -> long long {
+        const int p = 1024 * i + 4 * tid;
+        return row_stride ? (long long)(p >> 6) * row_stride + (p & 63) : (long long)p;
+    };
+    // asynchronous loads of one unit into stage s; always commits one group (empty for short chunks)
+    auto issue_unit = [&](int s, const ChunkDesc& d, int r) {
+        if (d.len == kChunk) {
+            const float* __restrict__ tl = ptrs.theta_local[r] + d.base;
+            const float* __restrict__ er = EF ? ptrs.e[r] + d.base : nullptr;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            long long off[2];
-            float4 a[2], l[2], ev[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) off[i] = chunk_elem_offset(cd.row_stride, 1024 * (2 * h + i) + 4 * tid);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) a[i] = __ldg(reinterpret_cast<const float4*>(ts + off[i]));
-#pragma unroll
-            for (int i = 0; i < 2; ++i) l[i] = __ldcs(reinterpret_cast<const float4*>(tl + off[i]));
-            if (EF) {
-#pragma unroll
-                for (int i = 0; i < 2; ++i) ev[i] = __ldcs(reinterpret_cast<const float4*>(er + off[i]));
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                float4 u;
-                u.x = __fsub_rn(a[i].x, l[i].x);
-                u.y = __fsub_rn(a[i].y, l[i].y);
-                u.z = __fsub_rn(a[i].z, l[i].z);
-                u.w = __fsub_rn(a[i].w, l[i].w);
-                if (EF) {
-                    u.x = __fmaf_rn(beta, ev[i].x, u.x);
-                    u.y = __fmaf_rn(beta, ev[i].y, u.y);
-                    u.z = __fmaf_rn(beta, ev[i].z, u.z);
-                    u.w = __fmaf_rn(beta, ev[i].w, u.w);
-                    *reinterpret_cast<float4*>(er + off[i]) = u;
-                }
-                const int q0 = 4 * (2 * h + i);
-                ub[q0 + 0] = __float_as_uint(u.x);
-                ub[q0 + 1] = __float_as_uint(u.y);
-                ub[q0 + 2] = __float_as_uint(u.z);
-                ub[q0 + 3] = __float_as_uint(u.w);
+            for (int i = 0; i < 4; ++i) {
+                const long long off = vec_off(d.row_stride, i);
+                cp_async16(&sm.theta_l[s][1024 * i + 4 * tid], tl + off);
+                if (EF) cp_async16(&sm.e[s][1024 * i + 4 * tid], er + off);
             }
         }
-    } else {  // short tail of a flat tensor: element-wise with bounds
+        cp_async_commit();
+    };
+    auto load_theta_s = [&](float4 (&ts)[4], const ChunkDesc& d) {
+        if (d.len == kChunk) {
 #pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            const int p = owned_index(tid, q);
-            float u = 0.0f;
-            if (p < cd.len) {
-                u = __fsub_rn(ts[p], tl[p]);
+            for (int i = 0; i < 4; ++i)
+                ts[i] = __ldg(reinterpret_cast<const float4*>(theta_sync + d.base + vec_off(d.row_stride, i)));
+        }
+    };
+
+    // descriptors of this CTA's current chunk and the two after it
+    ChunkDesc cd = chunks[first], cd1 = cd, cd2 = cd;
+    if (my_chunks > 1) cd1 = chunks[first + grid];
+    if (my_chunks > 2) cd2 = chunks[first + 2 * grid];
+
+    // prologue: units 0 and 1
+    {
+        issue_unit(0, cd, 0);
+        if (n_units > 1)
+            issue_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
+        else
+            cp_async_commit();
+    }
+    float4 ts[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) ts[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    load_theta_s(ts, cd);
+
+    long long c = 0;  // chunk ordinal within this CTA
+    int r = 0;
+    for (long long n = 0; n < n_units; ++n) {
+        const int s = (int)(n & 1);
+        const bool full = cd.len == kChunk;
+        float* __restrict__ er = EF ? ptrs.e[r] + cd.base : nullptr;
+        float* tile = sm.e[s];
+
+        cp_async_wait<1>();  // this unit's copies have landed (only the next unit's may be in flight)
+
+        unsigned ub[kPerThread];
+        if (full) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int v = 1024 * i + 4 * tid;
+                const float4 a = ts[i];
+                const float4 l = *reinterpret_cast<const float4*>(&sm.theta_l[s][v]);
+                float4 u;
+                u.x = __fsub_rn(a.x, l.x);
+                u.y = __fsub_rn(a.y, l.y);
+                u.z = __fsub_rn(a.z, l.z);
+                u.w = __fsub_rn(a.w, l.w);
                 if (EF) {
-                    u = __fmaf_rn(beta, er[p], u);
-                    er[p] = u;
+                    const float4 ev = *reinterpret_cast<const float4*>(&tile[v]);
+                    u.x = __fmaf_rn(beta, ev.x, u.x);
+                    u.y = __fmaf_rn(beta, ev.y, u.y);
+                    u.z = __fmaf_rn(beta, ev.z, u.z);
+                    u.w = __fmaf_rn(beta, ev.w, u.w);
+                    *reinterpret_cast<float4*>(er + vec_off(cd.row_stride, i)) = u;
                 }
+                *reinterpret_cast<float4*>(&tile[v]) = u;
+                ub[4 * i + 0] = __float_as_uint(u.x);
+                ub[4 * i + 1] = __float_as_uint(u.y);
+                ub[4 * i + 2] = __float_as_uint(u.z);
+                ub[4 * i + 3] = __float_as_uint(u.w);
             }
-            ub[q] = __float_as_uint(u);
+        } else {  // short tail of a flat tensor: element-wise with bounds
+            const float* __restrict__ tsp = theta_sync + cd.base;
+            const float* __restrict__ tl = ptrs.theta_local[r] + cd.base;
+#pragma unroll
+            for (int q = 0; q < kPerThread; ++q) {
+                const int p = owned_index(tid, q);
+                float u = 0.0f;
+                if (p < cd.len) {
+                    u = __fsub_rn(tsp[p], tl[p]);
+                    if (EF) {
+                        u = __fmaf_rn(beta, er[p], u);
+                        er[p] = u;
+                    }
+                }
+                tile[p] = u;
+                ub[q] = __float_as_uint(u);
+            }
+        }
+        // theta_sync of the next chunk, once the last worker of this one has used the registers
+        if (r == n_workers - 1 && c + 1 < my_chunks) load_theta_s(ts, cd1);
+
+        const int keff = min(k, cd.len);
+        unsigned* bitmap = sm.sel.bitmap[s];
+        Picked pk;
+        pk.e0 = pk.e1 = pk.e2 = pk.e3 = make_uint2(0u, 0u);
+        bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), keff, sm.sel, pk);
+        if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
+
+        // the stage is consumed (the selection no longer reads the tile): refill it for unit n + 2
+        {
+            int r2 = r + 2;
+            int dc = 0;
+            while (r2 >= n_workers) {
+                r2 -= n_workers;
+                ++dc;
+            }
+            if (c + dc < my_chunks) {
+                ChunkDesc d2 = cd;  // picked field by field: keeps the three descriptors in registers
+                d2.base = dc == 0 ? cd.base : (dc == 1 ? cd1.base : cd2.base);
+                d2.row_stride = dc == 0 ? cd.row_stride : (dc == 1 ? cd1.row_stride : cd2.row_stride);
+                d2.len = dc == 0 ? cd.len : (dc == 1 ? cd1.len : cd2.len);
+                issue_unit(s, d2, r2);
+            } else {
+                cp_async_commit();
+            }
+        }
+
+        if (!exact) {
+            __syncthreads();
+            exact = select_rank(keff, sm.sel, bitmap, pk);
+        }
+        if (exact) {
+            unsigned tmp[kPerThread];
+            bool nonzero = false;
+#pragma unroll
+            for (int q = 0; q < kPerThread; ++q) {
+                tmp[q] = ub[q];
+                nonzero |= (ub[q] & 0x7FFFFFFFu) != 0;
+            }
+            select_exact_search(tmp, nonzero, cd.len, keff, sm.sel, bitmap);
+        }
+        __syncthreads();  // the map is complete
+        if (exact) {
+            pk.mask = 0;
+            if (tid < (int)sm.sel.n_exact) {
+                pk.e0 = sm.sel.list[0][tid];
+                pk.mask = 1u;
+            }
+        }
+        const long long g = first + c * grid;
+        const long long slot_base = ((long long)r * n_chunks + g) * kp;
+        emit_picked(pk, bitmap, keff, ws.idx + slot_base, ws.val + slot_base);
+
+        if (++r == n_workers) {
+            r = 0;
+            ++c;
+            cd = cd1;
+            cd1 = cd2;
+            if (c + 2 < my_chunks) cd2 = chunks[first + (c + 2) * grid];
         }
     }
-
-    const int keff = min(k, cd.len);
-    const long long slot_base = ((long long)r * n_chunks + g) * kp;
-    if (cd.len == kChunk)
-        select_topk<true>(ub, kChunk, keff, sm, ws.idx + slot_base, ws.val + slot_base);
-    else
-        select_topk<false>(ub, cd.len, keff, sm, ws.idx + slot_base, ws.val + slot_base);
+    cp_async_wait<0>();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -791,6 +880,7 @@ struct sl_ctx {
     std::vector<sl_tensor_desc> tensors;
     ChunkDesc* d_chunks;
     TensorInfo* d_tinfo;
+    int ef_ctas;  // resident CTAs of the persistent compression kernel on this device
     void* ws_ptr;
     size_t ws_bytes;
     int last_workers;  // worker count the workspace was last laid out for
@@ -860,12 +950,13 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     const bool ef = c->cfg.ef_enabled != 0;
 
     prof_mark(c, -1, st);
+    const unsigned ef_grid = (unsigned)(G < c->ef_ctas ? G : c->ef_ctas);  // persistent CTAs
     if (ef)
-        ef_topk_kernel<true><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                theta_sync, ptrs, ws);
+        ef_topk_kernel<true><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                         theta_sync, ptrs, ws);
     else
-        ef_topk_kernel<false><<<(unsigned)WG, kThreads, 0, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                 theta_sync, ptrs, ws);
+        ef_topk_kernel<false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                          theta_sync, ptrs, ws);
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T * 32, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
@@ -958,6 +1049,7 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->kp = (cfg->k + 3) / 4 * 4;
     c->d_chunks = nullptr;
     c->d_tinfo = nullptr;
+    c->ef_ctas = 0;
     c->ws_ptr = nullptr;
     c->ws_bytes = 0;
     c->last_workers = cfg->R;
@@ -1021,6 +1113,15 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->flat_elems = flat;
 
     cudaError_t e = cudaGetDevice(&c->device);
+    int n_sms = 0, per_sm = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true>, kThreads, sizeof(PipeSmem));
+    c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkDesc));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_tinfo, tinfo.size() * sizeof(TensorInfo));
     if (e == cudaSuccess)
