@@ -188,10 +188,10 @@ __device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzer
     }
 }
 
-// A thread's selected entries: up to four (one of the cut class, one per class above the cut).
+// A thread's selected entries: at most two.
 struct Picked {
-    uint2 e0, e1, e2, e3;  // (key, in-chunk index | sign << 12): cut class, classes 3, 2, 1
-    unsigned mask;         // bit i: entry i is selected
+    uint2 e0, e1;   // (key, in-chunk index | sign << 12): one of the cut class, one of the classes above
+    unsigned mask;  // bit i: entry i is selected
 };
 
 // First half of the selection: threshold and class lists.  `ub` = the thread's 16 value bit patterns
@@ -204,10 +204,13 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     out.mask = 0;
 
-    // -- 1. threshold
-    unsigned m = 0;
+    // -- 1. threshold.  The lane maximum is taken on floats (|x|; a NaN is skipped, which can only
+    // lower T); keys of non-NaN values order like their magnitudes.
+    float mf = 0.0f;
 #pragma unroll
-    for (int q = 0; q < kPerThread; ++q) m = max(m, ub[q] & 0x7FFFFFFFu);
+    for (int q = 0; q < kPerThread; q += 2)
+        mf = fmaxf(mf, fmaxf(fabsf(__uint_as_float(ub[q])), fabsf(__uint_as_float(ub[q + 1]))));
+    const unsigned m = __float_as_uint(mf);
     {
         const int rounds = (keff + 7) >> 3;  // <= 32
         unsigned cur = (m & ~31u) | (unsigned)lane, tw = 0;
@@ -235,15 +238,16 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
 
     bool exact = T == 0;  // uniform over the CTA
     if (!exact) {
-        // -- 2. candidates into class lists.  (T - 1 - key) has its top bit set exactly when key >= T.
+        // -- 2. candidates into class lists.  key >= T as "not (|x| < T)" on floats: T is the bit
+        // pattern of a non-negative non-NaN float and a NaN (the largest keys) passes the test.
         unsigned hits = 0;
-        const unsigned tm1 = T - 1u;
+        const float Tf = __uint_as_float(T);
 #pragma unroll
-        for (int q = 0; q < kPerThread; ++q) hits = __funnelshift_l(tm1 - (ub[q] & 0x7FFFFFFFu), hits, 1);  // bit 15 - q
+        for (int q = 0; q < kPerThread; ++q) hits |= !(fabsf(__uint_as_float(ub[q])) < Tf) ? (1u << q) : 0u;
         while (hits) {
             const int b = 31 - __clz(hits);
             hits &= ~(1u << b);
-            const int p = owned_index(tid, 15 - b);
+            const int p = owned_index(tid, b);
             const unsigned bits = tile[p];
             const unsigned kq = bits & 0x7FFFFFFFu;
             const unsigned cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
@@ -269,16 +273,22 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
     }
     if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)kClassCap) return true;  // overflow: exact search
     const unsigned want = (unsigned)keff - above;  // 1 <= want <= L
-    // classes above the cut: selected whole, one entry per thread
-    if (cstar < 3 && tid < (int)cn.w) { out.e1 = sm.list[3][tid]; out.mask |= 2u; set_bit(bitmap, out.e1.y & 0xFFFu); }
-    if (cstar < 2 && tid < (int)cn.z) { out.e2 = sm.list[2][tid]; out.mask |= 4u; set_bit(bitmap, out.e2.y & 0xFFFu); }
-    if (cstar < 1 && tid < (int)cn.y) { out.e3 = sm.list[1][tid]; out.mask |= 8u; set_bit(bitmap, out.e3.y & 0xFFFu); }
-    // the cut class: entry i = tid / nseg is ranked by nseg adjacent lanes, each over one segment
+    // classes above the cut are selected whole: `above` (< keff <= 256) entries, one per thread
+    if (tid < (int)above) {
+        uint2 ent;
+        if (tid < (int)cn.w) ent = sm.list[3][tid];
+        else if (tid < (int)(cn.w + cn.z)) ent = sm.list[2][tid - cn.w];
+        else ent = sm.list[1][tid - cn.w - cn.z];
+        out.e1 = ent;
+        out.mask |= 2u;
+        set_bit(bitmap, ent.y & 0xFFFu);
+    }
+    // the cut class: entry i = tid >> sh is ranked by 2^sh adjacent lanes, each over one segment
     const uint2* __restrict__ lst = sm.list[cstar];
-    unsigned nseg = 1;
-    while (nseg < 8 && L * (nseg * 2) <= 64u) nseg *= 2;
-    const unsigned i = tid / nseg, seg = tid & (nseg - 1);
-    const unsigned seglen = (L + nseg - 1) / nseg;
+    unsigned sh = 0;
+    while (sh < 3 && (L << (sh + 1)) <= 64u) ++sh;
+    const unsigned i = tid >> sh, seg = tid & ((1u << sh) - 1u);
+    const unsigned seglen = (L + (1u << sh) - 1u) >> sh;
     unsigned beat = 0;
     uint2 me = make_uint2(0u, 0u);
     if (i < L) {
@@ -290,7 +300,7 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
             beat += (o.x > me.x || (o.x == me.x && (o.y & 0xFFFu) < mp)) ? 1u : 0u;
         }
     }
-    for (unsigned d = 1; d < nseg; d <<= 1) beat += __shfl_xor_sync(kFull, beat, d);
+    for (unsigned d = 1; d < (1u << sh); d <<= 1) beat += __shfl_xor_sync(kFull, beat, d);
     if (i < L && seg == 0 && beat < want) {
         out.e0 = me;
         out.mask |= 1u;
@@ -339,8 +349,6 @@ __device__ __forceinline__ void emit_picked(const Picked& pk, const unsigned* __
     };
     write_one(pk.mask & 1u, pk.e0);
     write_one(pk.mask & 2u, pk.e1);
-    write_one(pk.mask & 4u, pk.e2);
-    write_one(pk.mask & 8u, pk.e3);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -376,30 +384,31 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
     }
     __syncthreads();
 
-    // element offset (from ChunkDesc::base) of this thread's i-th vector
-    auto vec_off = [&](int row_stride, int i) -> long long {
-        const int p = 1024 * i + 4 * tid;
-        return row_stride ? (long long)(p >> 6) * row_stride + (p & 63) : (long long)p;
-    };
+    // This thread's i-th vector (in-chunk indices 1024 i + 4 tid ..+3) sits at element offset
+    // off0 + 16 i rs from ChunkDesc::base, rs = the block's row stride (64 for a flat run).
+    const int sub_row = tid >> 4, sub_col = (4 * tid) & 63;
+    auto row_elems = [](const ChunkDesc& d) { return d.row_stride ? d.row_stride : kTile; };
+    auto first_off = [&](const ChunkDesc& d) { return (long long)sub_row * row_elems(d) + sub_col; };
     // asynchronous loads of one unit into stage s; always commits one group (empty for short chunks)
     auto issue_unit = [&](int s, const ChunkDesc& d, int r) {
         if (d.len == kChunk) {
-            const float* __restrict__ tl = ptrs.theta_local[r] + d.base;
-            const float* __restrict__ er = EF ? ptrs.e[r] + d.base : nullptr;
+            const long long off0 = d.base + first_off(d), step = 16ll * row_elems(d);
+            const float* __restrict__ tl = ptrs.theta_local[r] + off0;
+            const float* __restrict__ er = EF ? ptrs.e[r] + off0 : nullptr;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const long long off = vec_off(d.row_stride, i);
-                cp_async16(&sm.theta_l[s][1024 * i + 4 * tid], tl + off);
-                if (EF) cp_async16(&sm.e[s][1024 * i + 4 * tid], er + off);
+                cp_async16(&sm.theta_l[s][1024 * i + 4 * tid], tl + i * step);
+                if (EF) cp_async16(&sm.e[s][1024 * i + 4 * tid], er + i * step);
             }
         }
         cp_async_commit();
     };
     auto load_theta_s = [&](float4 (&ts)[4], const ChunkDesc& d) {
         if (d.len == kChunk) {
+            const float* __restrict__ src = theta_sync + d.base + first_off(d);
+            const long long step = 16ll * row_elems(d);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                ts[i] = __ldg(reinterpret_cast<const float4*>(theta_sync + d.base + vec_off(d.row_stride, i)));
+            for (int i = 0; i < 4; ++i) ts[i] = __ldg(reinterpret_cast<const float4*>(src + i * step));
         }
     };
 
@@ -427,6 +436,8 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         const int s = (int)(n & 1);
         const bool full = cd.len == kChunk;
         float* __restrict__ er = EF ? ptrs.e[r] + cd.base : nullptr;
+        float* __restrict__ er_vec = EF ? er + first_off(cd) : nullptr;  // this thread's first vector (full chunks)
+        const long long er_step = 16ll * row_elems(cd);
         float* tile = sm.e[s];
 
         cp_async_wait<1>();  // this unit's copies have landed (only the next unit's may be in flight)
@@ -449,7 +460,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                     u.y = __fmaf_rn(beta, ev.y, u.y);
                     u.z = __fmaf_rn(beta, ev.z, u.z);
                     u.w = __fmaf_rn(beta, ev.w, u.w);
-                    *reinterpret_cast<float4*>(er + vec_off(cd.row_stride, i)) = u;
+                    *reinterpret_cast<float4*>(er_vec + i * er_step) = u;
                 }
                 *reinterpret_cast<float4*>(&tile[v]) = u;
                 ub[4 * i + 0] = __float_as_uint(u.x);
@@ -481,7 +492,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         const int keff = min(k, cd.len);
         unsigned* bitmap = sm.sel.bitmap[s];
         Picked pk;
-        pk.e0 = pk.e1 = pk.e2 = pk.e3 = make_uint2(0u, 0u);
+        pk.e0 = pk.e1 = make_uint2(0u, 0u);
         bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), keff, sm.sel, pk);
         if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
 
