@@ -627,14 +627,18 @@ chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
     pc[0] = n0; pc[1] = n1; pc[2] = n2; pc[3] = n3;
 }
 
-// One warp per (worker, tensor): left-to-right fp64 sum of the tensor's chunk partials.
+// One warp per (worker, tensor): left-to-right fp64 sum of the tensor's chunk partials.  The order is
+// fixed, so the sum is one dependent chain; the warp only feeds it: all lanes fetch the next 32
+// partials while lane 0 adds the previous 32 out of shared memory.
 // STAGE 0: psum -> mu.  STAGE 1: psum -> sigma, 3 sigma.  STAGE 2: pbin/pcnt -> table (+ payload header).
 template <int STAGE>
 __global__ void __launch_bounds__(128)
 tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, int n_workers, int n_tensors,
                      Workspace ws, WorkerPtrs ptrs) {
-    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
+    constexpr int NV = STAGE < 2 ? 1 : 4;  // running sums
+    __shared__ double buf[4][2][NV][32];
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long w = (long long)blockIdx.x * 4 + wib;
     if (w >= (long long)n_workers * n_tensors) return;
     const int r = (int)(w / n_tensors), t = (int)(w - (long long)r * n_tensors);
     const TensorInfo ti = tinfo[t];
@@ -642,54 +646,74 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
     TStat* st = ws.tstat + (long long)r * n_tensors + t;
     const double n = (double)ti.n_slots;
 
-    if (STAGE < 2) {
-        double acc = 0.0;
-        for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32) {
-            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
-            const double x = lane < cnt ? ws.psum[first + c0 + lane] : 0.0;
-            for (int l = 0; l < cnt; ++l) acc += __shfl_sync(kFull, x, l);
+    double acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = 0.0;
+    unsigned long long cn[4] = {0, 0, 0, 0};
+    auto fetch = [&](long long c0, double (&x)[NV]) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) x[v] = 0.0;
+        if (c0 + lane < ti.n_chunks) {
+            if (STAGE < 2) {
+                x[0] = ws.psum[first + c0 + lane];
+            } else {
+                const double2* pb = reinterpret_cast<const double2*>(ws.pbin + (first + c0 + lane) * 4);
+                const double2 lo = pb[0], hi = pb[1];
+                x[0] = lo.x; x[1 % NV] = lo.y; x[2 % NV] = hi.x; x[3 % NV] = hi.y;
+                const uint4 pc = *reinterpret_cast<const uint4*>(ws.pcnt + (first + c0 + lane) * 4);
+                cn[0] += pc.x; cn[1] += pc.y; cn[2] += pc.z; cn[3] += pc.w;
+            }
         }
+    };
+    double x[NV];
+    fetch(0, x);
+    int b = 0;
+    for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32, b ^= 1) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) buf[wib][b][v][lane] = x[v];
+        __syncwarp();
+        if (c0 + 32 < ti.n_chunks) fetch(c0 + 32, x);  // in flight during the chain below
+        if (lane == 0) {
+            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
+            if (cnt == 32) {  // unrolled: the shared loads run ahead of the additions
+#pragma unroll
+                for (int l = 0; l < 32; ++l) {
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) acc[v] += buf[wib][b][v][l];
+                }
+            } else {
+                for (int l = 0; l < cnt; ++l) {
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) acc[v] += buf[wib][b][v][l];
+                }
+            }
+        }
+        // the buffer written two iterations from now is this one: lane 0 must be done with it
+        __syncwarp();
+    }
+
+    if (STAGE < 2) {
         if (lane == 0) {
             if (STAGE == 0) {
-                st->mu = (float)(acc / n);
+                st->mu = (float)(acc[0] / n);
             } else {
-                const float sigma = (float)sqrt(acc / n);
+                const float sigma = (float)sqrt(acc[0] / n);
                 st->sigma = sigma;
                 st->t3 = __fmul_rn(3.0f, sigma);
             }
         }
     } else {
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-        unsigned long long cn[4] = {0, 0, 0, 0};
-        for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32) {
-            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
-            double x0 = 0.0, x1 = 0.0, x2 = 0.0, x3 = 0.0;
-            if (lane < cnt) {
-                const double* pb = ws.pbin + (first + c0 + lane) * 4;
-                x0 = pb[0]; x1 = pb[1]; x2 = pb[2]; x3 = pb[3];
-                const unsigned* pc = ws.pcnt + (first + c0 + lane) * 4;
-                cn[0] += pc[0]; cn[1] += pc[1]; cn[2] += pc[2]; cn[3] += pc[3];
-            }
-            for (int l = 0; l < cnt; ++l) {
-                a0 += __shfl_sync(kFull, x0, l);
-                a1 += __shfl_sync(kFull, x1, l);
-                a2 += __shfl_sync(kFull, x2, l);
-                a3 += __shfl_sync(kFull, x3, l);
-            }
-        }
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
+        for (int bb = 0; bb < 4; ++bb) {
 #pragma unroll
-            for (int d = 16; d > 0; d >>= 1) cn[b] += __shfl_xor_sync(kFull, cn[b], d);
+            for (int d = 16; d > 0; d >>= 1) cn[bb] += __shfl_xor_sync(kFull, cn[bb], d);
         }
         if (lane == 0) {
             float lut[4];
-            lut[0] = cn[0] ? (float)(a0 / (double)cn[0]) : 0.0f;
-            lut[1] = cn[1] ? (float)(a1 / (double)cn[1]) : 0.0f;
-            lut[2] = cn[2] ? (float)(a2 / (double)cn[2]) : 0.0f;
-            lut[3] = cn[3] ? (float)(a3 / (double)cn[3]) : 0.0f;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) st->lut[b] = lut[b];
+            for (int bb = 0; bb < 4; ++bb) lut[bb] = cn[bb] ? (float)(acc[bb % NV] / (double)cn[bb]) : 0.0f;
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb) st->lut[bb] = lut[bb];
             st->pad = 0.0f;
             float4* hdr = reinterpret_cast<float4*>(ptrs.payload[r] + 16ll * t);
             *hdr = make_float4(lut[0], lut[1], lut[2], lut[3]);
@@ -710,8 +734,8 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long i = (long long)blockIdx.x * 4 + warp;
     if (i >= n_chunks * n_workers) return;
-    const long long g = i / n_workers;
-    const int r = (int)(i - g * n_workers);
+    const int r = (int)(i / n_chunks);  // worker-major: neighbouring warps patch neighbouring blocks of one buffer
+    const long long g = i - (long long)r * n_chunks;
     const ChunkDesc cd = chunks[g];
     const int keff = min(k, cd.len);
     const int stride = record_stride(k), words = stride / 4;
