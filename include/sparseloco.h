@@ -128,6 +128,25 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
 
+/* Deferred error-feedback subtraction (a storage choice; the paper has no counterpart).  Writing
+ * e = u - Dhat at the k selected positions of every chunk after the table is known costs a
+ * scattered read-modify-write of one 32-byte sector per selected value.  With deferral on,
+ * sl_outer_step() leaves e_r = u_r at those positions and keeps the corrected values (u - Dhat) in
+ * the workspace; the next sl_outer_step() substitutes them while it streams e_r, with identical
+ * arithmetic, so payloads, theta_sync and the true error are bit-for-bit those of the default mode.
+ * While values wait (sl_ef_pending): the error state of worker r is its buffer e[r] with those
+ * entries substituted; the workspace must be left untouched and stay lent; the next
+ * sl_outer_step() must be given the same e pointers (else INVALID_ARG).
+ *   sl_ef_flush(ctx, e, keep_pending, stream) writes the waiting values into e (HOST array of R
+ *   DEVICE pointers; NULL = the buffers of the last step), which then hold the true error.  With
+ *   keep_pending != 0 the values keep waiting (use it to materialise a copy, e.g. for a checkpoint).
+ * A step that cannot substitute them (error feedback frozen, deferral switched off, sl_compress(),
+ * sl_outer_step_host()) writes them into the buffers of the last step first.  Only sl_outer_step()
+ * defers. */
+sl_status sl_set_ef_deferred(sl_ctx* ctx, int32_t on);
+sl_status sl_ef_pending(const sl_ctx* ctx, int32_t* pending);
+sl_status sl_ef_flush(sl_ctx* ctx, float* const* e, int32_t keep_pending, void* cuda_stream);
+
 /* Same step with the workers' parameters in HOST memory (pinned for full speed), the shape a
  * deployment has when the inner loop's result arrives over the host (Alg. 1: every worker's
  * Dhat_r is gathered before the update).  theta_local_host is a host array of R host pointers;

@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
 PROFILE_SLOTS = 9
 
@@ -71,6 +71,9 @@ def _load():
     L.sl_profile_name.argtypes = [C.c_int32]
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_set_ef_deferred.argtypes = [P, C.c_int32]
+    L.sl_ef_pending.argtypes = [P, C.POINTER(C.c_int32)]
+    L.sl_ef_flush.argtypes = [P, P, C.c_int32, P]
     L.sl_read_stats.argtypes = [P, C.c_int32, P, P]
     L.sl_strerror.argtypes = [C.c_int]
     L.sl_strerror.restype = C.c_char_p
@@ -225,6 +228,18 @@ class SparseLoCo:
         _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
                                      _dev_ptr(dev_stage, torch.float32), dev_stage.numel(), ea, pa, hp,
                                      _stream()))
+
+    def set_ef_deferred(self, on: bool = True) -> None:
+        _check(_L.sl_set_ef_deferred(self._h, int(on)))
+
+    def ef_pending(self) -> bool:
+        v = C.c_int32()
+        _check(_L.sl_ef_pending(self._h, C.byref(v)))
+        return bool(v.value)
+
+    def ef_flush(self, e: Optional[List[torch.Tensor]] = None, keep_pending: bool = False) -> None:
+        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        _check(_L.sl_ef_flush(self._h, ea, int(keep_pending), _stream()))
 
     def profile_enable(self, on: bool = True) -> None:
         _check(_L.sl_profile_enable(self._h, int(on)))

@@ -110,13 +110,15 @@ __device__ __forceinline__ void cp_async_wait() {
 //
 // key = float bits without the sign (31 bits); the order is (key descending, index ascending), so
 // every element has a distinct rank and "the keff first" is exactly Top-k with the lowest-index
-// tie-break.  Thread t owns in-chunk indices p = 1024 i + 4 t + j, i, j in 0..3; its 16 values are
-// in registers and, for indexing by a run-time position, in its own slots of a shared tile.
+// tie-break.  Warp w owns in-chunk indices 512 w .. 512 w + 511; lane l of it owns
+// p = 512 w + 128 i + 4 l + j, i, j in 0..3.  The 16 values are in registers and, for indexing by a
+// run-time position, in the thread's own slots of a shared tile.
 //
 // 1. every lane takes the maximum key of its 16 values; every warp takes the ceil(keff/8)-th
 //    largest of its 32 lane maxima (low 5 bits replaced by the lane number, so that the maxima
 //    are distinct and one reduction per round suffices); T = the minimum over the 8 warps,
-//    rounded down to a multiple of 32.  At least keff values have key >= T.
+//    rounded down to a multiple of 32.  At least keff values have key >= T.  (In a short chunk
+//    only the ceil(len/512) warps that own elements take part, ceil(keff/that) rounds each.)
 // 2. the 8 warp values cluster around the keff-th largest key, so three splitters between their
 //    minimum and maximum cut the candidates (key >= T, about 2 keff of them) into four classes.
 //    Every candidate is appended to its class list; the class counts say which class holds the
@@ -127,27 +129,31 @@ __device__ __forceinline__ void cp_async_wait() {
 // If T is 0 or a class list overflows (constant chunks, heavy ties, large k) an exact bitwise
 // search over all 4096 (key, index) composites finds the keff-th largest instead.
 // ------------------------------------------------------------------------------------------------
-constexpr int kClassCap = 256;  // entries per class list (= threads: one thread per entry suffices)
+constexpr int kClassCap = 224;  // entries per class list (<= threads: one thread per entry suffices)
 
 struct SelectSmem {
-    uint2 list[4][kClassCap];  // (key, in-chunk index | sign << 12) per class
+    unsigned lkey[4][kClassCap];  // candidates per class: key
+    uint16_t lpos[4][kClassCap];  //                        in-chunk index | sign << 12
     unsigned bitmap[2][128];   // selected positions, double-buffered by unit parity
     unsigned warp_t[8];
     unsigned cnt[4];
     unsigned warp_cnt[2][8];
-    unsigned n_exact;          // entries the exact search appended to list[0]
+    unsigned n_exact;          // entries the exact search appended
 };
 
 __device__ __forceinline__ unsigned long long make_composite(unsigned key, int p) {
     return ((unsigned long long)key << 12) | (unsigned long long)(4095 - p);
 }
 
-__device__ __forceinline__ int owned_index(int tid, int q) { return 1024 * (q >> 2) + 4 * tid + (q & 3); }
+__device__ __forceinline__ int owned_index(int tid, int q) {
+    return 512 * (tid >> 5) + 128 * (q >> 2) + 4 * (tid & 31) + (q & 3);
+}
 
 __device__ __forceinline__ void set_bit(unsigned* bitmap, unsigned p) { atomicOr(&bitmap[p >> 5], 1u << (p & 31)); }
 
 // Exact fallback: bitwise search for the keff-th largest composite over all elements; the keff
-// elements at or above it are appended to list[0] (count in n_exact) and marked in the map.
+// elements at or above it are appended to the class lists taken as one array (count in n_exact)
+// and marked in the map.
 // Contains CTA barriers.  Rare path, kept out of line.
 __device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzero, int len, int keff,
                                                  SelectSmem& sm, unsigned* bitmap) {
@@ -182,7 +188,10 @@ __device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzer
         const unsigned key = ub[q] & 0x7FFFFFFFu;
         if (p < len && make_composite(key, p) >= res) {
             const unsigned pos = atomicAdd(&sm.n_exact, 1u);
-            if (pos < kClassCap) sm.list[0][pos] = make_uint2(key, (unsigned)p | ((ub[q] >> 31) << 12));
+            if (pos < (unsigned)kMaxK) {  // the four lists taken as one array: room for kMaxK entries
+                (&sm.lkey[0][0])[pos] = key;
+                (&sm.lpos[0][0])[pos] = (uint16_t)((unsigned)p | ((ub[q] >> 31) << 12));
+            }
             set_bit(bitmap, (unsigned)p);
         }
     }
@@ -190,8 +199,9 @@ __device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzer
 
 // A thread's selected entries: at most two.
 struct Picked {
-    uint2 e0, e1;   // (key, in-chunk index | sign << 12): one of the cut class, one of the classes above
-    unsigned mask;  // bit i: entry i is selected
+    unsigned p0, v0;  // in-chunk index and value bits: one entry of the cut class
+    unsigned p1, v1;  // one entry of the classes above the cut
+    unsigned mask;    // bit i: entry i is selected
 };
 
 // First half of the selection: threshold and class lists.  `ub` = the thread's 16 value bit patterns
@@ -200,7 +210,7 @@ struct Picked {
 // it, and must synchronise again before select_rank().  Returns true when the threshold is 0, in
 // which case nothing was listed and the exact search has to run instead.
 __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], const unsigned* __restrict__ tile,
-                                            int keff, SelectSmem& sm, Picked& out) {
+                                            int len, int keff, SelectSmem& sm, Picked& out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     out.mask = 0;
 
@@ -211,14 +221,17 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
     for (int q = 0; q < kPerThread; q += 2)
         mf = fmaxf(mf, fmaxf(fabsf(__uint_as_float(ub[q])), fabsf(__uint_as_float(ub[q + 1]))));
     const unsigned m = __float_as_uint(mf);
+    // warps whose 512 indices lie beyond a short chunk have nothing to offer: the others share keff
+    const int n_warps = min(8, (len + 511) >> 9);
     {
-        const int rounds = (keff + 7) >> 3;  // <= 32
+        // more than 32 rounds cannot be served by 32 lanes: tw ends as 0 and the exact search takes over
+        const int rounds = n_warps == 8 ? (keff + 7) >> 3 : min(33, (keff + n_warps - 1) / n_warps);
         unsigned cur = (m & ~31u) | (unsigned)lane, tw = 0;
         for (int i = 0; i < rounds; ++i) {
             tw = __reduce_max_sync(kFull, cur);
             cur = cur == tw ? 0u : cur;  // retire the holder (tagged values are distinct, or all 0)
         }
-        if (lane == 0) sm.warp_t[warp] = tw & ~31u;
+        if (lane == 0) sm.warp_t[warp] = warp < n_warps ? (tw & ~31u) : 0xFFFFFFFFu;
         if (tid < 4) sm.cnt[tid] = 0;
     }
     __syncthreads();
@@ -227,9 +240,17 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
         const uint4 a = *reinterpret_cast<const uint4*>(&sm.warp_t[0]);
         const uint4 b = *reinterpret_cast<const uint4*>(&sm.warp_t[4]);
         const unsigned lo = min(min(min(a.x, a.y), min(a.z, a.w)), min(min(b.x, b.y), min(b.z, b.w)));
-        const unsigned hi = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w)));
-        const unsigned mean = (a.x >> 3) + (a.y >> 3) + (a.z >> 3) + (a.w >> 3) + (b.x >> 3) + (b.y >> 3) +
-                              (b.z >> 3) + (b.w >> 3);
+        unsigned hi, mean;
+        if (n_warps == 8) {
+            hi = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w)));
+            mean = (a.x >> 3) + (a.y >> 3) + (a.z >> 3) + (a.w >> 3) + (b.x >> 3) + (b.y >> 3) + (b.z >> 3) +
+                   (b.w >> 3);
+        } else {  // short chunk: any splitters do; take them between the extremes of the warps that count
+            hi = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) hi = max(hi, w < n_warps ? sm.warp_t[w] : 0u);
+            mean = (lo >> 1) + (hi >> 1);
+        }
         T = lo;
         s2 = max(mean, lo);
         s1 = (lo >> 1) + (s2 >> 1);
@@ -252,13 +273,17 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
             const unsigned kq = bits & 0x7FFFFFFFu;
             const unsigned cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
             const unsigned pos = atomicAdd(&sm.cnt[cls], 1u);
-            if (pos < kClassCap) sm.list[cls][pos] = make_uint2(kq, (unsigned)p | ((bits >> 31) << 12));
+            if (pos < kClassCap) {
+                sm.lkey[cls][pos] = kq;
+                sm.lpos[cls][pos] = (uint16_t)((unsigned)p | ((bits >> 31) << 12));
+            }
         }
     }
     return exact;
 }
 
-// Second half of the selection, after the barrier that completes the class lists.
+// Second half of the selection, after the barrier that completes the class lists.  Returns true
+// when a list overflowed: nothing was marked and the exact search has to run instead.
 __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* bitmap, Picked& out) {
     const int tid = threadIdx.x;
     const uint4 cn = *reinterpret_cast<const uint4*>(&sm.cnt[0]);
@@ -275,36 +300,46 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
     const unsigned want = (unsigned)keff - above;  // 1 <= want <= L
     // classes above the cut are selected whole: `above` (< keff <= 256) entries, one per thread
     if (tid < (int)above) {
-        uint2 ent;
-        if (tid < (int)cn.w) ent = sm.list[3][tid];
-        else if (tid < (int)(cn.w + cn.z)) ent = sm.list[2][tid - cn.w];
-        else ent = sm.list[1][tid - cn.w - cn.z];
-        out.e1 = ent;
+        unsigned c = 3, j = tid;
+        if (j >= cn.w) {
+            j -= cn.w;
+            c = 2;
+            if (j >= cn.z) {
+                j -= cn.z;
+                c = 1;
+            }
+        }
+        out.p1 = sm.lpos[c][j];
+        out.v1 = sm.lkey[c][j] | ((out.p1 >> 12) << 31);
+        out.p1 &= 0xFFFu;
         out.mask |= 2u;
-        set_bit(bitmap, ent.y & 0xFFFu);
+        set_bit(bitmap, out.p1);
     }
     // the cut class: entry i = tid >> sh is ranked by 2^sh adjacent lanes, each over one segment
-    const uint2* __restrict__ lst = sm.list[cstar];
+    const unsigned* __restrict__ lk = sm.lkey[cstar];
+    const uint16_t* __restrict__ lp = sm.lpos[cstar];
     unsigned sh = 0;
     while (sh < 3 && (L << (sh + 1)) <= 64u) ++sh;
     const unsigned i = tid >> sh, seg = tid & ((1u << sh) - 1u);
     const unsigned seglen = (L + (1u << sh) - 1u) >> sh;
-    unsigned beat = 0;
-    uint2 me = make_uint2(0u, 0u);
+    unsigned beat = 0, mp = 0, mk = 0, msign = 0;
     if (i < L) {
-        me = lst[i];
-        const unsigned mp = me.y & 0xFFFu;
+        mk = lk[i];
+        mp = lp[i];
+        msign = mp >> 12;
+        mp &= 0xFFFu;
         const unsigned j0 = seg * seglen, j1 = min(j0 + seglen, L);
         for (unsigned j = j0; j < j1; ++j) {
-            const uint2 o = lst[j];
-            beat += (o.x > me.x || (o.x == me.x && (o.y & 0xFFFu) < mp)) ? 1u : 0u;
+            const unsigned ok = lk[j], op = lp[j] & 0xFFFu;
+            beat += (ok > mk || (ok == mk && op < mp)) ? 1u : 0u;
         }
     }
     for (unsigned d = 1; d < (1u << sh); d <<= 1) beat += __shfl_xor_sync(kFull, beat, d);
     if (i < L && seg == 0 && beat < want) {
-        out.e0 = me;
+        out.p0 = mp;
+        out.v0 = mk | (msign << 31);
         out.mask |= 1u;
-        set_bit(bitmap, me.y & 0xFFFu);
+        set_bit(bitmap, mp);
     }
     return false;
 }
@@ -329,10 +364,9 @@ __device__ __forceinline__ void emit_picked(const Picked& pk, const unsigned* __
         }
         pack = (inc - tot) | (c0 << 13) | (c1 << 19) | (c2 << 25);
     }
-    auto write_one = [&](bool active, uint2 ent) {
+    auto write_one = [&](bool active, unsigned pos, unsigned bits) {
         if (!__any_sync(kFull, active)) return;
-        const unsigned info = active ? ent.y : 0u, key = ent.x;
-        const unsigned p = info & 0xFFFu, w = p >> 5;
+        const unsigned p = active ? pos : 0u, w = p >> 5;
         const unsigned pq = __shfl_sync(kFull, pack, w >> 2);
         if (active) {
             const unsigned sub = w & 3u;
@@ -343,12 +377,12 @@ __device__ __forceinline__ void emit_picked(const Picked& pk, const unsigned* __
             const unsigned slot = before + __popc(bitmap[w] & ((1u << (p & 31)) - 1u));
             if (slot < (unsigned)keff) {
                 out_idx[slot] = (uint16_t)p;
-                out_val[slot] = __uint_as_float(key | ((info >> 12) << 31));
+                out_val[slot] = __uint_as_float(bits);
             }
         }
     };
-    write_one(pk.mask & 1u, pk.e0);
-    write_one(pk.mask & 2u, pk.e1);
+    write_one(pk.mask & 1u, pk.p0, pk.v0);
+    write_one(pk.mask & 2u, pk.p1, pk.v1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -358,95 +392,161 @@ __device__ __forceinline__ void emit_picked(const Picked& pk, const unsigned* __
 // in turn ("units"), so the chunk of theta_sync is fetched once per chunk and kept in registers.
 // theta_r and e of a unit travel global -> shared as asynchronous 16-byte copies issued two units
 // ahead (two stages); every thread copies exactly the vectors it will consume itself, so no barrier
-// guards the stages.  u is formed in registers, stored to e with 128-bit stores and kept in the
-// thread's own slots of the e stage for the selection.  Short tail chunks take plain loads.
+// guards their arrival.  u is formed in registers, stored to e with 128-bit stores and kept in the
+// e stage for the selection.  Short tail chunks take plain loads.
+//
+// PENDING: the error buffers hold u of the previous step and the corrected values (u - Dhat) of the
+// selected entries wait in the staging arrays (deferred error-feedback subtraction).  The lists of
+// the next units ride along three units ahead; before u is formed every warp substitutes the
+// entries that fall into its 512 indices (the lists are sorted, so they form one run).
 // ------------------------------------------------------------------------------------------------
 struct PipeSmem {
     float theta_l[2][kChunk];
     float e[2][kChunk];  // e on arrival, u after the update
     SelectSmem sel;
+    __align__(16) float pend_val[3][kMaxK];
+    __align__(16) uint16_t pend_idx[3][kMaxK];
 };
 
-template <bool EF>
+// The part of a ChunkDesc the compression kernel needs (its first 16 bytes).
+struct ChunkGeo {
+    long long base;
+    int row_stride;
+    int len;
+};
+__device__ __forceinline__ ChunkGeo load_geo(const ChunkDesc* d) {
+    const int4 v = __ldg(reinterpret_cast<const int4*>(d));
+    ChunkGeo g;
+    g.base = ((long long)v.y << 32) | (unsigned)v.x;
+    g.row_stride = v.z;
+    g.len = v.w;
+    return g;
+}
+
+template <bool EF, bool PENDING>
 __global__ void __launch_bounds__(kThreads, 3)
 ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     PipeSmem& sm = *reinterpret_cast<PipeSmem*>(dyn_smem);
-    const int tid = threadIdx.x;
-    const long long grid = gridDim.x, first = blockIdx.x;
-    const long long my_chunks = (n_chunks - first + grid - 1) / grid;  // >= 1: the grid never exceeds n_chunks
-    const long long n_units = my_chunks * n_workers;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // 32-bit counters: chunks x workers < 2^31 is checked on the host
+    const int grid = (int)gridDim.x, first = (int)blockIdx.x;
+    const int my_chunks = ((int)n_chunks - first + grid - 1) / grid;  // >= 1: the grid never exceeds n_chunks
+    const int n_units = my_chunks * n_workers;
 
     if (tid < 128) {
         sm.sel.bitmap[0][tid] = 0;
         sm.sel.bitmap[1][tid] = 0;
     }
-    __syncthreads();
 
-    // This thread's i-th vector (in-chunk indices 1024 i + 4 tid ..+3) sits at element offset
-    // off0 + 16 i rs from ChunkDesc::base, rs = the block's row stride (64 for a flat run).
-    const int sub_row = tid >> 4, sub_col = (4 * tid) & 63;
-    auto row_elems = [](const ChunkDesc& d) { return d.row_stride ? d.row_stride : kTile; };
-    auto first_off = [&](const ChunkDesc& d) { return (long long)sub_row * row_elems(d) + sub_col; };
-    // asynchronous loads of one unit into stage s; always commits one group (empty for short chunks)
-    auto issue_unit = [&](int s, const ChunkDesc& d, int r) {
+    // This thread's i-th vector (in-chunk indices 512 warp + 128 i + 4 lane ..+3) lies in block row
+    // 8 warp + 2 i + lane / 16 at column 4 (lane % 16): element offset off0 + 2 i rs from
+    // ChunkDesc::base, rs = the block's row stride (64 for a flat run).
+    const int sub_row = 8 * warp + (lane >> 4), sub_col = 4 * (lane & 15);
+    const int slot0 = 512 * warp + 4 * lane;  // shared-tile index of the first vector; +128 per vector
+    auto row_elems = [](const ChunkGeo& d) { return d.row_stride ? d.row_stride : kTile; };
+    auto first_off = [&](const ChunkGeo& d) { return (long long)sub_row * row_elems(d) + sub_col; };
+    // asynchronous loads of one unit into stage s (nothing for short chunks)
+    auto issue_unit = [&](int s, const ChunkGeo& d, int r) {
         if (d.len == kChunk) {
-            const long long off0 = d.base + first_off(d), step = 16ll * row_elems(d);
+            const long long off0 = d.base + first_off(d), step = 2ll * row_elems(d);
             const float* __restrict__ tl = ptrs.theta_local[r] + off0;
             const float* __restrict__ er = EF ? ptrs.e[r] + off0 : nullptr;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                cp_async16(&sm.theta_l[s][1024 * i + 4 * tid], tl + i * step);
-                if (EF) cp_async16(&sm.e[s][1024 * i + 4 * tid], er + i * step);
+                cp_async16(&sm.theta_l[s][slot0 + 128 * i], tl + i * step);
+                if (EF) cp_async16(&sm.e[s][slot0 + 128 * i], er + i * step);
             }
         }
-        cp_async_commit();
     };
-    auto load_theta_s = [&](float4 (&ts)[4], const ChunkDesc& d) {
+    // warp 0: the pending list of unit (chunk g, worker r) into ring slot `ring`
+    auto issue_pending = [&](int ring, int g, int r) {
+        const long long slot_base = ((long long)r * n_chunks + g) * kp;  // kp is a multiple of 8
+        if (lane < (kp >> 3)) cp_async16(&sm.pend_idx[ring][8 * lane], ws.idx + slot_base + 8 * lane);
+        for (int v = lane; v < (kp >> 2); v += 32) cp_async16(&sm.pend_val[ring][4 * v], ws.val + slot_base + 4 * v);
+    };
+    auto load_theta_s = [&](float4 (&ts)[4], const ChunkGeo& d) {
         if (d.len == kChunk) {
             const float* __restrict__ src = theta_sync + d.base + first_off(d);
-            const long long step = 16ll * row_elems(d);
+            const long long step = 2ll * row_elems(d);
 #pragma unroll
             for (int i = 0; i < 4; ++i) ts[i] = __ldg(reinterpret_cast<const float4*>(src + i * step));
         }
     };
+    // (chunk ordinal, worker) of the unit `by` units after (c, r)
+    auto ahead = [&](int c, int r, int by, int& c2, int& r2) {
+        r2 = r + by;
+        c2 = c;
+        while (r2 >= n_workers) {
+            r2 -= n_workers;
+            ++c2;
+        }
+    };
 
     // descriptors of this CTA's current chunk and the two after it
-    ChunkDesc cd = chunks[first], cd1 = cd, cd2 = cd;
-    if (my_chunks > 1) cd1 = chunks[first + grid];
-    if (my_chunks > 2) cd2 = chunks[first + 2 * grid];
+    ChunkGeo cd = load_geo(chunks + first), cd1 = cd, cd2 = cd;
+    if (my_chunks > 1) cd1 = load_geo(chunks + first + grid);
+    if (my_chunks > 2) cd2 = load_geo(chunks + first + 2 * grid);
 
-    // prologue: units 0 and 1
-    {
-        issue_unit(0, cd, 0);
-        if (n_units > 1)
-            issue_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
-        else
-            cp_async_commit();
+    // prologue: pending lists of units 0..2 (published by the barrier), then units 0 and 1
+    if (PENDING) {
+        if (warp == 0) {
+            for (int j = 0; j < 3 && j < n_units; ++j) {
+                int c2, r2;
+                ahead(0, 0, j, c2, r2);
+                issue_pending(j, first + c2 * grid, r2);
+            }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
     }
+    __syncthreads();
+    issue_unit(0, cd, 0);
+    cp_async_commit();
+    if (n_units > 1) issue_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
+    cp_async_commit();
+
     float4 ts[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) ts[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     load_theta_s(ts, cd);
 
-    long long c = 0;  // chunk ordinal within this CTA
-    int r = 0;
-    for (long long n = 0; n < n_units; ++n) {
-        const int s = (int)(n & 1);
+    int c = 0, r = 0;  // chunk ordinal within this CTA, worker
+    for (int n = 0; n < n_units; ++n) {
+        const int s = n & 1;
         const bool full = cd.len == kChunk;
+        const int keff = min(k, cd.len);
         float* __restrict__ er = EF ? ptrs.e[r] + cd.base : nullptr;
         float* __restrict__ er_vec = EF ? er + first_off(cd) : nullptr;  // this thread's first vector (full chunks)
-        const long long er_step = 16ll * row_elems(cd);
+        const long long er_step = 2ll * row_elems(cd);
         float* tile = sm.e[s];
 
         cp_async_wait<1>();  // this unit's copies have landed (only the next unit's may be in flight)
+
+        if (PENDING && EF) {  // substitute the corrected values of the previous step
+            const int ring = n % 3;
+            if (full) {
+                __syncwarp();  // the whole warp's copies have landed
+                for (int j = lane; j < keff; j += 32) {
+                    const unsigned p = sm.pend_idx[ring][j];
+                    if ((p >> 9) == (unsigned)warp) tile[p] = sm.pend_val[ring][j];
+                }
+                __syncwarp();
+            } else {  // short chunk: patch global memory, which the plain loads below read
+                for (int j = tid; j < keff; j += kThreads) {
+                    const unsigned p = sm.pend_idx[ring][j];
+                    if (p < (unsigned)cd.len) er[p] = sm.pend_val[ring][j];
+                }
+                __syncthreads();
+            }
+        }
 
         unsigned ub[kPerThread];
         if (full) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int v = 1024 * i + 4 * tid;
+                const int v = slot0 + 128 * i;
                 const float4 a = ts[i];
                 const float4 l = *reinterpret_cast<const float4*>(&sm.theta_l[s][v]);
                 float4 u;
@@ -489,34 +589,34 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         // theta_sync of the next chunk, once the last worker of this one has used the registers
         if (r == n_workers - 1 && c + 1 < my_chunks) load_theta_s(ts, cd1);
 
-        const int keff = min(k, cd.len);
         unsigned* bitmap = sm.sel.bitmap[s];
         Picked pk;
-        pk.e0 = pk.e1 = make_uint2(0u, 0u);
-        bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), keff, sm.sel, pk);
+        pk.p0 = pk.v0 = pk.p1 = pk.v1 = 0u;
+        bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), cd.len, keff, sm.sel, pk);
         if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
 
-        // the stage is consumed (the selection no longer reads the tile): refill it for unit n + 2
+        // the stage is consumed (nothing below reads the tile): refill it for unit n + 2; warp 0 also
+        // fetches the pending list of unit n + 3 (its ring slot was last read before the barrier above)
         {
-            int r2 = r + 2;
-            int dc = 0;
-            while (r2 >= n_workers) {
-                r2 -= n_workers;
-                ++dc;
-            }
-            if (c + dc < my_chunks) {
-                ChunkDesc d2 = cd;  // picked field by field: keeps the three descriptors in registers
+            int c2, r2;
+            ahead(c, r, 2, c2, r2);
+            if (c2 < my_chunks) {
+                const int dc = c2 - c;
+                ChunkGeo d2;  // picked field by field: keeps the three descriptors in registers
                 d2.base = dc == 0 ? cd.base : (dc == 1 ? cd1.base : cd2.base);
                 d2.row_stride = dc == 0 ? cd.row_stride : (dc == 1 ? cd1.row_stride : cd2.row_stride);
                 d2.len = dc == 0 ? cd.len : (dc == 1 ? cd1.len : cd2.len);
                 issue_unit(s, d2, r2);
-            } else {
-                cp_async_commit();
             }
+            if (PENDING && warp == 0) {
+                ahead(c, r, 3, c2, r2);
+                if (c2 < my_chunks) issue_pending(n % 3, first + c2 * grid, r2);
+            }
+            cp_async_commit();
         }
 
         if (!exact) {
-            __syncthreads();
+            __syncthreads();  // class lists complete
             exact = select_rank(keff, sm.sel, bitmap, pk);
         }
         if (exact) {
@@ -533,12 +633,14 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         if (exact) {
             pk.mask = 0;
             if (tid < (int)sm.sel.n_exact) {
-                pk.e0 = sm.sel.list[0][tid];
+                pk.p0 = (&sm.sel.lpos[0][0])[tid];
+                pk.v0 = (&sm.sel.lkey[0][0])[tid] | ((pk.p0 >> 12) << 31);
+                pk.p0 &= 0xFFFu;
                 pk.mask = 1u;
             }
         }
-        const long long g = first + c * grid;
-        const long long slot_base = ((long long)r * n_chunks + g) * kp;
+
+        const long long slot_base = ((long long)r * n_chunks + (first + c * grid)) * kp;
         emit_picked(pk, bitmap, keff, ws.idx + slot_base, ws.val + slot_base);
 
         if (++r == n_workers) {
@@ -546,7 +648,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             ++c;
             cd = cd1;
             cd1 = cd2;
-            if (c + 2 < my_chunks) cd2 = chunks[first + (c + 2) * grid];
+            if (c + 2 < my_chunks) cd2 = load_geo(chunks + first + (c + 2) * grid);
         }
     }
     cp_async_wait<0>();
@@ -726,7 +828,9 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
 // indices and 2-bit codes OR-ed into a shared-memory record, record written as 16-byte vectors,
 // e[index] = value - table[code] at the selected positions (Eq. 2 line 2).
 // ------------------------------------------------------------------------------------------------
-template <bool EF>
+// MODE 0: records only (error feedback frozen).  MODE 1: e[index] = value - table[code].
+// MODE 2: the corrected value replaces the staged value instead (deferred subtraction).
+template <int MODE>
 __global__ void __launch_bounds__(128)
 pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
                 int k, int kp, Workspace ws, WorkerPtrs ptrs) {
@@ -754,15 +858,35 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
         if ((bit & 31) > 20) atomicOr(&rec[warp][(bit >> 5) + 1], p >> (32 - (bit & 31)));
         const int cbit = code_word0 * 8 + 2 * s;
         atomicOr(&rec[warp][cbit >> 5], (unsigned)c << (cbit & 31));
-        if (EF && p < (unsigned)cd.len) {
+        if (MODE == 1 && p < (unsigned)cd.len) {
             float* er = ptrs.e[r] + cd.base + chunk_elem_offset(cd.row_stride, (int)p);
             *er = __fsub_rn(v, st.lut[c]);
         }
+        if (MODE == 2) ws.val[slot_base + s] = __fsub_rn(v, st.lut[c]);
     }
     __syncwarp();
     uint4* dst = reinterpret_cast<uint4*>(ptrs.payload[r] + cd.rec_off);
     const uint4* src = reinterpret_cast<const uint4*>(rec[warp]);
     for (int w = lane; w < stride / 16; w += 32) dst[w] = src[w];
+}
+
+// Writes the corrected values waiting in the staging arrays into the error buffers (deferred
+// subtraction made good).  One warp per (worker, chunk).
+__global__ void __launch_bounds__(128)
+ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, Workspace ws,
+                WorkerPtrs ptrs) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long i = (long long)blockIdx.x * 4 + warp;
+    if (i >= n_chunks * n_workers) return;
+    const int r = (int)(i / n_chunks);
+    const long long g = i - (long long)r * n_chunks;
+    const ChunkDesc cd = chunks[g];
+    const int keff = min(k, cd.len);
+    const long long slot_base = ((long long)r * n_chunks + g) * kp;
+    for (int s = lane; s < keff; s += 32) {
+        const unsigned p = ws.idx[slot_base + s];
+        if (p < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = ws.val[slot_base + s];
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -916,6 +1040,9 @@ struct sl_ctx {
     ChunkDesc* d_chunks;
     TensorInfo* d_tinfo;
     int ef_ctas;  // resident CTAs of the persistent compression kernel on this device
+    bool deferred;              // deferred error-feedback subtraction (sl_set_ef_deferred)
+    bool pending;               // corrected values of the last step still wait in the workspace
+    float* pending_e[kMaxR];    // the error buffers they belong to
     void* ws_ptr;
     size_t ws_bytes;
     int last_workers;  // worker count the workspace was last laid out for
@@ -973,9 +1100,19 @@ inline void prof_mark(sl_ctx* c, int slot, cudaStream_t st) {
     cudaEventRecord(c->prof_events[(size_t)c->prof_steps * (kProfSlots + 1) + (slot + 1)], st);
 }
 
-// Compression of `workers` workers whose pointers are in `ptrs` (kernels 1-8).
+sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
+    const int R = c->cfg.R;
+    const Workspace ws = carve(c, R);
+    ef_flush_kernel<<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp, ws,
+                                                                    ptrs);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+// Compression of `workers` workers whose pointers are in `ptrs` (kernels 1-8).  `defer`: leave the
+// corrected values in the workspace instead of writing them into e (only with all R workers).
 sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const WorkerPtrs& ptrs,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool defer) {
     if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, workers)) return SL_ERR_NOMEM;
     const Workspace ws = carve(c, workers);
     c->last_workers = workers;
@@ -983,17 +1120,34 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     const int k = c->cfg.k, kp = c->kp, T = c->n_tensors;
     if (WG > 0x7FFFFFFFll) return SL_ERR_TOO_LARGE;
     const bool ef = c->cfg.ef_enabled != 0;
+    bool consume = false;  // this step substitutes the waiting values while it streams e
+    if (c->pending) {
+        if (ef && defer) {
+            consume = true;
+        } else {  // nothing will read them in flight (frozen step): write them out first
+            WorkerPtrs fp;
+            memset(&fp, 0, sizeof(fp));
+            for (int r = 0; r < c->cfg.R; ++r) fp.e[r] = c->pending_e[r];
+            sl_status s = launch_flush(c, fp, st);
+            if (s != SL_OK) return s;
+        }
+        c->pending = false;
+    }
 
     prof_mark(c, -1, st);
     const unsigned ef_grid = (unsigned)(G < c->ef_ctas ? G : c->ef_ctas);  // persistent CTAs
-    if (ef)
-        ef_topk_kernel<true><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                         theta_sync, ptrs, ws);
+    const size_t smem = sizeof(PipeSmem);
+    if (!ef)
+        ef_topk_kernel<false, false><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                      theta_sync, ptrs, ws);
+    else if (consume)
+        ef_topk_kernel<true, true><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                    theta_sync, ptrs, ws);
     else
-        ef_topk_kernel<false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                          theta_sync, ptrs, ws);
+        ef_topk_kernel<true, false><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
+                                                                     theta_sync, ptrs, ws);
     prof_mark(c, 0, st);
-    const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T * 32, 128);
+    const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
     prof_mark(c, 1, st);
     tensor_reduce_kernel<0><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
@@ -1006,12 +1160,19 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     prof_mark(c, 5, st);
     tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 6, st);
-    if (ef)
-        pack_fix_kernel<true><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    const unsigned pb = blocks_for(WG, 4);
+    if (!ef)
+        pack_fix_kernel<0><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    else if (defer)
+        pack_fix_kernel<2><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     else
-        pack_fix_kernel<false><<<blocks_for(WG, 4), 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+        pack_fix_kernel<1><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     prof_mark(c, 7, st);
     SL_CUDA(cudaGetLastError());
+    if (ef && defer) {
+        c->pending = true;
+        for (int r = 0; r < workers; ++r) c->pending_e[r] = ptrs.e[r];
+    }
     return SL_OK;
 }
 
@@ -1081,10 +1242,12 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (!c) return SL_ERR_INVALID_ARG;
     c->cfg = *cfg;
     c->n_tensors = n_tensors;
-    c->kp = (cfg->k + 3) / 4 * 4;
+    c->kp = (cfg->k + 7) / 8 * 8;
     c->d_chunks = nullptr;
     c->d_tinfo = nullptr;
     c->ef_ctas = 0;
+    c->deferred = false;
+    c->pending = false;
     c->ws_ptr = nullptr;
     c->ws_bytes = 0;
     c->last_workers = cfg->R;
@@ -1151,11 +1314,13 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     int n_sms = 0, per_sm = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+        e = cudaFuncSetAttribute(ef_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+        e = cudaFuncSetAttribute(ef_topk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
     if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true>, kThreads, sizeof(PipeSmem));
+        e = cudaFuncSetAttribute(ef_topk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true>, kThreads, sizeof(PipeSmem));
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkDesc));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_tinfo, tinfo.size() * sizeof(TensorInfo));
@@ -1228,6 +1393,7 @@ sl_status sl_workspace_bytes(const sl_ctx* c, size_t* bytes) {
 
 sl_status sl_set_workspace(sl_ctx* c, void* dev_ptr, size_t bytes) {
     if (!c) return SL_ERR_INVALID_ARG;
+    if (c->pending) return SL_ERR_INVALID_ARG;  // the workspace holds part of the error state: sl_ef_flush() first
     if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return SL_ERR_ALIGNMENT;
     c->ws_ptr = dev_ptr;
     c->ws_bytes = dev_ptr ? bytes : 0;
@@ -1247,7 +1413,7 @@ sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
     ptrs.theta_local[0] = theta_local;
     ptrs.e[0] = e;
     ptrs.payload[0] = payload;
-    return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream));
+    return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream), false);
 }
 
 sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
@@ -1291,7 +1457,12 @@ sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    sl_status s = launch_compress(c, R, theta_sync, ptrs, st);
+    const bool defer = c->deferred && c->cfg.ef_enabled;
+    if (c->pending && defer) {  // the waiting values can only be substituted into the buffers they came from
+        for (int r = 0; r < R; ++r)
+            if (e[r] != c->pending_e[r]) return SL_ERR_INVALID_ARG;
+    }
+    sl_status s = launch_compress(c, R, theta_sync, ptrs, st, defer);
     if (s != SL_OK) return s;
     return launch_apply(c, pl, R, theta_sync, st);
 }
@@ -1340,7 +1511,7 @@ sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* t
         ptrs.theta_local[0] = stage;
         ptrs.e[0] = e ? e[r] : nullptr;
         ptrs.payload[0] = payloads[r];
-        sl_status s = launch_compress(c, 1, theta_sync, ptrs, st);
+        sl_status s = launch_compress(c, 1, theta_sync, ptrs, st, false);
         if (s != SL_OK) return s;
         SL_CUDA(cudaEventRecord(c->ev_consumed[bsel], st));
         pl.p[r] = payloads[r];
@@ -1389,6 +1560,37 @@ const char* sl_profile_name(int32_t slot) {
     static const char* names[kProfSlots] = {"ef_topk", "chunk_sum", "tensor_mean", "chunk_var", "tensor_sigma",
                                             "chunk_bins", "tensor_lut", "pack_fix", "decode_avg_apply"};
     return slot >= 0 && slot < kProfSlots ? names[slot] : "";
+}
+
+sl_status sl_set_ef_deferred(sl_ctx* c, int32_t on) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    c->deferred = on != 0;
+    return SL_OK;
+}
+
+sl_status sl_ef_pending(const sl_ctx* c, int32_t* pending) {
+    if (!c || !pending) return SL_ERR_INVALID_ARG;
+    *pending = c->pending ? 1 : 0;
+    return SL_OK;
+}
+
+sl_status sl_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* stream) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    if (!c->pending) return SL_OK;
+    WorkerPtrs ptrs;
+    memset(&ptrs, 0, sizeof(ptrs));
+    for (int r = 0; r < c->cfg.R; ++r) {
+        float* dst = e ? e[r] : c->pending_e[r];
+        if (!dst) return SL_ERR_INVALID_ARG;
+        if (misaligned(dst)) return SL_ERR_ALIGNMENT;
+        ptrs.e[r] = dst;
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    sl_status s = launch_flush(c, ptrs, static_cast<cudaStream_t>(stream));
+    if (s != SL_OK) return s;
+    if (!keep_pending) c->pending = false;
+    return SL_OK;
 }
 
 sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {

@@ -68,13 +68,14 @@ class DeviceCase:
     def snapshot(self, tensor_ids: Sequence[int]) -> Dict[int, dict]:
         """CPU copies of theta_sync / theta_local / e slices of the given tensors (pre-step)."""
         snap = {}
+        e_dev = self.true_error()
         for j in tensor_ids:
             t, off = self.wl.tensors[j], self.offs[j]
             sl = slice(off, off + t.numel)
             snap[j] = {
                 "theta": self.theta[sl].cpu().numpy().copy(),
                 "local": [self.local_of(r)[sl].cpu().numpy().copy() for r in range(self.wl.R)],
-                "e": [self.e[r][sl].cpu().numpy().copy() for r in range(self.wl.R)],
+                "e": [e_dev[r][sl].cpu().numpy().copy() for r in range(self.wl.R)],
             }
         return snap
 
@@ -87,8 +88,19 @@ class DeviceCase:
         recs = p[self.rec_off[j]:self.rec_off[j] + self.n_chunks[j] * self.stride].cpu().numpy()
         return np.concatenate([hdr, recs])
 
+    def true_error(self) -> List[torch.Tensor]:
+        """The error buffers as the method defines them.  With the deferred subtraction on, the values
+        still waiting in the workspace are written into copies (they keep waiting for the next step)."""
+        if not self.sl.ef_pending():
+            return self.e
+        copies = [x.clone() for x in self.e]
+        self.sl.ef_flush(copies, keep_pending=True)
+        return copies
+
     def check(self, snap: Dict[int, dict], ef_enabled: bool = True, present: Optional[List[bool]] = None) -> dict:
         """Run the oracle on the snapshot tensors and compare with the device state after step()."""
+        torch.cuda.synchronize()
+        e_dev = self.true_error()
         torch.cuda.synchronize()
         R = self.wl.R
         worst = 0.0
@@ -109,7 +121,7 @@ class DeviceCase:
                     raise AssertionError(
                         f"payload mismatch: tensor {j} ({t.name}) worker {r}: {bad.size} bytes differ, first at "
                         f"{bad[0]} (record {(bad[0] - 16) // self.stride if bad[0] >= 16 else 'header'})")
-                e_g = self.e[r][off:off + t.numel].cpu().numpy()
+                e_g = e_dev[r][off:off + t.numel].cpu().numpy()
                 if not np.array_equal(e_g.view(np.uint32), e_o.view(np.uint32)):
                     bad = np.nonzero(e_g.view(np.uint32) != e_o.view(np.uint32))[0]
                     raise AssertionError(f"error buffer mismatch: tensor {j} ({t.name}) worker {r}: "

@@ -99,6 +99,51 @@ def test_error_feedback_freeze():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("k", [41, 64, 200])
+def test_deferred_subtraction_is_bit_identical(k):
+    """Deferred error-feedback subtraction: payloads, theta_sync and the true error buffers match the
+    oracle after every step, through a frozen step (which writes the waiting values out first), and
+    the buffers themselves hold the true error after a flush."""
+    wl = I.Workload("deferred", SMALL, R=3, k=k, recipe="student_t4", seed=90 + k, outer_lr=0.9)
+    c = _case(wl, e_scale=0.5)
+    c.sl.set_ef_deferred(True)
+    for step in range(5):
+        frozen = step == 3
+        c.sl.set_hyper(ef_enabled=not frozen)
+        c.fill_local(step)
+        snap = c.snapshot(range(len(SMALL)))
+        c.step()
+        assert c.sl.ef_pending() == (not frozen)
+        c.check(snap, ef_enabled=not frozen)
+    assert c.sl.ef_pending()
+    want = [x.clone() for x in c.true_error()]
+    c.sl.ef_flush()
+    torch.cuda.synchronize()
+    assert not c.sl.ef_pending()
+    for a, b in zip(c.e, want):
+        assert torch.equal(a, b)
+    # pointers of other buffers are refused while values wait
+    c.fill_local(9)
+    c.step()
+    from paper_2508_15706_b200 import binding as B
+    with pytest.raises(B.SlError) as ei:
+        c.sl.outer_step(c.theta, [c.local_of(r) for r in range(3)], [x.clone() for x in c.e], c.payloads)
+    assert ei.value.status == B.SL_ERR_INVALID_ARG
+    # a default-mode twin ends in the same state
+    d = _case(wl, e_scale=0.5)
+    c2 = _case(wl, e_scale=0.5)
+    c2.sl.set_ef_deferred(True)
+    for step in range(3):
+        for x in (d, c2):
+            x.fill_local(step)
+            x.step()
+    c2.sl.ef_flush()
+    torch.cuda.synchronize()
+    assert torch.equal(d.theta, c2.theta)
+    for r in range(3):
+        assert torch.equal(d.e[r], c2.e[r]) and torch.equal(d.payloads[r], c2.payloads[r])
+
+
 def test_compress_then_aggregate_equals_outer_step_and_absent_workers():
     import oracle as O
     wl = I.Workload("split", SMALL, R=3, k=64, recipe="normal", seed=51, outer_lr=0.8)
