@@ -103,6 +103,22 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: the job's time when every rank runs its own replica."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(params: int, steps: int, ms_max: float, world: int) -> float:
+    """Whole-job params/s: every rank processed `params` per step in `ms_max` milliseconds."""
+    return world * params * steps / (ms_max * 1e-3)
+
+
 def pick_distinct_locals(torch, wl, k: int, flat: int, payload_bytes: int, workspace_bytes: int) -> int:
     """How many distinct theta_local buffers fit (worker r reads buffer r % D)."""
     free, _total = torch.cuda.mem_get_info()
@@ -183,14 +199,9 @@ def run_ours(args) -> dict:
     clocks = sampler.stop(t0, t1)
     prof = sl.profile_read()
     sl.profile_enable(False)
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_max = float(tmax.item())
-    else:
-        ms_max = ms
+    ms_max = max_over_ranks(ms, world, dev)
     ms_per_step = ms_max / args.steps
-    value = world * N * args.steps / (ms_max * 1e-3)
+    value = job_value(N, args.steps, ms_max, world)
 
     # roofline of the dominant kernel, timed live with CUDA events inside the timed region
     top = max(prof.items(), key=lambda kv: kv[1][0])
