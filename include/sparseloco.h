@@ -181,6 +181,41 @@ sl_status sl_profile_enable(sl_ctx* ctx, int32_t enable);
 sl_status sl_profile_read(sl_ctx* ctx, float* ms_total, int64_t* launches);
 const char* sl_profile_name(int32_t slot);
 
+/* Compression of ONE tensor of ONE worker that allocates nothing (the paper has no counterpart:
+ * this is sl_compress() for callers that cannot allocate device memory).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a training loop that has handed
+ * all device memory to a caching allocator or a fixed arena, a latency-critical section that must
+ * not take the allocator's device-wide synchronisation, a plug-in that is only given buffers.  Such
+ * a caller cannot create a context (sl_create allocates the chunk table) nor lend a workspace.
+ *
+ * Instead, the chunk table, the staged (index, value) pairs, the partial sums and the tensor
+ * statistics live in a fixed array of sl_static_scratch_bytes() = 4 MiB inside the library, one copy
+ * per GPU that loads the library, held until the process exits.  The caller still passes inputs
+ * and outputs:
+ *   theta_sync, theta_local : the tensor, rows x cols fp32 row-major (rows == 1 for a vector), read only
+ *   e       : same shape, updated in place to u - Dhat (error feedback always on, coefficient beta)
+ *   payload : 16 + sl_record_stride(k) * chunks bytes, fully overwritten: the 16-byte table, then
+ *             the records, i.e. the payload sl_compress() writes for a one-tensor table
+ * Results are bit-identical to sl_compress() on a context holding this single tensor.
+ *
+ * Limits and rules:
+ *   - the tensor must fit the scratch: about (88 + 6 roundup8(k)) bytes per chunk, i.e. about 8,800
+ *     chunks (36 M elements) at k = 64; larger calls return SL_ERR_TOO_LARGE and do nothing.
+ *   - the first call on a device looks up the array's device address and sizes the launch (no
+ *     allocation, but host-side queries): make that first call before any stream capture.
+ *   - every call on a GPU shares the one array: calls whose kernels overlap on the GPU (different
+ *     streams, different threads) race; serialise them.  Nothing has to be cleared between calls:
+ *     each call rewrites every scratch location before reading it, whatever the previous call left.
+ *   - no cudaMalloc, cudaFree or other allocating routine is called; all work is enqueued on
+ *     `cuda_stream` and the call does not synchronise.
+ * Errors: INVALID_ARG (NULL, rows/cols/k < 1, beta outside [0,1]), ALIGNMENT (a pointer not 16-byte
+ * aligned), UNSUPPORTED (k > 256), TOO_LARGE, CUDA. */
+size_t sl_static_scratch_bytes(void);
+sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_local, float* e,
+                                    uint8_t* payload, int64_t rows, int64_t cols, int32_t k, float beta,
+                                    void* cuda_stream);
+
 const char* sl_strerror(sl_status s);
 const char* sl_last_cuda_error(void); /* text of the last CUDA error seen by this thread */
 

@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
 PROFILE_SLOTS = 9
 
@@ -71,6 +71,8 @@ def _load():
     L.sl_profile_name.argtypes = [C.c_int32]
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_static_scratch_bytes.restype = C.c_size_t
+    L.sl_compress_tensor_static.argtypes = [P, P, P, P, C.c_int64, C.c_int64, C.c_int32, C.c_float, P]
     L.sl_set_ef_deferred.argtypes = [P, C.c_int32]
     L.sl_ef_pending.argtypes = [P, C.POINTER(C.c_int32)]
     L.sl_ef_flush.argtypes = [P, P, C.c_int32, P]
@@ -114,6 +116,18 @@ def _stream() -> int:
 
 def record_stride(k: int) -> int:
     return _L.sl_record_stride(k)
+
+
+def static_scratch_bytes() -> int:
+    return _L.sl_static_scratch_bytes()
+
+
+def compress_tensor_static(theta_sync, theta_local, e, payload, rows: int, cols: int, k: int, beta: float) -> None:
+    """sl_compress_tensor_static: one tensor of one worker, scratch inside the library, no allocation.
+    Raises SlError (status SL_ERR_TOO_LARGE) when the tensor does not fit the fixed scratch."""
+    _check(_L.sl_compress_tensor_static(_dev_ptr(theta_sync, torch.float32), _dev_ptr(theta_local, torch.float32),
+                                        _dev_ptr(e, torch.float32), _dev_ptr(payload, torch.uint8), rows, cols, k,
+                                        beta, _stream()))
 
 
 class SparseLoCo:

@@ -1620,3 +1620,143 @@ sl_status sl_read_stats(sl_ctx* c, int32_t worker, float* dev_out, void* stream)
 }
 
 }  // extern "C"
+
+// ================================================================================================
+// Compression of one tensor without any allocation (sl_compress_tensor_static)
+// ================================================================================================
+
+namespace {
+
+constexpr size_t kStaticScratchBytes = 4u << 20;
+// Scratch of sl_compress_tensor_static(): chunk table, staged (index, value) pairs, partial sums and
+// tensor statistics of one call.  One copy per GPU that loads the library, held until the process
+// exits; shared by every call on that GPU.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticSetup {  // per device: address of the array above, launch shape of the persistent kernel
+    void* scratch;
+    int ef_ctas;
+    bool ready;
+};
+StaticSetup g_static_setup[64];
+
+// Chunk table of a single tensor at element offset 0 (same rules as sl_create()).
+__global__ void __launch_bounds__(128)
+build_single_tensor_table_kernel(long long rows, long long cols, int k, long long n_chunks, ChunkDesc* chunks,
+                                 TensorInfo* tinfo) {
+    const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long n = rows * cols;
+    const bool tiled = rows > 1 && rows % kTile == 0 && cols % kTile == 0;
+    if (g == 0) {
+        long long slots = 0;
+        if (tiled) {
+            slots = n_chunks * min((long long)k, (long long)kChunk);
+        } else {
+            const long long tail = n - (n_chunks - 1) * kChunk;
+            slots = (n_chunks - 1) * min((long long)k, (long long)kChunk) + min((long long)k, tail);
+        }
+        tinfo->first_chunk = 0;
+        tinfo->n_chunks = n_chunks;
+        tinfo->n_slots = slots;
+    }
+    if (g >= n_chunks) return;
+    ChunkDesc d;
+    if (tiled) {
+        const long long tc = cols / kTile, a = g / tc, b = g - a * tc;
+        d.base = a * kTile * cols + b * kTile;
+        d.row_stride = (int)cols;
+        d.len = kChunk;
+    } else {
+        d.base = g * kChunk;
+        d.row_stride = 0;
+        const long long rest = n - g * kChunk;
+        d.len = (int)(rest < kChunk ? rest : kChunk);
+    }
+    d.tensor = 0;
+    d.chunk_in_tensor = (int)g;
+    d.rec_off = 16 + (long long)record_stride(k) * g;
+    chunks[g] = d;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t sl_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
+                                    int64_t rows, int64_t cols, int32_t k, float beta, void* stream) {
+    if (!theta_sync || !theta_local || !e || !payload) return SL_ERR_INVALID_ARG;
+    if (rows < 1 || cols < 1 || k < 1 || !(beta >= 0.0f && beta <= 1.0f)) return SL_ERR_INVALID_ARG;
+    if (k > kMaxK) return SL_ERR_UNSUPPORTED;
+    if (misaligned(theta_sync) || misaligned(theta_local) || misaligned(e) || misaligned(payload)) return SL_ERR_ALIGNMENT;
+    if (cols > 0x7FFFFFFFll || rows > (1ll << 40) / cols) return SL_ERR_TOO_LARGE;
+    const long long n = rows * cols;
+    const bool tiled = rows > 1 && rows % kTile == 0 && cols % kTile == 0;
+    const long long G = tiled ? (rows / kTile) * (cols / kTile) : (n + kChunk - 1) / kChunk;
+    const int kp = (k + 7) / 8 * 8;
+    // layout of the scratch: chunk table | tensor info | the arrays of a one-worker workspace
+    const size_t WG = (size_t)G;
+    const size_t off_tinfo = up256(WG * sizeof(ChunkDesc));
+    const size_t off_val = off_tinfo + up256(sizeof(TensorInfo));
+    const size_t off_idx = off_val + up256(WG * kp * sizeof(float));
+    const size_t off_psum = off_idx + up256(WG * kp * sizeof(uint16_t));
+    const size_t off_pbin = off_psum + up256(WG * sizeof(double));
+    const size_t off_pcnt = off_pbin + up256(WG * 4 * sizeof(double));
+    const size_t off_tstat = off_pcnt + up256(WG * 4 * sizeof(unsigned));
+    const size_t need = off_tstat + up256(sizeof(TStat));
+    if (need > kStaticScratchBytes) return SL_ERR_TOO_LARGE;  // the fixed scratch cannot hold this tensor
+
+    int dev = -1;
+    SL_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SL_ERR_UNSUPPORTED;
+    StaticSetup& su = g_static_setup[dev];
+    if (!su.ready) {  // first call on this device: resolve the array's device address, size the launch
+        void* ptr = nullptr;
+        SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        int n_sms = 0, per_sm = 0;
+        SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(PipeSmem)));
+        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false>, kThreads,
+                                                              sizeof(PipeSmem)));
+        su.scratch = ptr;
+        su.ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
+        su.ready = true;
+    }
+    char* base = static_cast<char*>(su.scratch);
+    ChunkDesc* d_chunks = reinterpret_cast<ChunkDesc*>(base);
+    TensorInfo* d_tinfo = reinterpret_cast<TensorInfo*>(base + off_tinfo);
+    Workspace ws;
+    ws.val = reinterpret_cast<float*>(base + off_val);
+    ws.idx = reinterpret_cast<uint16_t*>(base + off_idx);
+    ws.psum = reinterpret_cast<double*>(base + off_psum);
+    ws.pbin = reinterpret_cast<double*>(base + off_pbin);
+    ws.pcnt = reinterpret_cast<unsigned*>(base + off_pcnt);
+    ws.tstat = reinterpret_cast<TStat*>(base + off_tstat);
+    WorkerPtrs ptrs;
+    memset(&ptrs, 0, sizeof(ptrs));
+    ptrs.theta_local[0] = theta_local;
+    ptrs.e[0] = e;
+    ptrs.payload[0] = payload;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Every array is fully rewritten by the kernels below before it is read, so nothing left behind
+    // by an earlier call (of any size) is ever consumed and nothing has to be cleared.
+    build_single_tensor_table_kernel<<<blocks_for(G, 128), 128, 0, st>>>(rows, cols, k, G, d_chunks, d_tinfo);
+    const unsigned ef_grid = (unsigned)(G < su.ef_ctas ? G : su.ef_ctas);
+    ef_topk_kernel<true, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
+                                                                            ptrs, ws);
+    const unsigned cb = blocks_for(G, 128);
+    chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
+    tensor_reduce_kernel<0><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);
+    chunk_sum_kernel<1><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
+    tensor_reduce_kernel<1><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);
+    chunk_bins_kernel<<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
+    tensor_reduce_kernel<2><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);
+    pack_fix_kernel<1><<<blocks_for(G, 4), 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws, ptrs);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+}  // extern "C"
