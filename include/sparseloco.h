@@ -139,7 +139,8 @@ sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* thet
  * sl_outer_step() must be given the same e pointers (else INVALID_ARG).
  *   sl_ef_flush(ctx, e, keep_pending, stream) writes the waiting values into e (HOST array of R
  *   DEVICE pointers; NULL = the buffers of the last step), which then hold the true error.  With
- *   keep_pending != 0 the values keep waiting (use it to materialise a copy, e.g. for a checkpoint).
+ *   keep_pending != 0 the values keep waiting (use it to materialise a copy, e.g. for a checkpoint),
+ *   and NULL entries of e skip that worker (one spare buffer then serves all workers in turn).
  * A step that cannot substitute them (error feedback frozen, deferral switched off, sl_compress(),
  * sl_outer_step_host()) writes them into the buffers of the last step first.  Only sl_outer_step()
  * defers. */

@@ -252,7 +252,7 @@ class SparseLoCo:
         return bool(v.value)
 
     def ef_flush(self, e: Optional[List[torch.Tensor]] = None, keep_pending: bool = False) -> None:
-        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        ea = _ptr_array([_dev_ptr(t, torch.float32) if t is not None else None for t in e]) if e is not None else None
         _check(_L.sl_ef_flush(self._h, ea, int(keep_pending), _stream()))
 
     def profile_enable(self, on: bool = True) -> None:

@@ -879,6 +879,7 @@ ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const long long i = (long long)blockIdx.x * 4 + warp;
     if (i >= n_chunks * n_workers) return;
     const int r = (int)(i / n_chunks);
+    if (!ptrs.e[r]) return;  // this worker was left out of the flush
     const long long g = i - (long long)r * n_chunks;
     const ChunkDesc cd = chunks[g];
     const int keff = min(k, cd.len);
@@ -1581,7 +1582,7 @@ sl_status sl_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* st
     memset(&ptrs, 0, sizeof(ptrs));
     for (int r = 0; r < c->cfg.R; ++r) {
         float* dst = e ? e[r] : c->pending_e[r];
-        if (!dst) return SL_ERR_INVALID_ARG;
+        if (!dst && !keep_pending) return SL_ERR_INVALID_ARG;  // a worker may be skipped only if its values stay
         if (misaligned(dst)) return SL_ERR_ALIGNMENT;
         ptrs.e[r] = dst;
     }

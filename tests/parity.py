@@ -68,14 +68,14 @@ class DeviceCase:
     def snapshot(self, tensor_ids: Sequence[int]) -> Dict[int, dict]:
         """CPU copies of theta_sync / theta_local / e slices of the given tensors (pre-step)."""
         snap = {}
-        e_dev = self.true_error()
+        e_cpu = self.error_slices(tensor_ids)
         for j in tensor_ids:
             t, off = self.wl.tensors[j], self.offs[j]
             sl = slice(off, off + t.numel)
             snap[j] = {
                 "theta": self.theta[sl].cpu().numpy().copy(),
                 "local": [self.local_of(r)[sl].cpu().numpy().copy() for r in range(self.wl.R)],
-                "e": [e_dev[r][sl].cpu().numpy().copy() for r in range(self.wl.R)],
+                "e": [e_cpu[r][j] for r in range(self.wl.R)],
             }
         return snap
 
@@ -97,11 +97,28 @@ class DeviceCase:
         self.sl.ef_flush(copies, keep_pending=True)
         return copies
 
+    def error_slices(self, tensor_ids: Sequence[int]) -> List[Dict[int, np.ndarray]]:
+        """CPU copies of the true error of the given tensors, per worker.  Large cases materialise
+        one worker at a time into a single spare buffer."""
+        def cut(buf):
+            return {j: buf[self.offs[j]:self.offs[j] + self.wl.tensors[j].numel].cpu().numpy().copy()
+                    for j in tensor_ids}
+        if not self.sl.ef_pending():
+            return [cut(x) for x in self.e]
+        out = []
+        spare = torch.empty_like(self.e[0])
+        for r in range(self.wl.R):
+            spare.copy_(self.e[r])
+            self.sl.ef_flush([spare if q == r else None for q in range(self.wl.R)], keep_pending=True)
+            torch.cuda.synchronize()
+            out.append(cut(spare))
+        del spare
+        return out
+
     def check(self, snap: Dict[int, dict], ef_enabled: bool = True, present: Optional[List[bool]] = None) -> dict:
         """Run the oracle on the snapshot tensors and compare with the device state after step()."""
         torch.cuda.synchronize()
-        e_dev = self.true_error()
-        torch.cuda.synchronize()
+        e_cpu = self.error_slices(list(snap.keys()))
         R = self.wl.R
         worst = 0.0
         report = {"tensors": 0, "payload_bytes": 0, "theta_max_err_over_rms": 0.0}
@@ -121,7 +138,7 @@ class DeviceCase:
                     raise AssertionError(
                         f"payload mismatch: tensor {j} ({t.name}) worker {r}: {bad.size} bytes differ, first at "
                         f"{bad[0]} (record {(bad[0] - 16) // self.stride if bad[0] >= 16 else 'header'})")
-                e_g = e_dev[r][off:off + t.numel].cpu().numpy()
+                e_g = e_cpu[r][j]
                 if not np.array_equal(e_g.view(np.uint32), e_o.view(np.uint32)):
                     bad = np.nonzero(e_g.view(np.uint32) != e_o.view(np.uint32))[0]
                     raise AssertionError(f"error buffer mismatch: tensor {j} ({t.name}) worker {r}: "

@@ -1,0 +1,82 @@
+"""GPU parity at the full sizes of the benchmark's configurations, in the launch configuration that
+bench.py times (deferred error-feedback subtraction on, theta_local buffers shared by r mod D for
+the 2B case).  The CUDA path runs on the whole model; the oracle recomputes a sample of tensors
+(one of every kind: blocked matrices, norm vectors shorter than a chunk, the flat-path router,
+experts with exactly zero drift) from copies taken before the step.  Bars as everywhere: payload
+bytes and error buffers bit-exact, theta_sync within 1e-6 x RMS of the tensor."""
+import gc
+
+import pytest
+import torch
+
+from paper_2508_15706_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(wl, **kw):
+    from parity import DeviceCase, oracle_threads
+    gc.collect()
+    torch.cuda.empty_cache()
+    oracle_threads()
+    c = DeviceCase(wl, **kw)
+    c.sl.set_ef_deferred(True)
+    return c
+
+
+def _ids(wl, names):
+    from parity import sample_tensor_ids
+    ids = sample_tensor_ids(wl, names)
+    assert len(ids) == len(names), "sample names must exist in the workload"
+    return ids
+
+
+def _run(c, ids, steps):
+    for step in range(steps):
+        c.fill_local(step)
+        snap = c.snapshot(ids)
+        c.step()
+        rep = c.check(snap)
+        assert rep["tensors"] == len(ids)
+    return rep
+
+
+def test_config2_dense_d768_three_steps():
+    wl = I.workload("c2_dense_d768")
+    c = _case(wl)
+    assert c.sl.payload_bytes() == 4445152
+    _run(c, _ids(wl, ["l0.q", "l5.gate", "l11.down", "l3.norm1", "final_norm"]), steps=3)
+
+
+@pytest.mark.parametrize("k", [41, 82, 123])
+def test_config3_dense_d1280_k_sweep(k):
+    wl = I.workload("c3_dense_d1280")
+    c = _case(wl, k=k)
+    assert c.sl.payload_bytes() == {41: 13895424, 82: 25008960, 123: 38900880}[k]
+    _run(c, _ids(wl, ["l0.k", "l12.up", "l23.down", "l7.norm2"]), steps=2)
+
+
+def test_config4_moe_zero_experts_two_steps():
+    wl = I.workload("c4_moe_d1024")
+    c = _case(wl)
+    assert c.sl.payload_bytes() == 19694816
+    names = ["l0.router", "l0.o", "l11.norm1"] + [f"l2.x{x}.gate" for x in range(8)] + ["l5.x3.down", "l5.x6.down"]
+    _run(c, _ids(wl, names), steps=2)
+
+
+def test_config5_dense_d2048_as_benchmarked():
+    wl = I.workload("c5_dense_d2048")
+    c = _case(wl, distinct_local=6, e_scale=0.5)  # 23 model-sized buffers + one spare for the checks
+    assert c.sl.payload_bytes() == 47633184
+    ids = _ids(wl, ["l0.q", "l9.v", "l23.down", "l17.norm1", "final_norm"])
+    _run(c, ids, steps=2)
+    # the waiting values can be written out and leave the true error in the buffers themselves
+    want = c.error_slices(ids[:2])
+    c.sl.ef_flush()
+    torch.cuda.synchronize()
+    assert not c.sl.ef_pending()
+    got = c.error_slices(ids[:2])
+    import numpy as np
+    for r in range(wl.R):
+        for j in ids[:2]:
+            assert np.array_equal(got[r][j].view(np.uint32), want[r][j].view(np.uint32))
