@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "c5_dense_d2048"
 
 # DRAM bytes per ef_topk launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
 # on a smaller case of the same kernel, as bytes per (parameter x worker); see profiles/.
-NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = None
+NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = 12.400  # profiles/ncu_full_c5_layer0_top3_kernels.md
 
 
 def record_stride(k: int) -> int:
@@ -236,7 +236,7 @@ def run_ours(args) -> dict:
                    "l2": "inputs larger than L2 (every buffer is %.1f GB; state evolves every step)" % (4 * flat / 1e9),
                    "multi_gpu": "replicas only (no data-path collective)"},
         "clocks": clocks,
-        "gpu_launches": 9 * args.steps,
+        "gpu_launches": 9 * args.steps + (1 if deferred else 0),
         "roofline": {"bound": "hbm", "kernel": "ef_topk", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": ef_bytes, "avg_launch_ms": ef_avg_ms,
