@@ -891,9 +891,15 @@ ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Decode + average + outer update.  One CTA per chunk: all present workers' records are copied to
-// shared memory, warp 0 adds table[code] into a 4096-float shared tile worker by worker (fixed
-// order => reproducible bits), then every thread applies theta = fma(-alpha/D, sum, theta).
+// Decode + average + outer update.  One CTA per chunk.  Every (worker, slot) entry of the chunk is
+// decoded by its own thread and ORs its worker's bit into a per-position mask in shared memory.
+// The mask gives the entry its rank among the workers that selected the same position (bits
+// below its own), and the entries are added into a 4096-float shared tile in rounds: rank 0
+// first, then rank 1, ... with a barrier in between.  Every position thus receives its values in
+// ascending worker order (reproducible bits), one writer per position and round, and the number
+// of rounds is the largest number of workers that meet at one position (3 or 4 at R = 16).  Then
+// every thread applies theta = fma(-alpha/D, sum, theta) to its own 16 positions.
+// Workers are taken in batches of at most 32 (one mask bit each, 8 entries per thread).
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned get12(const unsigned* rec, int s) {
     const int bit = 12 * s;
@@ -904,73 +910,129 @@ __device__ __forceinline__ unsigned get2(const unsigned* rec, int code_byte0, in
     return (rec[bit >> 5] >> (bit & 31)) & 3u;
 }
 
-__global__ void __launch_bounds__(kThreads)
+constexpr int kApplyEntries = 8;  // entries per thread and batch
+
+template <int SPL>  // slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8
+__global__ void __launch_bounds__(kThreads, 4)
 decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale,
                         PayloadPtrs pl, float* __restrict__ theta_sync) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    float* acc = reinterpret_cast<float*>(dyn);                       // 4096 floats
-    float* luts = acc + kChunk;                                       // n_workers x 4
-    unsigned* recs = reinterpret_cast<unsigned*>(luts + 4 * n_workers);  // n_workers x (stride + 16) bytes
+    float* acc = reinterpret_cast<float*>(dyn);                            // 4096 sums
+    unsigned* wmask = reinterpret_cast<unsigned*>(acc + kChunk);           // 4096 worker masks
+    float* luts = reinterpret_cast<float*>(wmask + kChunk);                // 32 x 4
+    unsigned* recs = reinterpret_cast<unsigned*>(luts + 4 * 32);           // batch x (stride + 16) bytes
     const int stride = record_stride(k), rwords = stride / 4 + 4;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const ChunkDesc cd = chunks[blockIdx.x];
     const int keff = min(k, cd.len);
+    const int code_byte0 = record_index_bytes(k);
     float* __restrict__ th = theta_sync + cd.base;
 
-    // theta loads first (in flight while the records are staged)
+    // theta loads first (in flight while the records are decoded);
+    // vector i of this thread (in-chunk indices 1024 i + 4 tid ..+3) sits at th_vec + i * vec_step
     float4 a[4];
-    long long off[4];
+    const int rs = cd.row_stride ? cd.row_stride : kTile;
+    float* __restrict__ th_vec = th + (long long)(tid >> 4) * rs + (4 * tid & 63);
+    const long long vec_step = 16ll * rs;
     const bool full = cd.len == kChunk;
     if (full) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            off[i] = chunk_elem_offset(cd.row_stride, 1024 * i + 4 * tid);
-            a[i] = *reinterpret_cast<const float4*>(th + off[i]);
-        }
+        for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(th_vec + i * vec_step);
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    // entry e of a thread: worker warp + 8 (e / SPL), slot lane + 32 (e % SPL)
+    constexpr int WPW = kApplyEntries / SPL;  // workers per warp and batch
+    constexpr int batch = 8 * WPW < 32 ? 8 * WPW : 32;
     const int vec_per_rec = stride / 16;
-    for (int v = tid; v < n_workers * vec_per_rec; v += kThreads) {
-        const int r = v / vec_per_rec, w = v - r * vec_per_rec;
-        if (pl.p[r]) {
-            const uint4 x = __ldg(reinterpret_cast<const uint4*>(pl.p[r] + cd.rec_off) + w);
-            *reinterpret_cast<uint4*>(recs + r * rwords + 4 * w) = x;
-        }
-    }
-    for (int v = tid; v < n_workers; v += kThreads) {
-        if (pl.p[v]) {
-            const float4 x = __ldg(reinterpret_cast<const float4*>(pl.p[v] + 16ll * cd.tensor));
-            *reinterpret_cast<float4*>(luts + 4 * v) = x;
-        }
-        recs[v * rwords + stride / 4] = 0;  // word read past the index block by get12
-    }
-    __syncthreads();
-    if (tid < 32) {
-        const int code_byte0 = record_index_bytes(k);
-        for (int r = 0; r < n_workers; ++r) {
-            if (!pl.p[r]) continue;
-            const unsigned* rec = recs + r * rwords;
-            for (int s = tid; s < keff; s += 32) {
-                const unsigned p = get12(rec, s);
-                const unsigned c = get2(rec, code_byte0, s);
-                if (p < (unsigned)cd.len) acc[p] += luts[4 * r + c];
+
+    for (int r0 = 0; r0 < n_workers; r0 += batch) {
+        const int nb = min(batch, n_workers - r0);
+        // clear the masks, stage this batch's records and tables (the last barrier of the
+        // previous batch's rounds has released both)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(wmask + 1024 * i + 4 * tid) = make_uint4(0u, 0u, 0u, 0u);
+        for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
+            const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
+            const uint8_t* src = pl.p[r0 + rb];
+            if (src) {
+                const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + cd.rec_off) + w);
+                *reinterpret_cast<uint4*>(recs + rb * rwords + 4 * w) = x;
             }
-            __syncwarp();
+        }
+        if (tid < nb) {
+            const uint8_t* src = pl.p[r0 + tid];
+            if (src) *reinterpret_cast<float4*>(luts + 4 * tid) = __ldg(reinterpret_cast<const float4*>(src + 16ll * cd.tensor));
+            recs[tid * rwords + stride / 4] = 0;  // word read past the index block by get12
+        }
+        __syncthreads();
+
+        unsigned ent_p[kApplyEntries];  // position | worker bit number << 12; 0xFFFFFFFF = no entry
+        float ent_v[kApplyEntries];
+#pragma unroll
+        for (int e = 0; e < kApplyEntries; ++e) {
+            ent_p[e] = 0xFFFFFFFFu;
+            ent_v[e] = 0.f;
+        }
+#pragma unroll
+        for (int wi = 0; wi < WPW; ++wi) {
+            const int rb = warp + 8 * wi;
+            if (rb < nb && pl.p[r0 + rb]) {  // uniform over the warp
+                const unsigned* rec = recs + rb * rwords;
+#pragma unroll
+                for (int si = 0; si < SPL; ++si) {
+                    const int sl = lane + 32 * si;
+                    if (sl < keff) {
+                        const unsigned p = get12(rec, sl);
+                        if (p < (unsigned)cd.len) {
+                            ent_v[wi * SPL + si] = luts[4 * rb + get2(rec, code_byte0, sl)];
+                            ent_p[wi * SPL + si] = p | ((unsigned)rb << 12);
+                            atomicOr(&wmask[p], 1u << rb);
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        // rank of every entry among the workers at its position; round 0
+        int my_max = 0;
+#pragma unroll
+        for (int e = 0; e < kApplyEntries; ++e) {
+            if (ent_p[e] != 0xFFFFFFFFu) {
+                const unsigned p = ent_p[e] & 0xFFFu, rb = ent_p[e] >> 12;
+                const unsigned wm = wmask[p];
+                const int rank = __popc(wm & ((1u << rb) - 1u));
+                my_max = max(my_max, __popc(wm));
+                if (rank == 0) {
+                    acc[p] = __fadd_rn(acc[p], ent_v[e]);
+                    ent_p[e] = 0xFFFFFFFFu;
+                } else {
+                    ent_p[e] = p | ((unsigned)rank << 12);  // from here on: position | rank << 12
+                }
+            }
+        }
+        for (int t = 1; __syncthreads_or(my_max > t); ++t) {
+#pragma unroll
+            for (int e = 0; e < kApplyEntries; ++e) {
+                if (ent_p[e] != 0xFFFFFFFFu && (int)(ent_p[e] >> 12) == t) {
+                    const unsigned p = ent_p[e] & 0xFFFu;
+                    acc[p] = __fadd_rn(acc[p], ent_v[e]);
+                }
+            }
         }
     }
-    __syncthreads();
+
     if (full) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float4 s = *reinterpret_cast<const float4*>(acc + 1024 * i + 4 * tid);
+            const float4 sv = *reinterpret_cast<const float4*>(acc + 1024 * i + 4 * tid);
             float4 o;
-            o.x = __fmaf_rn(scale, s.x, a[i].x);
-            o.y = __fmaf_rn(scale, s.y, a[i].y);
-            o.z = __fmaf_rn(scale, s.z, a[i].z);
-            o.w = __fmaf_rn(scale, s.w, a[i].w);
-            *reinterpret_cast<float4*>(th + off[i]) = o;
+            o.x = __fmaf_rn(scale, sv.x, a[i].x);
+            o.y = __fmaf_rn(scale, sv.y, a[i].y);
+            o.z = __fmaf_rn(scale, sv.z, a[i].z);
+            o.w = __fmaf_rn(scale, sv.w, a[i].w);
+            *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
         }
     } else {
         for (int p = tid; p < cd.len; p += kThreads) th[p] = __fmaf_rn(scale, acc[p], th[p]);
@@ -1183,13 +1245,18 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const double D = c->cfg.divide_by_present ? (double)present : (double)R;
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
     const int stride = record_stride(c->cfg.k);
-    const size_t smem = (size_t)kChunk * 4 + (size_t)R * 16 + (size_t)R * (stride + 16);
+    const int nb = R < 32 ? R : 32;  // the kernel never stages more than 32 records at once
+    const size_t smem = (size_t)kChunk * 8 + 32 * 16 + (size_t)nb * (stride + 16);
     if (smem > 48 * 1024) {
-        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)smem));
+        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    decode_avg_apply_kernel<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl,
-                                                                          theta_sync);
+    const int spl = (c->cfg.k + 31) / 32;
+    auto kern = spl <= 1 ? decode_avg_apply_kernel<1> : spl <= 2 ? decode_avg_apply_kernel<2>
+              : spl <= 4 ? decode_avg_apply_kernel<4> : decode_avg_apply_kernel<8>;
+    kern<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, theta_sync);
     prof_mark(c, 8, st);
     if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
     SL_CUDA(cudaGetLastError());
