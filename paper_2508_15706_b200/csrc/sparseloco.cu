@@ -659,6 +659,32 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
 // bits: fp64, slot by slot inside a chunk, then chunk by chunk inside the tensor.
 // ------------------------------------------------------------------------------------------------
 
+// Visits the keff staged values of one unit in slot order: four 128-bit loads in flight at a time.
+template <typename F>
+__device__ __forceinline__ void for_each_staged(const float* __restrict__ v, int keff, F f) {
+    int s0 = 0;
+    for (; s0 + 16 <= keff; s0 += 16) {
+        float4 x[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) x[q] = __ldcs(reinterpret_cast<const float4*>(v + s0) + q);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            f(x[q].x);
+            f(x[q].y);
+            f(x[q].z);
+            f(x[q].w);
+        }
+    }
+    for (; s0 < keff; ++s0) f(v[s0]);
+}
+
+// (worker, chunk) of work item i; chunks x workers < 2^31 (checked on the host)
+__device__ __forceinline__ void split_unit(long long i, long long n_chunks, int& r, int& g) {
+    const unsigned ui = (unsigned)i, nc = (unsigned)n_chunks;
+    r = (int)(ui / nc);
+    g = (int)(ui - (unsigned)r * nc);
+}
+
 // mode 0: sum of values; mode 1: sum of squared fp32-centred values.  One thread per (worker, chunk).
 template <int MODE>
 __global__ void __launch_bounds__(128)
@@ -666,27 +692,21 @@ chunk_sum_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
                  int k, int kp, Workspace ws) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_chunks * n_workers) return;
-    const long long r = i / n_chunks, g = i - r * n_chunks;
-    const int len = chunks[g].len, keff = min(k, len);
+    int r, g;
+    split_unit(i, n_chunks, r, g);
+    const int keff = min(k, chunks[g].len);
     const float* __restrict__ v = ws.val + i * kp;
     float mu = 0.0f;
-    if (MODE == 1) mu = ws.tstat[r * n_tensors + chunks[g].tensor].mu;
+    if (MODE == 1) mu = ws.tstat[(long long)r * n_tensors + chunks[g].tensor].mu;
     double acc = 0.0;
-    for (int s0 = 0; s0 < keff; s0 += 4) {
-        const float4 x = *reinterpret_cast<const float4*>(v + s0);
-        const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (s0 + j < keff) {
-                if (MODE == 0) {
-                    acc += (double)xs[j];
-                } else {
-                    const double d = (double)__fsub_rn(xs[j], mu);
-                    acc += d * d;  // d*d is exact in fp64, so fusing or not gives the same sum
-                }
-            }
+    for_each_staged(v, keff, [&](float x) {
+        if (MODE == 0) {
+            acc += (double)x;
+        } else {
+            const double d = (double)__fsub_rn(x, mu);
+            acc += d * d;  // d*d is exact in fp64, so fusing or not gives the same sum
         }
-    }
+    });
     ws.psum[i] = acc;
 }
 
@@ -701,32 +721,27 @@ chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
                   int k, int kp, Workspace ws) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_chunks * n_workers) return;
-    const long long r = i / n_chunks, g = i - r * n_chunks;
-    const int len = chunks[g].len, keff = min(k, len);
+    int r, g;
+    split_unit(i, n_chunks, r, g);
+    const int keff = min(k, chunks[g].len);
     const float* __restrict__ v = ws.val + i * kp;
-    const TStat st = ws.tstat[r * n_tensors + chunks[g].tensor];
+    const TStat st = ws.tstat[(long long)r * n_tensors + chunks[g].tensor];
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
     unsigned n0 = 0, n1 = 0, n2 = 0, n3 = 0;
-    for (int sb = 0; sb < keff; sb += 4) {
-        const float4 x = *reinterpret_cast<const float4*>(v + sb);
-        const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (sb + j < keff) {
-                const int c = quant_code(xs[j], st.mu, st.t3);
-                const double d = (double)xs[j];
-                // add only to the value's own bin (adding +0 elsewhere could flip a -0 sum)
-                if (c == 0) { s0 += d; ++n0; }
-                else if (c == 1) { s1 += d; ++n1; }
-                else if (c == 2) { s2 += d; ++n2; }
-                else { s3 += d; ++n3; }
-            }
-        }
-    }
-    double* pb = ws.pbin + i * 4;
-    pb[0] = s0; pb[1] = s1; pb[2] = s2; pb[3] = s3;
-    unsigned* pc = ws.pcnt + i * 4;
-    pc[0] = n0; pc[1] = n1; pc[2] = n2; pc[3] = n3;
+    for_each_staged(v, keff, [&](float x) {
+        const int c = quant_code(x, st.mu, st.t3);
+        const double d = (double)x;
+        // add only to the value's own bin (adding +0 elsewhere could flip a -0 sum); nearly all
+        // selected values sit in the two inner bins, so the branches diverge two ways at most
+        if (c == 1) { s1 += d; ++n1; }
+        else if (c == 2) { s2 += d; ++n2; }
+        else if (c == 0) { s0 += d; ++n0; }
+        else { s3 += d; ++n3; }
+    });
+    double2* pb = reinterpret_cast<double2*>(ws.pbin + i * 4);
+    pb[0] = make_double2(s0, s1);
+    pb[1] = make_double2(s2, s3);
+    *reinterpret_cast<uint4*>(ws.pcnt + i * 4) = make_uint4(n0, n1, n2, n3);
 }
 
 // One warp per (worker, tensor): left-to-right fp64 sum of the tensor's chunk partials.  The order is
