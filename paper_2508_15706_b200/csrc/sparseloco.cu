@@ -853,8 +853,8 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long i = (long long)blockIdx.x * 4 + warp;
     if (i >= n_chunks * n_workers) return;
-    const int r = (int)(i / n_chunks);  // worker-major: neighbouring warps patch neighbouring blocks of one buffer
-    const long long g = i - (long long)r * n_chunks;
+    int r, g;  // worker-major: neighbouring warps handle neighbouring blocks of one buffer
+    split_unit(i, n_chunks, r, g);
     const ChunkDesc cd = chunks[g];
     const int keff = min(k, cd.len);
     const int stride = record_stride(k), words = stride / 4;
@@ -893,9 +893,9 @@ ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long i = (long long)blockIdx.x * 4 + warp;
     if (i >= n_chunks * n_workers) return;
-    const int r = (int)(i / n_chunks);
+    int r, g;
+    split_unit(i, n_chunks, r, g);
     if (!ptrs.e[r]) return;  // this worker was left out of the flush
-    const long long g = i - (long long)r * n_chunks;
     const ChunkDesc cd = chunks[g];
     const int keff = min(k, cd.len);
     const long long slot_base = ((long long)r * n_chunks + g) * kp;
