@@ -319,7 +319,7 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
     const unsigned* __restrict__ lk = sm.lkey[cstar];
     const uint16_t* __restrict__ lp = sm.lpos[cstar];
     unsigned sh = 0;
-    while (sh < 3 && (L << (sh + 1)) <= 64u) ++sh;
+    while (sh < 3 && (L << (sh + 1)) <= 32u) ++sh;
     const unsigned i = tid >> sh, seg = tid & ((1u << sh) - 1u);
     const unsigned seglen = (L + (1u << sh) - 1u) >> sh;
     unsigned beat = 0, mp = 0, mk = 0, msign = 0;
