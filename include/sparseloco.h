@@ -25,7 +25,7 @@
  * Quantiser (Sec. 4): per (worker, tensor), over all selected values: mean mu, population sigma of
  * the centred values, bins (-inf,-3s) [-3s,0) [0,3s) [3s,inf) on centred values, table entry =
  * mean of the raw values in the bin (+0 when empty).  Sums are fp64, slot by slot inside a chunk,
- * then chunk by chunk.
+ * then chunk by chunk inside a group of 64 consecutive chunks of the tensor, then group by group.
  *
  * Payload of one worker (little-endian; App. "Compression of indices": 12 bits per index):
  *     bytes [16 j, 16 j + 16)          table of tensor j: 4 x fp32

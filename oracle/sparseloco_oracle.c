@@ -30,8 +30,9 @@
  *   - u = fmaf(beta, e, theta - theta_r): one fp32 subtraction, one fused
  *     multiply-add, round-to-nearest, denormals kept.
  *   - sigma is the population standard deviation (divide by n) of the fp32
- *     centred values; sums are fp64, taken slot by slot inside a chunk and then
- *     chunk by chunk.  Bin edges on centred values are -3 sigma, 0, +3 sigma
+ *     centred values; sums are fp64, taken slot by slot inside a chunk, then
+ *     chunk by chunk inside a group of 64 consecutive chunks, then group by group.
+ *     Bin edges on centred values are -3 sigma, 0, +3 sigma
  *     with the lower edge inclusive; values beyond +-6 sigma fall in the outer
  *     bins.  Centroids are means of the raw (uncentred) values; an empty bin
  *     stores +0.
@@ -196,6 +197,8 @@ int32_t orc_topk_chunk(const float* u, int32_t L, int32_t k, int32_t* idx_out) {
 
 /* ---------------------------------------------------------------- quantiser Q of one tensor */
 
+#define ORC_SUM_GROUP 64 /* chunks per group in the three-level summation order */
+
 /* v: the tensor's selected values, chunk after chunk, each chunk's `cnt[c]` values in slot order.
  * Outputs: mu, sigma, lut[4], code per value.  Sec. 4: centre by the mean, [-6 sigma, 6 sigma]
  * in four uniform bins (edges -3 sigma, 0, 3 sigma on centred values), centroid table. */
@@ -208,14 +211,20 @@ void orc_quantize_tensor(const float* v, const int32_t* cnt, int64_t n_chunks, f
     *sigma_out = 0.0f;
     if (n == 0) return;
 
+    /* Every sum over the tensor is taken in three fixed levels, all fp64, each left to right:
+     * the slots of a chunk, the chunks of a group of ORC_SUM_GROUP consecutive chunks, the groups. */
     double S = 0.0;
     {
         const float* q = v;
-        for (int64_t c = 0; c < n_chunks; ++c) {
-            double sc = 0.0;
-            for (int32_t s = 0; s < cnt[c]; ++s) sc += (double)q[s];
-            S += sc;
-            q += cnt[c];
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double sg = 0.0;
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double sc = 0.0;
+                for (int32_t s = 0; s < cnt[c]; ++s) sc += (double)q[s];
+                sg += sc;
+                q += cnt[c];
+            }
+            S += sg;
         }
     }
     float mu = (float)(S / (double)n);
@@ -223,15 +232,19 @@ void orc_quantize_tensor(const float* v, const int32_t* cnt, int64_t n_chunks, f
     double V = 0.0;
     {
         const float* q = v;
-        for (int64_t c = 0; c < n_chunks; ++c) {
-            double vc = 0.0;
-            for (int32_t s = 0; s < cnt[c]; ++s) {
-                float cen = q[s] - mu;
-                double d = (double)cen;
-                vc += d * d;
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double vg = 0.0;
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double vc = 0.0;
+                for (int32_t s = 0; s < cnt[c]; ++s) {
+                    float cen = q[s] - mu;
+                    double d = (double)cen;
+                    vc += d * d;
+                }
+                vg += vc;
+                q += cnt[c];
             }
-            V += vc;
-            q += cnt[c];
+            V += vg;
         }
     }
     float sigma = (float)sqrt(V / (double)n);
@@ -242,18 +255,22 @@ void orc_quantize_tensor(const float* v, const int32_t* cnt, int64_t n_chunks, f
     {
         const float* q = v;
         uint8_t* cq = code;
-        for (int64_t c = 0; c < n_chunks; ++c) {
-            double sb[4] = {0.0, 0.0, 0.0, 0.0};
-            for (int32_t s = 0; s < cnt[c]; ++s) {
-                float cen = q[s] - mu;
-                int b = (cen >= -t) + (cen >= 0.0f) + (cen >= t);
-                cq[s] = (uint8_t)b;
-                sb[b] += (double)q[s];
-                nb[b] += 1;
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double sgb[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double sb[4] = {0.0, 0.0, 0.0, 0.0};
+                for (int32_t s = 0; s < cnt[c]; ++s) {
+                    float cen = q[s] - mu;
+                    int b = (cen >= -t) + (cen >= 0.0f) + (cen >= t);
+                    cq[s] = (uint8_t)b;
+                    sb[b] += (double)q[s];
+                    nb[b] += 1;
+                }
+                for (int b = 0; b < 4; ++b) sgb[b] += sb[b];
+                q += cnt[c];
+                cq += cnt[c];
             }
-            for (int b = 0; b < 4; ++b) Sb[b] += sb[b];
-            q += cnt[c];
-            cq += cnt[c];
+            for (int b = 0; b < 4; ++b) Sb[b] += sgb[b];
         }
     }
     for (int b = 0; b < 4; ++b) lut[b] = nb[b] ? (float)(Sb[b] / (double)nb[b]) : 0.0f;

@@ -656,7 +656,8 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
 
 // ------------------------------------------------------------------------------------------------
 // Quantiser statistics (Sec. 4).  The summation order is part of the definition of the payload
-// bits: fp64, slot by slot inside a chunk, then chunk by chunk inside the tensor.
+// bits: fp64, in three levels, each left to right: the slots of a chunk, the chunks of a group of 64
+// consecutive chunks of the tensor, the groups.
 // ------------------------------------------------------------------------------------------------
 
 // Visits the keff staged values of one unit in slot order: four 128-bit loads in flight at a time.
@@ -744,16 +745,17 @@ chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
     *reinterpret_cast<uint4*>(ws.pcnt + i * 4) = make_uint4(n0, n1, n2, n3);
 }
 
-// One warp per (worker, tensor): left-to-right fp64 sum of the tensor's chunk partials.  The order is
-// fixed, so the sum is one dependent chain; the warp only feeds it: all lanes fetch the next 32
-// partials while lane 0 adds the previous 32 out of shared memory.
+// One warp per (worker, tensor): the chunk partials are added group by group (64 consecutive chunks
+// per group, left to right inside the group: one lane per group, 32 groups at a time), then the
+// group sums are added left to right.
 // STAGE 0: psum -> mu.  STAGE 1: psum -> sigma, 3 sigma.  STAGE 2: pbin/pcnt -> table (+ payload header).
+constexpr int kSumGroup = 64;
+
 template <int STAGE>
 __global__ void __launch_bounds__(128)
 tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, int n_workers, int n_tensors,
                      Workspace ws, WorkerPtrs ptrs) {
     constexpr int NV = STAGE < 2 ? 1 : 4;  // running sums
-    __shared__ double buf[4][2][NV][32];
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long w = (long long)blockIdx.x * 4 + wib;
     if (w >= (long long)n_workers * n_tensors) return;
@@ -762,51 +764,62 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
     const long long first = (long long)r * n_chunks + ti.first_chunk;
     TStat* st = ws.tstat + (long long)r * n_tensors + t;
     const double n = (double)ti.n_slots;
+    const long long n_groups = (ti.n_chunks + kSumGroup - 1) / kSumGroup;
 
     double acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = 0.0;
     unsigned long long cn[4] = {0, 0, 0, 0};
-    auto fetch = [&](long long c0, double (&x)[NV]) {
+    for (long long g0 = 0; g0 < n_groups; g0 += 32) {
+        // this lane's group
+        double gs[NV];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) x[v] = 0.0;
-        if (c0 + lane < ti.n_chunks) {
-            if (STAGE < 2) {
-                x[0] = ws.psum[first + c0 + lane];
-            } else {
-                const double2* pb = reinterpret_cast<const double2*>(ws.pbin + (first + c0 + lane) * 4);
-                const double2 lo = pb[0], hi = pb[1];
-                x[0] = lo.x; x[1 % NV] = lo.y; x[2 % NV] = hi.x; x[3 % NV] = hi.y;
-                const uint4 pc = *reinterpret_cast<const uint4*>(ws.pcnt + (first + c0 + lane) * 4);
+        for (int v = 0; v < NV; ++v) gs[v] = 0.0;
+        const long long c0 = (g0 + lane) * kSumGroup;
+        const int cnt = (int)max(0ll, min((long long)kSumGroup, ti.n_chunks - c0));
+        if (STAGE < 2) {
+            const double* __restrict__ src = ws.psum + first + c0;
+            int c = 0;
+            for (; c + 8 <= cnt; c += 8) {
+                double x[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) x[q] = src[c + q];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) gs[0] += x[q];
+            }
+            for (; c < cnt; ++c) gs[0] += src[c];
+        } else {
+            const double2* __restrict__ src = reinterpret_cast<const double2*>(ws.pbin + (first + c0) * 4);
+            const uint4* __restrict__ csrc = reinterpret_cast<const uint4*>(ws.pcnt + (first + c0) * 4);
+            int c = 0;
+            for (; c + 4 <= cnt; c += 4) {  // loads of four chunks in flight, additions in chunk order
+                double2 lo[4], hi[4];
+                uint4 pc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    lo[q] = src[2 * (c + q)];
+                    hi[q] = src[2 * (c + q) + 1];
+                    pc[q] = csrc[c + q];
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    gs[0] += lo[q].x; gs[1 % NV] += lo[q].y; gs[2 % NV] += hi[q].x; gs[3 % NV] += hi[q].y;
+                    cn[0] += pc[q].x; cn[1] += pc[q].y; cn[2] += pc[q].z; cn[3] += pc[q].w;
+                }
+            }
+            for (; c < cnt; ++c) {
+                const double2 lo = src[2 * c], hi = src[2 * c + 1];
+                gs[0] += lo.x; gs[1 % NV] += lo.y; gs[2 % NV] += hi.x; gs[3 % NV] += hi.y;
+                const uint4 pc = csrc[c];
                 cn[0] += pc.x; cn[1] += pc.y; cn[2] += pc.z; cn[3] += pc.w;
             }
         }
-    };
-    double x[NV];
-    fetch(0, x);
-    int b = 0;
-    for (long long c0 = 0; c0 < ti.n_chunks; c0 += 32, b ^= 1) {
+        // the group sums of these 32 groups, in group order (every lane runs the same chain)
+        const int ng = (int)min(32ll, n_groups - g0);
+        for (int l = 0; l < ng; ++l) {
 #pragma unroll
-        for (int v = 0; v < NV; ++v) buf[wib][b][v][lane] = x[v];
-        __syncwarp();
-        if (c0 + 32 < ti.n_chunks) fetch(c0 + 32, x);  // in flight during the chain below
-        if (lane == 0) {
-            const int cnt = (int)min((long long)32, ti.n_chunks - c0);
-            if (cnt == 32) {  // unrolled: the shared loads run ahead of the additions
-#pragma unroll
-                for (int l = 0; l < 32; ++l) {
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) acc[v] += buf[wib][b][v][l];
-                }
-            } else {
-                for (int l = 0; l < cnt; ++l) {
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) acc[v] += buf[wib][b][v][l];
-                }
-            }
+            for (int v = 0; v < NV; ++v) acc[v] += __shfl_sync(kFull, gs[v], l);
         }
-        // the buffer written two iterations from now is this one: lane 0 must be done with it
-        __syncwarp();
     }
 
     if (STAGE < 2) {
