@@ -129,6 +129,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // If T is 0 or a class list overflows (constant chunks, heavy ties, large k) an exact bitwise
 // search over all 4096 (key, index) composites finds the keff-th largest instead.
 // ------------------------------------------------------------------------------------------------
+constexpr int kFetchWarp = 7;    // fetches the pending lists: the warp with the least selection work
 constexpr int kClassCap = 224;  // entries per class list (<= threads: one thread per entry suffices)
 
 struct SelectSmem {
@@ -460,7 +461,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             }
         }
     };
-    // warp 0: the pending list of unit (chunk g, worker r) into ring slot `ring`
+    // the fetch warp: the pending list of unit (chunk g, worker r) into ring slot `ring`
     auto issue_pending = [&](int ring, int g, int r) {
         const long long slot_base = ((long long)r * n_chunks + g) * kp;  // kp is a multiple of 8
         if (lane < (kp >> 3)) cp_async16(&sm.pend_idx[ring][8 * lane], ws.idx + slot_base + 8 * lane);
@@ -491,7 +492,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
 
     // prologue: pending lists of units 0..2 (published by the barrier), then units 0 and 1
     if (PENDING) {
-        if (warp == 0) {
+        if (warp == kFetchWarp) {
             for (int j = 0; j < 3 && j < n_units; ++j) {
                 int c2, r2;
                 ahead(0, 0, j, c2, r2);
@@ -595,8 +596,8 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), cd.len, keff, sm.sel, pk);
         if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
 
-        // the stage is consumed (nothing below reads the tile): refill it for unit n + 2; warp 0 also
-        // fetches the pending list of unit n + 3 (its ring slot was last read before the barrier above)
+        // the stage is consumed (nothing below reads the tile): refill it for unit n + 2; the fetch warp
+        // also fetches the pending list of unit n + 3 (its ring slot was last read before the barrier above)
         {
             int c2, r2;
             ahead(c, r, 2, c2, r2);
@@ -608,7 +609,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                 d2.len = dc == 0 ? cd.len : (dc == 1 ? cd1.len : cd2.len);
                 issue_unit(s, d2, r2);
             }
-            if (PENDING && warp == 0) {
+            if (PENDING && warp == kFetchWarp) {
                 ahead(c, r, 3, c2, r2);
                 if (c2 < my_chunks) issue_pending(n % 3, first + c2 * grid, r2);
             }
