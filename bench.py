@@ -158,6 +158,8 @@ def run_ours(args) -> dict:
     sl = SparseLoCo(shapes, offs, k=k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr, alloc_workspace=False)
     deferred = args.ef_subtract == "deferred"
     sl.set_ef_deferred(deferred)
+    if args.tile_copies != "auto":
+        sl.set_tile_copies(args.tile_copies == "tma")
     D = pick_distinct_locals(torch, wl, k, flat, sl.payload_bytes(), sl.workspace_bytes())
     ws = torch.empty(sl.workspace_bytes(), dtype=torch.uint8, device=dev)
     sl.set_workspace(ws)
@@ -229,7 +231,7 @@ def run_ours(args) -> dict:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "params": N, "tensors": len(wl.tensors), "R": wl.R, "k": k, "H": wl.H,
                    "chunk": 4096, "beta": wl.beta, "outer_lr": wl.outer_lr,
-                   "distinct_theta_local_buffers": D,
+                   "distinct_theta_local_buffers": D, "tile_copies": args.tile_copies,
                    "ef_subtract": args.ef_subtract + (" (each step substitutes the previous step's corrected values "
                                                       "while streaming e; a final flush is inside the timed region)"
                                                       if deferred else ""),
@@ -387,6 +389,9 @@ def main():
     ap.add_argument("--ef-subtract", default="deferred", choices=["deferred", "materialised"],
                     help="where e = u - Dhat is applied at the selected positions: in the next step's streaming "
                          "pass (deferred) or by a scattered write in this step (materialised)")
+    ap.add_argument("--tile-copies", default="auto", choices=["auto", "tma", "threads"],
+                    help="how the compression kernel moves 64x64 blocks: tensor-map block copies (the library's "
+                         "default when the table allows) or per-thread 16-byte asynchronous copies")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

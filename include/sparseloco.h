@@ -52,7 +52,8 @@ typedef enum {
     SL_ERR_BAD_PAYLOAD = 4, /* reported through the device status word of sl_validate_payload */
     SL_ERR_CUDA = 5,        /* a CUDA runtime call failed; see sl_last_cuda_error() */
     SL_ERR_NOMEM = 6,       /* workspace missing or too small */
-    SL_ERR_TOO_LARGE = 7    /* problem exceeds a fixed built-in capacity */
+    SL_ERR_TOO_LARGE = 7,   /* problem exceeds a fixed built-in capacity */
+    SL_ERR_TIMEOUT = 8      /* a bounded wait inside a kernel ran out; reported by sl_device_status() */
 } sl_status;
 
 /* One parameter tensor: rows x cols fp32, row-major, at element offset `offset` of every flat
@@ -127,6 +128,20 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
  *   each other; e and payload entries must not. */
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
+
+/* How the compression kernel moves the 64x64 blocks of theta_r and e (no counterpart in the paper).
+ * 1: one tensor-map (TMA) block copy per block and direction, completion on shared-memory barriers --
+ * the default whenever every full chunk starts on a 64-element boundary of the flat buffers (tensor
+ * offsets that are multiples of 64) and the table has at most 8 distinct row lengths; else
+ * UNSUPPORTED.  0: 16-byte asynchronous copies issued by every thread (works for any table).  Results
+ * are identical.  The tensor maps of a buffer are built the first time its pointer is passed in.
+ *
+ * The block-copy kernel waits for its copies with a bounded number of polls; if a wait ever runs
+ * out the kernel records SL_ERR_TIMEOUT in a device status word and returns early, leaving e and the
+ * staged selection of that call undefined.  sl_device_status() synchronises the stream, returns the
+ * recorded status (SL_OK when nothing went wrong) and clears it. */
+sl_status sl_set_tile_copies(sl_ctx* ctx, int32_t use_tensor_maps);
+sl_status sl_device_status(sl_ctx* ctx, void* cuda_stream);
 
 /* Deferred error-feedback subtraction (a storage choice; the paper has no counterpart).  Writing
  * e = u - Dhat at the k selected positions of every chunk after the table is known costs a

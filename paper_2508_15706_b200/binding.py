@@ -19,13 +19,13 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
 PROFILE_SLOTS = 9
 
 SL_OK = 0
 SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_BAD_PAYLOAD = 1, 2, 3, 4
-SL_ERR_CUDA, SL_ERR_NOMEM, SL_ERR_TOO_LARGE = 5, 6, 7
+SL_ERR_CUDA, SL_ERR_NOMEM, SL_ERR_TOO_LARGE, SL_ERR_TIMEOUT = 5, 6, 7, 8
 
 
 class SlError(RuntimeError):
@@ -71,6 +71,8 @@ def _load():
     L.sl_profile_name.argtypes = [C.c_int32]
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_set_tile_copies.argtypes = [P, C.c_int32]
+    L.sl_device_status.argtypes = [P, P]
     L.sl_static_scratch_bytes.restype = C.c_size_t
     L.sl_compress_tensor_static.argtypes = [P, P, P, P, C.c_int64, C.c_int64, C.c_int32, C.c_float, P]
     L.sl_set_ef_deferred.argtypes = [P, C.c_int32]
@@ -242,6 +244,13 @@ class SparseLoCo:
         _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
                                      _dev_ptr(dev_stage, torch.float32), dev_stage.numel(), ea, pa, hp,
                                      _stream()))
+
+    def set_tile_copies(self, use_tensor_maps: bool) -> None:
+        _check(_L.sl_set_tile_copies(self._h, int(use_tensor_maps)))
+
+    def device_status(self) -> int:
+        """Synchronises the current stream; returns (and clears) the status the kernels recorded."""
+        return int(_L.sl_device_status(self._h, _stream()))
 
     def set_ef_deferred(self, on: bool = True) -> None:
         _check(_L.sl_set_ef_deferred(self._h, int(on)))

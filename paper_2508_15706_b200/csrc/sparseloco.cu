@@ -13,6 +13,7 @@
 //
 // Everything is HBM-bound streaming except the per-chunk selection, which works on registers and
 // shared memory.  No tensor cores: nothing here is a dense contraction.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -407,13 +408,80 @@ struct PipeSmem {
     SelectSmem sel;
     __align__(16) float pend_val[3][kMaxK];
     __align__(16) uint16_t pend_idx[3][kMaxK];
+    unsigned long long full_bar[2];  // TMA variant: the stage's tiles have landed
+    int abort;                       // TMA variant: a bounded wait ran out
 };
+
+// ---- TMA variant: tile copies through tensor maps, completion on shared-memory barriers ----------
+// Every flat buffer is described, per distinct row length rs of the tensor table, as a 3-D array
+// [rows][rs / 64][64] (element address = x0 + 64 x1 + rs x2); a 64x64 block is the box {64, 1, 64} at
+// (0, x1, x2) and one copy instruction moves it.  The maps live in global memory, written by the
+// host before the launch.  Waits poll a bounded number of times; when one runs out the kernel
+// records SL_ERR_TIMEOUT and leaves.
+constexpr unsigned kSpinLimit = 1u << 22;
+constexpr int kMaxTmaClasses = 8;
+constexpr int kTmaThread = 32 * 6;  // issues the tile copies (a warp other than the fetch warp, also lightly loaded)
+
+struct TmaArgs {
+    const CUtensorMap* maps;  // [slot][n_classes]
+    int n_classes;
+    int class_rs[kMaxTmaClasses];
+    int slot_l[kMaxR], slot_e[kMaxR];  // map slot of theta_local[r], e[r]
+    int* status;
+};
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// true once the phase of this parity has completed; false after kSpinLimit polls
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity) {
+    const unsigned addr = smem_u32(bar);
+    for (unsigned it = 0; it < kSpinLimit; ++it) {
+        unsigned done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// one 64x64 fp32 block, global -> shared, counted on `bar`
+__device__ __forceinline__ void tma_load_block(void* dst_smem, const CUtensorMap* map, int x1, int x2,
+                                               unsigned long long* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(map), "r"(0), "r"(x1), "r"(x2), "r"(smem_u32(bar))
+        : "memory");
+}
+// one 64x64 fp32 block, shared -> global; joins the calling thread's open bulk group
+__device__ __forceinline__ void tma_store_block(const CUtensorMap* map, int x1, int x2, const void* src_smem) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
+                 "r"(x1), "r"(x2), "r"(smem_u32(src_smem))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// orders this thread's shared-memory writes before later asynchronous-copy reads of them
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // The part of a ChunkDesc the compression kernel needs (its first 16 bytes).
 struct ChunkGeo {
     long long base;
     int row_stride;
     int len;
+    int cls, x1, x2;  // TMA variant: row-length class and block coordinates (set by the kernel)
 };
 __device__ __forceinline__ ChunkGeo load_geo(const ChunkDesc* d) {
     const int4 v = __ldg(reinterpret_cast<const int4*>(d));
@@ -421,14 +489,15 @@ __device__ __forceinline__ ChunkGeo load_geo(const ChunkDesc* d) {
     g.base = ((long long)v.y << 32) | (unsigned)v.x;
     g.row_stride = v.z;
     g.len = v.w;
+    g.cls = g.x1 = g.x2 = 0;
     return g;
 }
 
-template <bool EF, bool PENDING>
+template <bool EF, bool PENDING, bool TMA>
 __global__ void __launch_bounds__(kThreads, 3)
 ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
-               const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
-    extern __shared__ __align__(128) unsigned char dyn_smem[];
+               const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma) {
+    extern __shared__ __align__(1024) unsigned char dyn_smem[];
     PipeSmem& sm = *reinterpret_cast<PipeSmem*>(dyn_smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // 32-bit counters: chunks x workers < 2^31 is checked on the host
@@ -439,6 +508,12 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
     if (tid < 128) {
         sm.sel.bitmap[0][tid] = 0;
         sm.sel.bitmap[1][tid] = 0;
+    }
+    if (TMA && tid == kTmaThread) {
+        mbar_init(&sm.full_bar[0], 1);
+        mbar_init(&sm.full_bar[1], 1);
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
     // This thread's i-th vector (in-chunk indices 512 warp + 128 i + 4 lane ..+3) lies in block row
@@ -460,6 +535,32 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                 if (EF) cp_async16(&sm.e[s][slot0 + 128 * i], er + i * step);
             }
         }
+    };
+    // TMA variant: block coordinates in the 3-D view of row length rs, once per chunk
+    auto with_coords = [&](ChunkGeo d) {
+        if (TMA) {
+            const int rs = row_elems(d);
+            d.cls = 0;
+            for (int q = 1; q < tma.n_classes; ++q) d.cls = tma.class_rs[q] == rs ? q : d.cls;
+            d.x2 = (int)(d.base / rs);
+            d.x1 = (int)(d.base - (long long)d.x2 * rs) >> 6;
+        }
+        return d;
+    };
+    // arms the stage barrier for one unit and starts its theta_r block (a short chunk moves nothing)
+    auto tma_begin_unit = [&](int s, const ChunkGeo& d, int r) {
+        unsigned long long* bar = &sm.full_bar[s];
+        if (d.len != kChunk) {
+            mbar_arrive(bar);
+            return;
+        }
+        mbar_arrive_expect_tx(bar, (EF ? 2u : 1u) * kChunk * (unsigned)sizeof(float));
+        tma_load_block(sm.theta_l[s], tma.maps + tma.slot_l[r] * tma.n_classes + d.cls, d.x1, d.x2, bar);
+    };
+    // the e block of a unit begun earlier
+    auto tma_load_e = [&](int s, const ChunkGeo& d, int r) {
+        if (!EF || d.len != kChunk) return;
+        tma_load_block(sm.e[s], tma.maps + tma.slot_e[r] * tma.n_classes + d.cls, d.x1, d.x2, &sm.full_bar[s]);
     };
     // the fetch warp: the pending list of unit (chunk g, worker r) into ring slot `ring`
     auto issue_pending = [&](int ring, int g, int r) {
@@ -486,9 +587,9 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
     };
 
     // descriptors of this CTA's current chunk and the two after it
-    ChunkGeo cd = load_geo(chunks + first), cd1 = cd, cd2 = cd;
-    if (my_chunks > 1) cd1 = load_geo(chunks + first + grid);
-    if (my_chunks > 2) cd2 = load_geo(chunks + first + 2 * grid);
+    ChunkGeo cd = with_coords(load_geo(chunks + first)), cd1 = cd, cd2 = cd;
+    if (my_chunks > 1) cd1 = with_coords(load_geo(chunks + first + grid));
+    if (my_chunks > 2) cd2 = with_coords(load_geo(chunks + first + 2 * grid));
 
     // prologue: pending lists of units 0..2 (published by the barrier), then units 0 and 1
     if (PENDING) {
@@ -503,9 +604,20 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         cp_async_wait<0>();
     }
     __syncthreads();
-    issue_unit(0, cd, 0);
+    if (TMA) {
+        if (tid == kTmaThread) {
+            tma_begin_unit(0, cd, 0);
+            tma_load_e(0, cd, 0);
+            if (n_units > 1) {
+                tma_begin_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
+                tma_load_e(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
+            }
+        }
+    } else {
+        issue_unit(0, cd, 0);
+    }
     cp_async_commit();
-    if (n_units > 1) issue_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
+    if (!TMA && n_units > 1) issue_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
     cp_async_commit();
 
     float4 ts[4];
@@ -514,7 +626,8 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
     load_theta_s(ts, cd);
 
     int c = 0, r = 0;  // chunk ordinal within this CTA, worker
-    for (int n = 0; n < n_units; ++n) {
+    int n = 0;
+    for (; n < n_units; ++n) {
         const int s = n & 1;
         const bool full = cd.len == kChunk;
         const int keff = min(k, cd.len);
@@ -524,6 +637,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         float* tile = sm.e[s];
 
         cp_async_wait<1>();  // this unit's copies have landed (only the next unit's may be in flight)
+        if (TMA && !mbar_wait(&sm.full_bar[s], (unsigned)((n >> 1) & 1))) sm.abort = 1;
 
         if (PENDING && EF) {  // substitute the corrected values of the previous step
             const int ring = n % 3;
@@ -561,7 +675,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                     u.y = __fmaf_rn(beta, ev.y, u.y);
                     u.z = __fmaf_rn(beta, ev.z, u.z);
                     u.w = __fmaf_rn(beta, ev.w, u.w);
-                    *reinterpret_cast<float4*>(er_vec + i * er_step) = u;
+                    if (!TMA) *reinterpret_cast<float4*>(er_vec + i * er_step) = u;
                 }
                 *reinterpret_cast<float4*>(&tile[v]) = u;
                 ub[4 * i + 0] = __float_as_uint(u.x);
@@ -569,6 +683,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                 ub[4 * i + 2] = __float_as_uint(u.z);
                 ub[4 * i + 3] = __float_as_uint(u.w);
             }
+            if (TMA && EF) fence_async_smem();  // the tile is about to be read by a block store
         } else {  // short tail of a flat tensor: element-wise with bounds
             const float* __restrict__ tsp = theta_sync + cd.base;
             const float* __restrict__ tl = ptrs.theta_local[r] + cd.base;
@@ -596,28 +711,50 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), cd.len, keff, sm.sel, pk);
         if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
 
-        // the stage is consumed (nothing below reads the tile): refill it for unit n + 2; the fetch warp
-        // also fetches the pending list of unit n + 3 (its ring slot was last read before the barrier above)
+        // refill for unit n + 2.  cp.async variant: the whole stage is consumed (nothing below reads
+        // the tile).  TMA variant: one thread stores u, re-arms the stage and starts theta_r; e follows
+        // once the selection and the store are done with the tile.  The fetch warp also fetches the
+        // pending list of unit n + 3 (its ring slot was last read before the barrier above).
+        if (TMA && *reinterpret_cast<volatile int*>(&sm.abort)) break;  // uniform: written before the barrier above
+        int c2, r2;  // unit n + 2 and its chunk
+        ahead(c, r, 2, c2, r2);
+        const bool have2 = c2 < my_chunks;
+        ChunkGeo d2;  // picked field by field: keeps the three descriptors in registers
         {
-            int c2, r2;
-            ahead(c, r, 2, c2, r2);
-            if (c2 < my_chunks) {
-                const int dc = c2 - c;
-                ChunkGeo d2;  // picked field by field: keeps the three descriptors in registers
-                d2.base = dc == 0 ? cd.base : (dc == 1 ? cd1.base : cd2.base);
-                d2.row_stride = dc == 0 ? cd.row_stride : (dc == 1 ? cd1.row_stride : cd2.row_stride);
-                d2.len = dc == 0 ? cd.len : (dc == 1 ? cd1.len : cd2.len);
-                issue_unit(s, d2, r2);
-            }
-            if (PENDING && warp == kFetchWarp) {
-                ahead(c, r, 3, c2, r2);
-                if (c2 < my_chunks) issue_pending(n % 3, first + c2 * grid, r2);
-            }
-            cp_async_commit();
+            const int dc = c2 - c;
+            d2.base = dc == 0 ? cd.base : (dc == 1 ? cd1.base : cd2.base);
+            d2.row_stride = dc == 0 ? cd.row_stride : (dc == 1 ? cd1.row_stride : cd2.row_stride);
+            d2.len = dc == 0 ? cd.len : (dc == 1 ? cd1.len : cd2.len);
+            d2.cls = dc == 0 ? cd.cls : (dc == 1 ? cd1.cls : cd2.cls);
+            d2.x1 = dc == 0 ? cd.x1 : (dc == 1 ? cd1.x1 : cd2.x1);
+            d2.x2 = dc == 0 ? cd.x2 : (dc == 1 ? cd1.x2 : cd2.x2);
         }
+        if (TMA) {
+            if (tid == kTmaThread) {
+                if (EF && full) {  // u back into e: every thread fenced its writes before the barrier above
+                    tma_store_block(tma.maps + tma.slot_e[r] * tma.n_classes + cd.cls, cd.x1, cd.x2, tile);
+                    bulk_commit();
+                }
+                if (have2) tma_begin_unit(s, d2, r2);  // the theta_r stage was last read before that barrier
+            }
+        } else if (have2) {
+            issue_unit(s, d2, r2);
+        }
+        if (PENDING && warp == kFetchWarp) {
+            int c3, r3;
+            ahead(c, r, 3, c3, r3);
+            if (c3 < my_chunks) issue_pending(n % 3, first + c3 * grid, r3);
+        }
+        cp_async_commit();
 
+        bool e_started = false;  // TMA variant: the e block of unit n + 2 is on its way
         if (!exact) {
-            __syncthreads();  // class lists complete
+            __syncthreads();  // class lists complete: nobody reads the tile any more except the block store
+            if (TMA && EF && tid == kTmaThread) {
+                if (full) bulk_wait_read_all();  // once the store has read the tile, refill it
+                if (have2) tma_load_e(s, d2, r2);
+            }
+            e_started = true;
             exact = select_rank(keff, sm.sel, bitmap, pk);
         }
         if (exact) {
@@ -631,6 +768,10 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             select_exact_search(tmp, nonzero, cd.len, keff, sm.sel, bitmap);
         }
         __syncthreads();  // the map is complete
+        if (TMA && EF && !e_started && tid == kTmaThread) {  // the exact search came straight from the threshold
+            if (full) bulk_wait_read_all();
+            if (have2) tma_load_e(s, d2, r2);
+        }
         if (exact) {
             pk.mask = 0;
             if (tid < (int)sm.sel.n_exact) {
@@ -649,10 +790,19 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             ++c;
             cd = cd1;
             cd1 = cd2;
-            if (c + 2 < my_chunks) cd2 = load_geo(chunks + first + (c + 2) * grid);
+            if (c + 2 < my_chunks) cd2 = with_coords(load_geo(chunks + first + (c + 2) * grid));
         }
     }
     cp_async_wait<0>();
+    if (TMA) {
+        if (n < n_units) {
+            // A wait ran out.  Report it, then give the copies still in flight a bounded time to
+            // land before the shared memory they target is released.
+            if (tid == 0) atomicExch(tma.status, (int)SL_ERR_TIMEOUT);
+            for (int u = n; u < n + 2 && u < n_units; ++u) mbar_wait(&sm.full_bar[u & 1], (unsigned)((u >> 1) & 1));
+        }
+        if (tid == kTmaThread) bulk_wait_all();
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1132,6 +1282,15 @@ struct sl_ctx {
     ChunkDesc* d_chunks;
     TensorInfo* d_tinfo;
     int ef_ctas;  // resident CTAs of the persistent compression kernel on this device
+    // tensor-map (TMA) block copies: usable when every full chunk starts on a 64-element boundary
+    bool tma_ok, tma_on;
+    int n_classes;
+    int class_rs[kMaxTmaClasses];       // distinct row lengths of full chunks (64 for flat runs)
+    CUtensorMap* d_maps;                // [kMapSlots][n_classes]
+    std::vector<CUtensorMap> h_maps;    // host copy the device array is filled from
+    std::vector<const void*> slot_ptr;  // buffer described by each slot
+    bool slots_cleared;                 // the slot table was emptied during the current assignment
+    int* d_status;                      // device status word (SL_OK or what a kernel recorded)
     bool deferred;              // deferred error-feedback subtraction (sl_set_ef_deferred)
     bool pending;               // corrected values of the last step still wait in the workspace
     float* pending_e[kMaxR];    // the error buffers they belong to
@@ -1149,6 +1308,24 @@ struct sl_ctx {
 };
 
 namespace {
+
+constexpr int kMapSlots = 2 * kMaxR + 2;  // buffers with tensor maps at one time: theta_local and e of every worker
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
+typedef CUresult (*TmaEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TmaEncodeFn tma_encode_fn() {
+    static TmaEncodeFn fn = []() -> TmaEncodeFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<TmaEncodeFn>(p);
+    }();
+    return fn;
+}
 
 sl_status cuda_fail(cudaError_t e, const char* what) {
     snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
@@ -1192,6 +1369,36 @@ inline void prof_mark(sl_ctx* c, int slot, cudaStream_t st) {
     cudaEventRecord(c->prof_events[(size_t)c->prof_steps * (kProfSlots + 1) + (slot + 1)], st);
 }
 
+// Slot of the tensor maps that describe the flat buffer at `ptr` (one map per row-length class);
+// encodes and uploads them (ordered on `st`) the first time the pointer is seen.  -1 on failure.
+int tma_map_slot(sl_ctx* c, const void* ptr, cudaStream_t st) {
+    for (size_t i = 0; i < c->slot_ptr.size(); ++i)
+        if (c->slot_ptr[i] == ptr) return (int)i;
+    if ((int)c->slot_ptr.size() == kMapSlots) {  // full: start over (uploads are ordered after earlier launches)
+        c->slot_ptr.clear();
+        c->slots_cleared = true;
+    }
+    const int slot = (int)c->slot_ptr.size();
+    TmaEncodeFn enc = tma_encode_fn();
+    for (int q = 0; q < c->n_classes; ++q) {
+        const cuuint64_t rs = (cuuint64_t)c->class_rs[q];
+        const cuuint64_t dims[3] = {(cuuint64_t)kTile, rs / kTile, ((cuuint64_t)c->flat_elems + rs - 1) / rs + 1};
+        const cuuint64_t strides[2] = {kTile * sizeof(float), rs * sizeof(float)};  // bytes, dimensions 1 and 2
+        const cuuint32_t box[3] = {(cuuint32_t)kTile, 1u, (cuuint32_t)kTile};
+        const cuuint32_t estr[3] = {1u, 1u, 1u};
+        CUtensorMap* m = &c->h_maps[(size_t)slot * c->n_classes + q];
+        if (enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return -1;
+    }
+    if (cudaMemcpyAsync(c->d_maps + (size_t)slot * c->n_classes, &c->h_maps[(size_t)slot * c->n_classes],
+                        sizeof(CUtensorMap) * c->n_classes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return -1;
+    c->slot_ptr.push_back(ptr);
+    return slot;
+}
+
 sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
     const int R = c->cfg.R;
     const Workspace ws = carve(c, R);
@@ -1226,18 +1433,44 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
         c->pending = false;
     }
 
+    // tile copies through tensor maps when the table allows it and every buffer got its maps
+    TmaArgs ta;
+    memset(&ta, 0, sizeof(ta));
+    bool use_tma = c->tma_on;
+    if (use_tma) {
+        ta.maps = c->d_maps;
+        ta.n_classes = c->n_classes;
+        ta.status = c->d_status;
+        for (int q = 0; q < c->n_classes; ++q) ta.class_rs[q] = c->class_rs[q];
+        for (int pass = 0; pass < 2 && use_tma; ++pass) {
+            // if the slot table fills up half-way, it is emptied and the assignment starts over: one
+            // call needs at most 2 R slots, which an empty table holds
+            c->slots_cleared = false;
+            for (int r = 0; r < workers && use_tma; ++r) {
+                ta.slot_l[r] = tma_map_slot(c, ptrs.theta_local[r], st);
+                ta.slot_e[r] = ef ? tma_map_slot(c, ptrs.e[r], st) : 0;
+                use_tma = ta.slot_l[r] >= 0 && ta.slot_e[r] >= 0;
+            }
+            if (!c->slots_cleared) break;
+        }
+    }
+
     prof_mark(c, -1, st);
     const unsigned ef_grid = (unsigned)(G < c->ef_ctas ? G : c->ef_ctas);  // persistent CTAs
     const size_t smem = sizeof(PipeSmem);
-    if (!ef)
-        ef_topk_kernel<false, false><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                      theta_sync, ptrs, ws);
-    else if (consume)
-        ef_topk_kernel<true, true><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                    theta_sync, ptrs, ws);
-    else
-        ef_topk_kernel<true, false><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta,
-                                                                     theta_sync, ptrs, ws);
+#define SL_LAUNCH_EF(EFV, PENDV, TMAV)                                                                          \
+    ef_topk_kernel<EFV, PENDV, TMAV><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta, \
+                                                                      theta_sync, ptrs, ws, ta)
+    if (use_tma) {
+        if (!ef) SL_LAUNCH_EF(false, false, true);
+        else if (consume) SL_LAUNCH_EF(true, true, true);
+        else SL_LAUNCH_EF(true, false, true);
+    } else {
+        if (!ef) SL_LAUNCH_EF(false, false, false);
+        else if (consume) SL_LAUNCH_EF(true, true, false);
+        else SL_LAUNCH_EF(true, false, false);
+    }
+#undef SL_LAUNCH_EF
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
@@ -1319,6 +1552,7 @@ const char* sl_strerror(sl_status s) {
         case SL_ERR_CUDA: return "CUDA error";
         case SL_ERR_NOMEM: return "workspace missing or too small";
         case SL_ERR_TOO_LARGE: return "problem exceeds a built-in capacity";
+        case SL_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     }
     return "unknown status";
 }
@@ -1343,6 +1577,11 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->d_chunks = nullptr;
     c->d_tinfo = nullptr;
     c->ef_ctas = 0;
+    c->tma_ok = c->tma_on = false;
+    c->slots_cleared = false;
+    c->n_classes = 0;
+    c->d_maps = nullptr;
+    c->d_status = nullptr;
     c->deferred = false;
     c->pending = false;
     c->ws_ptr = nullptr;
@@ -1405,20 +1644,50 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     }
     c->n_chunks = (long long)chunks.size();
     c->n_slots = slots;
+    {   // row-length classes of the full chunks; block copies need 64-element alignment of every block
+        bool ok = true;
+        int ncls = 0;
+        for (const ChunkDesc& d : chunks) {
+            if (d.len != kChunk) continue;
+            if (d.base % kTile != 0) { ok = false; break; }
+            const int rs = d.row_stride ? d.row_stride : kTile;
+            int q = 0;
+            while (q < ncls && c->class_rs[q] != rs) ++q;
+            if (q == ncls) {
+                if (ncls == kMaxTmaClasses) { ok = false; break; }
+                c->class_rs[ncls++] = rs;
+            }
+        }
+        c->n_classes = ncls;
+        c->tma_ok = ok && ncls > 0 && tma_encode_fn() != nullptr;
+        c->tma_on = c->tma_ok;
+    }
     c->flat_elems = flat;
 
     cudaError_t e = cudaGetDevice(&c->device);
     int n_sms = 0, per_sm = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    const int smem_bytes = (int)sizeof(PipeSmem);
+#define SL_SMEM_ATTR(...)                                                                                      \
+    if (e == cudaSuccess)                                                                                      \
+        e = cudaFuncSetAttribute(ef_topk_kernel<__VA_ARGS__>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)
+    SL_SMEM_ATTR(true, false, false);
+    SL_SMEM_ATTR(false, false, false);
+    SL_SMEM_ATTR(true, true, false);
+    SL_SMEM_ATTR(true, false, true);
+    SL_SMEM_ATTR(false, false, true);
+    SL_SMEM_ATTR(true, true, true);
+#undef SL_SMEM_ATTR
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_topk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_topk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PipeSmem));
-    if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true>, kThreads, sizeof(PipeSmem));
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true>, kThreads,
+                                                          sizeof(PipeSmem));
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
+    if (c->tma_ok) {
+        c->h_maps.resize((size_t)kMapSlots * c->n_classes);
+        if (e == cudaSuccess) e = cudaMalloc(&c->d_maps, sizeof(CUtensorMap) * kMapSlots * c->n_classes);
+    }
     if (e == cudaSuccess) e = cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkDesc));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_tinfo, tinfo.size() * sizeof(TensorInfo));
     if (e == cudaSuccess)
@@ -1429,6 +1698,8 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
         sl_status s = cuda_fail(e, "sl_create");
         if (c->d_chunks) cudaFree(c->d_chunks);
         if (c->d_tinfo) cudaFree(c->d_tinfo);
+        if (c->d_status) cudaFree(c->d_status);
+        if (c->d_maps) cudaFree(c->d_maps);
         delete c;
         return s;
     }
@@ -1441,6 +1712,8 @@ sl_status sl_destroy(sl_ctx* c) {
     DeviceGuard g(c->device);
     cudaFree(c->d_chunks);
     cudaFree(c->d_tinfo);
+    cudaFree(c->d_status);
+    cudaFree(c->d_maps);
     for (auto& ev : c->prof_events) cudaEventDestroy(ev);
     if (c->host_path_ready) {
         cudaStreamDestroy(c->copy_stream);
@@ -1659,6 +1932,25 @@ const char* sl_profile_name(int32_t slot) {
     return slot >= 0 && slot < kProfSlots ? names[slot] : "";
 }
 
+sl_status sl_set_tile_copies(sl_ctx* c, int32_t use_tensor_maps) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    if (use_tensor_maps && !c->tma_ok) return SL_ERR_UNSUPPORTED;
+    c->tma_on = use_tensor_maps != 0;
+    return SL_OK;
+}
+
+sl_status sl_device_status(sl_ctx* c, void* stream) {
+    if (!c) return SL_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    SL_CUDA(cudaMemcpyAsync(&v, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SL_CUDA(cudaStreamSynchronize(st));
+    if (v != (int)SL_OK) SL_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(int), st));
+    return (sl_status)v;
+}
+
 sl_status sl_set_ef_deferred(sl_ctx* c, int32_t on) {
     if (!c) return SL_ERR_INVALID_ARG;
     c->deferred = on != 0;
@@ -1813,9 +2105,9 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
         SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
         int n_sms = 0, per_sm = 0;
         SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)sizeof(PipeSmem)));
-        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false>, kThreads,
+        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false, false>, kThreads,
                                                               sizeof(PipeSmem)));
         su.scratch = ptr;
         su.ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
@@ -1842,8 +2134,10 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     // by an earlier call (of any size) is ever consumed and nothing has to be cleared.
     build_single_tensor_table_kernel<<<blocks_for(G, 128), 128, 0, st>>>(rows, cols, k, G, d_chunks, d_tinfo);
     const unsigned ef_grid = (unsigned)(G < su.ef_ctas ? G : su.ef_ctas);
-    ef_topk_kernel<true, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
-                                                                            ptrs, ws);
+    TmaArgs no_tma;
+    memset(&no_tma, 0, sizeof(no_tma));
+    ef_topk_kernel<true, false, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
+                                                                                   theta_sync, ptrs, ws, no_tma);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
     tensor_reduce_kernel<0><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);

@@ -81,6 +81,7 @@ class DeviceCase:
 
     def step(self) -> None:
         self.sl.outer_step(self.theta, [self.local_of(r) for r in range(self.wl.R)], self.e, self.payloads)
+        assert self.sl.device_status() == 0, "a kernel recorded a device-side error"
 
     def tensor_payload(self, r: int, j: int) -> np.ndarray:
         p = self.payloads[r]

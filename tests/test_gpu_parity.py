@@ -144,6 +144,43 @@ def test_deferred_subtraction_is_bit_identical(k):
         assert torch.equal(d.e[r], c2.e[r]) and torch.equal(d.payloads[r], c2.payloads[r])
 
 
+ALIGNED = [I.TensorSpec("a", 128, 192, 0), I.TensorSpec("flat", 1, 4096 * 2 + 1024, 0), I.TensorSpec("wide", 64, 512, 1),
+           I.TensorSpec("norm", 1, 768, 1), I.TensorSpec("b", 192, 64, 2), I.TensorSpec("tail", 1, 4096 + 64 * 7, 2)]
+
+
+@pytest.mark.parametrize("deferred", [False, True])
+def test_tensor_map_copies_match_oracle_and_per_thread_copies(deferred):
+    """A table whose blocks all start on 64-element boundaries takes the tensor-map (TMA) block copies;
+    the same steps with the per-thread copies must give the same bits, and both match the oracle."""
+    from paper_2508_15706_b200 import binding as B
+    wl = I.Workload("aligned", ALIGNED, R=3, k=64, recipe="student_t4", seed=77, outer_lr=0.9)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    a.sl.set_tile_copies(True)    # raises if the table were not eligible
+    b.sl.set_tile_copies(False)
+    for c in (a, b):
+        c.sl.set_ef_deferred(deferred)
+    for step in range(3):
+        for c in (a, b):
+            c.fill_local(step)
+        snap = a.snapshot(range(len(ALIGNED)))
+        a.step()
+        b.step()
+        a.check(snap)
+        assert torch.equal(a.theta, b.theta)
+        for r in range(3):
+            assert torch.equal(a.payloads[r], b.payloads[r])
+    ea, eb = a.true_error(), b.true_error()
+    torch.cuda.synchronize()
+    for x, y in zip(ea, eb):
+        assert torch.equal(x, y)
+    # a table with an odd offset cannot use block copies
+    sl = B.SparseLoCo([(1, 100), (64, 64)], k=8, R=1)
+    with pytest.raises(B.SlError) as ei:
+        sl.set_tile_copies(True)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+
+
 def test_compress_then_aggregate_equals_outer_step_and_absent_workers():
     import oracle as O
     wl = I.Workload("split", SMALL, R=3, k=64, recipe="normal", seed=51, outer_lr=0.8)
