@@ -238,7 +238,7 @@ def run_ours(args) -> dict:
                    "l2": "inputs larger than L2 (every buffer is %.1f GB; state evolves every step)" % (4 * flat / 1e9),
                    "multi_gpu": "replicas only (no data-path collective)"},
         "clocks": clocks,
-        "gpu_launches": 9 * args.steps + (1 if deferred else 0),
+        "gpu_launches": 8 * args.steps + (1 if deferred else 0),
         "roofline": {"bound": "hbm", "kernel": "ef_topk", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": ef_bytes, "avg_launch_ms": ef_avg_ms,

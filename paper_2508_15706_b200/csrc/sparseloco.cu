@@ -1091,15 +1091,26 @@ __device__ __forceinline__ unsigned get2(const unsigned* rec, int code_byte0, in
 
 constexpr int kApplyEntries = 8;  // entries per thread and batch
 
-template <int SPL>  // slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8
+// FUSE 0: the entries come from the payload records (sl_aggregate_apply).  FUSE 1 / 2: the whole outer
+// step is running and the records do not exist yet: the entries come from the staging arrays, get
+// their codes here, and the kernel also writes the records and the error correction, i.e. it does
+// what pack_fix_kernel<1> / <2> does, saving that kernel's pass and the re-read of the records.
+struct FuseArgs {
+    Workspace ws;
+    long long n_chunks;
+    int n_tensors, kp;
+};
+
+template <int SPL, int FUSE>  // SPL = slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8
 __global__ void __launch_bounds__(kThreads, 4)
 decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale,
-                        PayloadPtrs pl, float* __restrict__ theta_sync) {
+                        PayloadPtrs pl, float* __restrict__ theta_sync, FuseArgs fa, WorkerPtrs ptrs) {
     extern __shared__ __align__(16) unsigned char dyn[];
     float* acc = reinterpret_cast<float*>(dyn);                            // 4096 sums
     unsigned* wmask = reinterpret_cast<unsigned*>(acc + kChunk);           // 4096 worker masks
     float* luts = reinterpret_cast<float*>(wmask + kChunk);                // 32 x 4
-    unsigned* recs = reinterpret_cast<unsigned*>(luts + 4 * 32);           // batch x (stride + 16) bytes
+    float* mu_t3 = luts + 4 * 32;                                          // 32 x 2 (FUSE: mean, 3 sigma)
+    unsigned* recs = reinterpret_cast<unsigned*>(mu_t3 + 2 * 32);          // batch x (stride + 16) bytes
     const int stride = record_stride(k), rwords = stride / 4 + 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const ChunkDesc cd = chunks[blockIdx.x];
@@ -1128,22 +1139,53 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
 
     for (int r0 = 0; r0 < n_workers; r0 += batch) {
         const int nb = min(batch, n_workers - r0);
+        unsigned pre_p[kApplyEntries];
+        float pre_v[kApplyEntries];
+#pragma unroll
+        for (int e = 0; e < kApplyEntries; ++e) {
+            pre_p[e] = 0u;
+            pre_v[e] = 0.f;
+        }
         // clear the masks, stage this batch's records and tables (the last barrier of the
         // previous batch's rounds has released both)
 #pragma unroll
         for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(wmask + 1024 * i + 4 * tid) = make_uint4(0u, 0u, 0u, 0u);
-        for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
-            const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
-            const uint8_t* src = pl.p[r0 + rb];
-            if (src) {
-                const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + cd.rec_off) + w);
-                *reinterpret_cast<uint4*>(recs + rb * rwords + 4 * w) = x;
+        if (FUSE == 0) {
+            for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
+                const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
+                const uint8_t* src = pl.p[r0 + rb];
+                if (src) {
+                    const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + cd.rec_off) + w);
+                    *reinterpret_cast<uint4*>(recs + rb * rwords + 4 * w) = x;
+                }
             }
-        }
-        if (tid < nb) {
-            const uint8_t* src = pl.p[r0 + tid];
-            if (src) *reinterpret_cast<float4*>(luts + 4 * tid) = __ldg(reinterpret_cast<const float4*>(src + 16ll * cd.tensor));
-            recs[tid * rwords + stride / 4] = 0;  // word read past the index block by get12
+            if (tid < nb) {
+                const uint8_t* src = pl.p[r0 + tid];
+                if (src) *reinterpret_cast<float4*>(luts + 4 * tid) = __ldg(reinterpret_cast<const float4*>(src + 16ll * cd.tensor));
+                recs[tid * rwords + stride / 4] = 0;  // word read past the index block by get12
+            }
+        } else {
+            // staged (index, value) pairs of this thread's entries: loads in flight across the barrier
+#pragma unroll
+            for (int wi = 0; wi < WPW; ++wi) {
+                const int rb = warp + 8 * wi;
+                const long long slot_base = ((long long)(r0 + rb) * fa.n_chunks + blockIdx.x) * fa.kp;
+#pragma unroll
+                for (int si = 0; si < SPL; ++si) {
+                    const int sl = lane + 32 * si;
+                    if (rb < nb && sl < keff) {
+                        pre_p[wi * SPL + si] = fa.ws.idx[slot_base + sl];
+                        pre_v[wi * SPL + si] = fa.ws.val[slot_base + sl];
+                    }
+                }
+            }
+            for (int w = tid; w < nb * rwords; w += kThreads) recs[w] = 0;  // the records are assembled here
+            if (tid < nb) {
+                const TStat st = fa.ws.tstat[(long long)(r0 + tid) * fa.n_tensors + cd.tensor];
+                *reinterpret_cast<float4*>(luts + 4 * tid) = make_float4(st.lut[0], st.lut[1], st.lut[2], st.lut[3]);
+                mu_t3[2 * tid] = st.mu;
+                mu_t3[2 * tid + 1] = st.t3;
+            }
         }
         __syncthreads();
 
@@ -1158,14 +1200,32 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
         for (int wi = 0; wi < WPW; ++wi) {
             const int rb = warp + 8 * wi;
             if (rb < nb && pl.p[r0 + rb]) {  // uniform over the warp
-                const unsigned* rec = recs + rb * rwords;
+                unsigned* rec = recs + rb * rwords;
+                const long long slot_base = FUSE ? ((long long)(r0 + rb) * fa.n_chunks + blockIdx.x) * fa.kp : 0;
 #pragma unroll
                 for (int si = 0; si < SPL; ++si) {
                     const int sl = lane + 32 * si;
                     if (sl < keff) {
-                        const unsigned p = get12(rec, sl);
+                        unsigned p, code;
+                        if (FUSE == 0) {
+                            p = get12(rec, sl);
+                            code = get2(rec, code_byte0, sl);
+                        } else {
+                            p = pre_p[wi * SPL + si];
+                            const float v = pre_v[wi * SPL + si];
+                            code = (unsigned)quant_code(v, mu_t3[2 * rb], mu_t3[2 * rb + 1]);
+                            const int bit = 12 * sl;
+                            atomicOr(&rec[bit >> 5], p << (bit & 31));
+                            if ((bit & 31) > 20) atomicOr(&rec[(bit >> 5) + 1], p >> (32 - (bit & 31)));
+                            const int cbit = code_byte0 * 8 + 2 * sl;
+                            atomicOr(&rec[cbit >> 5], code << (cbit & 31));
+                            const float fixed = __fsub_rn(v, luts[4 * rb + code]);
+                            if (FUSE == 1 && p < (unsigned)cd.len)
+                                ptrs.e[r0 + rb][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = fixed;
+                            if (FUSE == 2) fa.ws.val[slot_base + sl] = fixed;
+                        }
                         if (p < (unsigned)cd.len) {
-                            ent_v[wi * SPL + si] = luts[4 * rb + get2(rec, code_byte0, sl)];
+                            ent_v[wi * SPL + si] = luts[4 * rb + code];
                             ent_p[wi * SPL + si] = p | ((unsigned)rb << 12);
                             atomicOr(&wmask[p], 1u << rb);
                         }
@@ -1174,6 +1234,13 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
             }
         }
         __syncthreads();
+        if (FUSE) {  // the records are complete: out they go
+            for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
+                const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
+                reinterpret_cast<uint4*>(ptrs.payload[r0 + rb] + cd.rec_off)[w] =
+                    *reinterpret_cast<const uint4*>(recs + rb * rwords + 4 * w);
+            }
+        }
         // rank of every entry among the workers at its position; round 0
         int my_max = 0;
 #pragma unroll
@@ -1410,8 +1477,9 @@ sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
 
 // Compression of `workers` workers whose pointers are in `ptrs` (kernels 1-8).  `defer`: leave the
 // corrected values in the workspace instead of writing them into e (only with all R workers).
+// `skip_pack`: the caller runs the packing step fused into the apply kernel right after.
 sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const WorkerPtrs& ptrs,
-                          cudaStream_t st, bool defer) {
+                          cudaStream_t st, bool defer, bool skip_pack = false) {
     if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, workers)) return SL_ERR_NOMEM;
     const Workspace ws = carve(c, workers);
     c->last_workers = workers;
@@ -1486,7 +1554,9 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 6, st);
     const unsigned pb = blocks_for(WG, 4);
-    if (!ef)
+    if (skip_pack)
+        ;  // records, error correction: done by decode_avg_apply_kernel<., 1 or 2>
+    else if (!ef)
         pack_fix_kernel<0><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     else if (defer)
         pack_fix_kernel<2><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
@@ -1501,24 +1571,41 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     return SL_OK;
 }
 
-sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* theta_sync, cudaStream_t st) {
+// fuse: 0 = payloads in, 1 / 2 = also do the packing step of a compression in flight (see the kernel)
+sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* theta_sync, cudaStream_t st, int fuse = 0,
+                       const WorkerPtrs* fuse_ptrs = nullptr) {
     if (present == 0) return SL_OK;
     const int R = c->cfg.R;
     const double D = c->cfg.divide_by_present ? (double)present : (double)R;
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
     const int stride = record_stride(c->cfg.k);
     const int nb = R < 32 ? R : 32;  // the kernel never stages more than 32 records at once
-    const size_t smem = (size_t)kChunk * 8 + 32 * 16 + (size_t)nb * (stride + 16);
-    if (smem > 48 * 1024) {
-        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    }
+    const size_t smem = (size_t)kChunk * 8 + 32 * 24 + (size_t)nb * (stride + 16);
     const int spl = (c->cfg.k + 31) / 32;
-    auto kern = spl <= 1 ? decode_avg_apply_kernel<1> : spl <= 2 ? decode_avg_apply_kernel<2>
-              : spl <= 4 ? decode_avg_apply_kernel<4> : decode_avg_apply_kernel<8>;
-    kern<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, theta_sync);
+    FuseArgs fa;
+    memset(&fa, 0, sizeof(fa));
+    WorkerPtrs wp;
+    memset(&wp, 0, sizeof(wp));
+    if (fuse) {
+        fa.ws = carve(c, R);
+        fa.n_chunks = c->n_chunks;
+        fa.n_tensors = c->n_tensors;
+        fa.kp = c->kp;
+        wp = *fuse_ptrs;
+    }
+#define SL_APPLY(SPLV)                                                                                          \
+    do {                                                                                                        \
+        auto kern = fuse == 0 ? decode_avg_apply_kernel<SPLV, 0>                                                \
+                  : fuse == 1 ? decode_avg_apply_kernel<SPLV, 1> : decode_avg_apply_kernel<SPLV, 2>;            \
+        if (smem > 48 * 1024)                                                                                   \
+            SL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
+        kern<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
+    } while (0)
+    if (spl <= 1) SL_APPLY(1);
+    else if (spl <= 2) SL_APPLY(2);
+    else if (spl <= 4) SL_APPLY(4);
+    else SL_APPLY(8);
+#undef SL_APPLY
     prof_mark(c, 8, st);
     if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
     SL_CUDA(cudaGetLastError());
@@ -1832,9 +1919,10 @@ sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
         for (int r = 0; r < R; ++r)
             if (e[r] != c->pending_e[r]) return SL_ERR_INVALID_ARG;
     }
-    sl_status s = launch_compress(c, R, theta_sync, ptrs, st, defer);
+    const int fuse = c->cfg.ef_enabled ? (defer ? 2 : 1) : 0;  // packing fused into the apply kernel
+    sl_status s = launch_compress(c, R, theta_sync, ptrs, st, defer, fuse != 0);
     if (s != SL_OK) return s;
-    return launch_apply(c, pl, R, theta_sync, st);
+    return launch_apply(c, pl, R, theta_sync, st, fuse, &ptrs);
 }
 
 sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* theta_local_host, float* dev_stage,
