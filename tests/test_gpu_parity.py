@@ -181,6 +181,39 @@ def test_tensor_map_copies_match_oracle_and_per_thread_copies(deferred):
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("R,deferred", [(1, True), (1, False), (40, True), (64, False)])
+def test_worker_count_extremes(R, deferred):
+    """One worker (every unit starts a new chunk) and more than 32 workers (the apply kernel takes them
+    in two batches), on a table that takes the tensor-map copies."""
+    wl = I.Workload("extremes", ALIGNED, R=R, k=64, recipe="normal", seed=300 + R, outer_lr=0.8)
+    c = _case(wl, e_scale=0.5, distinct_local=min(R, 4))
+    c.sl.set_ef_deferred(deferred)
+    for step in range(2):
+        c.fill_local(step)
+        snap = c.snapshot(range(len(ALIGNED)))
+        c.step()
+        c.check(snap)
+
+
+def test_sl_compress_on_an_aligned_table_matches_outer_step():
+    """sl_compress (one worker, tensor-map copies) leaves what sl_outer_step leaves for that worker."""
+    wl = I.Workload("single", ALIGNED, R=2, k=41, recipe="student_t4", seed=321)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    for step in range(2):
+        a.fill_local(step)
+        b.fill_local(step)
+        a.step()
+        for r in range(2):
+            b.sl.compress(b.theta, b.local[r], b.e[r], b.payloads[r])
+        b.sl.aggregate_apply(b.payloads, b.theta)
+        torch.cuda.synchronize()
+        assert b.sl.device_status() == 0
+        assert torch.equal(a.theta, b.theta)
+        for r in range(2):
+            assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+
+
 def test_compress_then_aggregate_equals_outer_step_and_absent_workers():
     import oracle as O
     wl = I.Workload("split", SMALL, R=3, k=64, recipe="normal", seed=51, outer_lr=0.8)
