@@ -1089,7 +1089,7 @@ __device__ __forceinline__ unsigned get2(const unsigned* rec, int code_byte0, in
     return (rec[bit >> 5] >> (bit & 31)) & 3u;
 }
 
-constexpr int kApplyEntries = 8;  // entries per thread and batch
+constexpr int kApplyEntries = 8;  // most entries per thread and batch
 
 // FUSE 0: the entries come from the payload records (sl_aggregate_apply).  FUSE 1 / 2: the whole outer
 // step is running and the records do not exist yet: the entries come from the staging arrays, get
@@ -1101,7 +1101,9 @@ struct FuseArgs {
     int n_tensors, kp;
 };
 
-template <int SPL, int FUSE>  // SPL = slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8
+// SPL = slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8; WPW = workers per warp and batch (1, 2 or
+// 4, SPL * WPW <= 8): a thread holds SPL * WPW entries and a batch is 8 * WPW workers
+template <int SPL, int WPW, int FUSE>
 __global__ void __launch_bounds__(kThreads, 4)
 decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale,
                         PayloadPtrs pl, float* __restrict__ theta_sync, FuseArgs fa, WorkerPtrs ptrs) {
@@ -1133,16 +1135,17 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
     for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
 
     // entry e of a thread: worker warp + 8 (e / SPL), slot lane + 32 (e % SPL)
-    constexpr int WPW = kApplyEntries / SPL;  // workers per warp and batch
-    constexpr int batch = 8 * WPW < 32 ? 8 * WPW : 32;
+    constexpr int kEnt = SPL * WPW;  // entries per thread and batch
+    static_assert(kEnt <= kApplyEntries && WPW <= 4, "entry budget");
+    constexpr int batch = 8 * WPW;
     const int vec_per_rec = stride / 16;
 
     for (int r0 = 0; r0 < n_workers; r0 += batch) {
         const int nb = min(batch, n_workers - r0);
-        unsigned pre_p[kApplyEntries];
-        float pre_v[kApplyEntries];
+        unsigned pre_p[kEnt];
+        float pre_v[kEnt];
 #pragma unroll
-        for (int e = 0; e < kApplyEntries; ++e) {
+        for (int e = 0; e < kEnt; ++e) {
             pre_p[e] = 0u;
             pre_v[e] = 0.f;
         }
@@ -1189,10 +1192,10 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
         }
         __syncthreads();
 
-        unsigned ent_p[kApplyEntries];  // position | worker bit number << 12; 0xFFFFFFFF = no entry
-        float ent_v[kApplyEntries];
+        unsigned ent_p[kEnt];  // position | worker bit number << 12; 0xFFFFFFFF = no entry
+        float ent_v[kEnt];
 #pragma unroll
-        for (int e = 0; e < kApplyEntries; ++e) {
+        for (int e = 0; e < kEnt; ++e) {
             ent_p[e] = 0xFFFFFFFFu;
             ent_v[e] = 0.f;
         }
@@ -1244,7 +1247,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
         // rank of every entry among the workers at its position; round 0
         int my_max = 0;
 #pragma unroll
-        for (int e = 0; e < kApplyEntries; ++e) {
+        for (int e = 0; e < kEnt; ++e) {
             if (ent_p[e] != 0xFFFFFFFFu) {
                 const unsigned p = ent_p[e] & 0xFFFu, rb = ent_p[e] >> 12;
                 const unsigned wm = wmask[p];
@@ -1260,7 +1263,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
         }
         for (int t = 1; __syncthreads_or(my_max > t); ++t) {
 #pragma unroll
-            for (int e = 0; e < kApplyEntries; ++e) {
+            for (int e = 0; e < kEnt; ++e) {
                 if (ent_p[e] != 0xFFFFFFFFu && (int)(ent_p[e] >> 12) == t) {
                     const unsigned p = ent_p[e] & 0xFFFu;
                     acc[p] = __fadd_rn(acc[p], ent_v[e]);
@@ -1593,19 +1596,27 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
         fa.kp = c->kp;
         wp = *fuse_ptrs;
     }
-#define SL_APPLY(SPLV)                                                                                          \
+#define SL_APPLY2(SPLV, WPWV)                                                                                   \
     do {                                                                                                        \
-        auto kern = fuse == 0 ? decode_avg_apply_kernel<SPLV, 0>                                                \
-                  : fuse == 1 ? decode_avg_apply_kernel<SPLV, 1> : decode_avg_apply_kernel<SPLV, 2>;            \
+        auto kern = fuse == 0 ? decode_avg_apply_kernel<SPLV, WPWV, 0>                                          \
+                  : fuse == 1 ? decode_avg_apply_kernel<SPLV, WPWV, 1> : decode_avg_apply_kernel<SPLV, WPWV, 2>; \
         if (smem > 48 * 1024)                                                                                   \
             SL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
         kern<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
     } while (0)
-    if (spl <= 1) SL_APPLY(1);
-    else if (spl <= 2) SL_APPLY(2);
-    else if (spl <= 4) SL_APPLY(4);
-    else SL_APPLY(8);
+    // workers per warp: as few as cover min(R, 32) workers in one batch, within 8 entries per thread
+#define SL_APPLY(SPLV, MAXW)                                             \
+    do {                                                                 \
+        if (R <= 8 || MAXW == 1) SL_APPLY2(SPLV, 1);                      \
+        else if (R <= 16 || MAXW == 2) SL_APPLY2(SPLV, (MAXW >= 2 ? 2 : 1)); \
+        else SL_APPLY2(SPLV, (MAXW >= 4 ? 4 : MAXW));                     \
+    } while (0)
+    if (spl <= 1) SL_APPLY(1, 4);
+    else if (spl <= 2) SL_APPLY(2, 4);
+    else if (spl <= 4) SL_APPLY(4, 2);
+    else SL_APPLY(8, 1);
 #undef SL_APPLY
+#undef SL_APPLY2
     prof_mark(c, 8, st);
     if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
     SL_CUDA(cudaGetLastError());
