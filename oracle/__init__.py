@@ -89,6 +89,11 @@ def lib():
         L.orc_decode_payload.argtypes = [P, P, C.c_int32, P, P, P]
         L.orc_aggregate_apply.argtypes = [P, P, C.c_int32, P, P]
         L.orc_outer_step.argtypes = [P, P, C.c_int32, P, P, P, P]
+        L.orc_ixc_encode_chunk.argtypes = [P, C.c_int32, C.c_int32, P, P]
+        L.orc_ixc_decode_chunk.argtypes = [P, P, C.c_int32, C.c_int32, P]
+        L.orc_ixc_encode_payload.argtypes = [P, P, C.c_int32, P, P]
+        L.orc_ixc_encode_payload.restype = C.c_int64
+        L.orc_ixc_decode_payload.argtypes = [P, P, C.c_int32, P, P]
         _lib = L
     return _lib
 
@@ -280,3 +285,42 @@ def outer_step(cfg: Config, tab: Table, theta: np.ndarray, theta_r: List[np.ndar
     lib().orc_outer_step(C.byref(c), tab.ref(), tab.n, _ptr(_chk(theta, np.float32)),
                          _ptr_array(theta_r), _ptr_array(e), _ptr_array(payloads))
     return payloads
+
+
+# ---------------------------------------------------------------- entropy-coded indices
+
+def ixc_encode_chunk(idx: np.ndarray, L: int) -> tuple:
+    """Golomb gap codes of one chunk's ascending indices: (bytes, number of bits)."""
+    idx = _chk(idx, np.int32)
+    pos = C.c_int64(0)
+    lib().orc_ixc_encode_chunk(_ptr(idx), idx.size, L, None, C.byref(pos))
+    nbits = pos.value
+    out = np.zeros((nbits + 7) // 8 + 1, np.uint8)
+    pos = C.c_int64(0)
+    lib().orc_ixc_encode_chunk(_ptr(idx), idx.size, L, _ptr(out), C.byref(pos))
+    return out, nbits
+
+
+def ixc_decode_chunk(stream: np.ndarray, m_sel: int, L: int) -> tuple:
+    stream = _chk(stream, np.uint8)
+    idx = np.zeros(m_sel, np.int32)
+    pos = C.c_int64(0)
+    lib().orc_ixc_decode_chunk(_ptr(stream), C.byref(pos), m_sel, L, _ptr(idx))
+    return idx, pos.value
+
+
+def ixc_encode_payload(cfg: Config, tab: Table, payload: np.ndarray) -> np.ndarray:
+    payload = _chk(payload, np.uint8)
+    c = cfg.c()
+    n = lib().orc_ixc_encode_payload(C.byref(c), tab.arr, tab.n, _ptr(payload), None)
+    out = np.zeros(n, np.uint8)
+    lib().orc_ixc_encode_payload(C.byref(c), tab.arr, tab.n, _ptr(payload), _ptr(out))
+    return out
+
+
+def ixc_decode_payload(cfg: Config, tab: Table, coded: np.ndarray) -> np.ndarray:
+    coded = _chk(coded, np.uint8)
+    c = cfg.c()
+    out = np.zeros(payload_bytes(cfg, tab), np.uint8)
+    lib().orc_ixc_decode_payload(C.byref(c), tab.arr, tab.n, _ptr(coded), _ptr(out))
+    return out
