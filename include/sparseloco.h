@@ -129,6 +129,39 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
 
+/* Entropy-coded indices for the wire (App. "Compression of indices": 12 bits per index is the naive
+ * cost, log2 C(4096, k) / k the bound, 8.9 / 6.6 / 5.6 bits at k = 32 / 128 / 256 what the paper
+ * reports from a scheme it does not describe).  The coding below is this library's own and reaches
+ * about 8.4 / 6.4 / 5.4 bits on uniformly drawn index sets.  sl_encode_payload() rewrites a 12-bit
+ * payload (as written by sl_compress / sl_outer_step) into the coded form for transmission;
+ * sl_decode_payload() restores the identical 12-bit payload, which sl_aggregate_apply() consumes.
+ *
+ * One chunk of length L with m = min(k, L) ascending indices p_0 < p_1 < ...: gaps g_0 = p_0,
+ * g_i = p_i - p_(i-1) - 1; divisor M = max(1, (693 (L - m) + 500 (m + 1)) / (1000 (m + 1))) in integer
+ * arithmetic; the code of g is g / M one-bits, a zero-bit, then g % M in truncated binary
+ * (b = ceil(log2 M), cut = 2^b - M: values below cut in b - 1 bits, else value + cut in b bits, most
+ * significant bit first; nothing when M = 1).  Bit i of a stream sits in byte i / 8 at bit i % 8.
+ * Coded payload (little-endian), T tensors, G chunks, cb = ceil(2 k / 8):
+ *     [0, 16 T)                 the tensor tables, unchanged
+ *     [16 T, 16 T + cb G)       the chunks' code blocks, copied from the records
+ *     next multiple of 4        ceil(G / 16) x uint32: bit offset in the index stream of the first
+ *                               chunk of every group of 16 chunks
+ *     then                      the index stream, chunk after chunk without padding,
+ *                               zero-filled to a multiple of 16 bytes
+ *   sl_coded_payload_capacity : bytes a coded payload can take at worst (size `coded` with it);
+ *                               TOO_LARGE if the stream could exceed 2^32 bits.
+ *   sl_encode_payload         : payload (12-bit form) -> coded; the coded size in bytes is written to
+ *                               *dev_coded_bytes (DEVICE uint64, 8-byte aligned).  Uses the lent
+ *                               workspace as scratch (NOMEM without one) and must not overlap a
+ *                               compression on another stream.
+ *   sl_decode_payload         : coded -> payload (sl_payload_bytes() bytes, fully overwritten).  A
+ *                               corrupted stream yields a wrong but well-bounded record, never an
+ *                               out-of-range access; run sl_validate_payload on the result. */
+sl_status sl_coded_payload_capacity(const sl_ctx* ctx, size_t* bytes);
+sl_status sl_encode_payload(sl_ctx* ctx, const uint8_t* payload, uint8_t* coded, uint64_t* dev_coded_bytes,
+                            void* cuda_stream);
+sl_status sl_decode_payload(sl_ctx* ctx, const uint8_t* coded, uint8_t* payload, void* cuda_stream);
+
 /* How the compression kernel moves the 64x64 blocks of theta_r and e (no counterpart in the paper).
  * 1: one tensor-map (TMA) block copy per block and direction, completion on shared-memory barriers --
  * the default whenever every full chunk starts on a 64-element boundary of the flat buffers (tensor

@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
 PROFILE_SLOTS = 9
 
@@ -71,6 +71,9 @@ def _load():
     L.sl_profile_name.argtypes = [C.c_int32]
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_coded_payload_capacity.argtypes = [P, C.POINTER(C.c_size_t)]
+    L.sl_encode_payload.argtypes = [P, P, P, P, P]
+    L.sl_decode_payload.argtypes = [P, P, P, P]
     L.sl_set_tile_copies.argtypes = [P, C.c_int32]
     L.sl_device_status.argtypes = [P, P]
     L.sl_static_scratch_bytes.restype = C.c_size_t
@@ -244,6 +247,20 @@ class SparseLoCo:
         _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
                                      _dev_ptr(dev_stage, torch.float32), dev_stage.numel(), ea, pa, hp,
                                      _stream()))
+
+    def coded_payload_capacity(self) -> int:
+        v = C.c_size_t()
+        _check(_L.sl_coded_payload_capacity(self._h, C.byref(v)))
+        return v.value
+
+    def encode_payload(self, payload, coded, coded_bytes: torch.Tensor) -> None:
+        """12-bit payload -> entropy-coded payload; the size lands in `coded_bytes` (device int64[1])."""
+        assert coded_bytes.dtype == torch.int64 and coded_bytes.numel() == 1
+        _check(_L.sl_encode_payload(self._h, _dev_ptr(payload, torch.uint8), _dev_ptr(coded, torch.uint8),
+                                    _dev_ptr(coded_bytes), _stream()))
+
+    def decode_payload(self, coded, payload) -> None:
+        _check(_L.sl_decode_payload(self._h, _dev_ptr(coded, torch.uint8), _dev_ptr(payload, torch.uint8), _stream()))
 
     def set_tile_copies(self, use_tensor_maps: bool) -> None:
         _check(_L.sl_set_tile_copies(self._h, int(use_tensor_maps)))
