@@ -249,6 +249,28 @@ def run_ours(args) -> dict:
         "kernel_ms_per_launch": kernel_ms,
     }
 
+    if rank == 0 and world == 1 and not args.no_dense:
+        # the paper's dense comparator on the same buffers: DiLoCo's outer step (Eq. 1), R reads of
+        # theta_local plus theta and momentum read + written = (4 R + 16) bytes per parameter.
+        # (Timed after the headline loop; it borrows one error buffer as the momentum.)
+        if deferred:
+            sl.ef_flush()
+        mom = e[-1]
+        mom.zero_()
+        for _ in range(2):
+            sl.diloco_step(theta, locals_r, mom, 0.9)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(5):
+            sl.diloco_step(theta, locals_r, mom, 0.9)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dms = d0.elapsed_time(d1) / 5
+        dbytes = (4 * wl.R + 16) * N
+        result["dense_diloco_step"] = {"ms_per_step": dms, "params_per_s": N / (dms * 1e-3),
+                                       "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
+                                       "frac_of_measured_peak": dbytes / (dms * 1e-3) / 1e9 / peak,
+                                       "entry_point": "sl_diloco_step", "beta_outer": 0.9}
     if rank == 0 and world == 1 and not args.no_e2e:
         del local, locals_r
         torch.cuda.empty_cache()
@@ -394,6 +416,7 @@ def main():
                          "default when the table allows) or per-thread 16-byte asynchronous copies")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense DiLoCo comparator line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")

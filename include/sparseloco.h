@@ -129,6 +129,15 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
 
+/* Dense baseline on the same buffers: DiLoCo's outer step with Nesterov outer momentum (Eq. 1),
+ *     Dbar = (1/R) sum_r (theta - theta_r);  m = beta_outer m + Dbar;
+ *     theta = theta - alpha (Dbar + beta_outer m),        alpha = the context's outer_lr.
+ *   theta_sync, momentum : flat fp32, updated in place (only the elements of the tensor table);
+ *   theta_local : HOST array of R DEVICE pointers, read only, may alias.
+ * No compression, no workspace.  Errors: INVALID_ARG (NULL, beta_outer outside [0, 1]), ALIGNMENT, CUDA. */
+sl_status sl_diloco_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local, float* momentum,
+                         float beta_outer, void* cuda_stream);
+
 /* Entropy-coded indices for the wire (App. "Compression of indices": 12 bits per index is the naive
  * cost, log2 C(4096, k) / k the bound, 8.9 / 6.6 / 5.6 bits at k = 32 / 128 / 256 what the paper
  * reports from a scheme it does not describe).  The coding below is this library's own and reaches

@@ -89,6 +89,8 @@ def lib():
         L.orc_decode_payload.argtypes = [P, P, C.c_int32, P, P, P]
         L.orc_aggregate_apply.argtypes = [P, P, C.c_int32, P, P]
         L.orc_outer_step.argtypes = [P, P, C.c_int32, P, P, P, P]
+        L.orc_diloco_step.argtypes = [P, C.c_int32, C.c_int32, C.c_float, C.c_float, P, P, P]
+        L.orc_diloco_lom_step.argtypes = [P, C.c_int32, C.c_int32, C.c_float, C.c_float, P, P, P]
         L.orc_ixc_encode_chunk.argtypes = [P, C.c_int32, C.c_int32, P, P]
         L.orc_ixc_decode_chunk.argtypes = [P, P, C.c_int32, C.c_int32, P]
         L.orc_ixc_encode_payload.argtypes = [P, P, C.c_int32, P, P]
@@ -324,3 +326,22 @@ def ixc_decode_payload(cfg: Config, tab: Table, coded: np.ndarray) -> np.ndarray
     out = np.zeros(payload_bytes(cfg, tab), np.uint8)
     lib().orc_ixc_decode_payload(C.byref(c), tab.arr, tab.n, _ptr(coded), _ptr(out))
     return out
+
+
+# ---------------------------------------------------------------- dense baselines
+
+def diloco_step(tab: Table, theta: np.ndarray, theta_r: List[np.ndarray], m: np.ndarray, beta_outer: float,
+                alpha: float) -> None:
+    """Eq. 1 in place on theta and the global momentum m (fp32 arrays)."""
+    _chk(theta, np.float32); _chk(m, np.float32)
+    arr = _ptr_array([_chk(a, np.float32) for a in theta_r])
+    lib().orc_diloco_step(tab.arr, tab.n, len(theta_r), beta_outer, alpha, _ptr(theta), arr, _ptr(m))
+
+
+def diloco_lom_step(tab: Table, theta: np.ndarray, theta_r: List[np.ndarray], m_r: List[np.ndarray],
+                    beta_outer: float, alpha: float) -> None:
+    """DiLoCo-LOM in place on theta and the per-replica momenta m_r (fp64 arrays)."""
+    _chk(theta, np.float32)
+    arr = _ptr_array([_chk(a, np.float32) for a in theta_r])
+    marr = _ptr_array([_chk(a, np.float64) for a in m_r])
+    lib().orc_diloco_lom_step(tab.arr, tab.n, len(theta_r), beta_outer, alpha, _ptr(theta), arr, marr)

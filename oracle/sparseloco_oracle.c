@@ -688,3 +688,44 @@ void orc_ixc_decode_payload(const orc_config* c, const orc_tensor* ts, int32_t n
     free(idx);
     free(code);
 }
+
+/* ================================================================ dense baselines (Sec. 3.1, 3.2)
+ *
+ * DiLoCo's outer step, Eq. 1:  Dbar = (1/R) sum_r (theta - theta_r);  m = beta m + Dbar;
+ * theta = theta - alpha (Dbar + beta m)   (Nesterov outer momentum, one global m).
+ * DiLoCo-LOM (Sec. 3.2): every replica keeps its own momentum m_r = beta m_r + Delta_r, sends
+ * Delta_r + beta m_r, and theta moves by alpha times their mean.  Proposition 1 states that the two
+ * coincide when the m_r start equal; the tests use that as a pin.  fp64 throughout, results rounded
+ * to fp32 once.  Only the elements of the tensor table are touched.
+ */
+void orc_diloco_step(const orc_tensor* ts, int32_t nt, int32_t R, float beta_outer, float alpha,
+                     float* theta, const float* const* theta_r, float* m) {
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+        for (int64_t i = o; i < o + n; ++i) {
+            double acc = 0.0;
+            for (int32_t r = 0; r < R; ++r) acc += (double)theta[i] - (double)theta_r[r][i];
+            const double dbar = acc / (double)R;
+            const double mm = (double)beta_outer * (double)m[i] + dbar;
+            theta[i] = (float)((double)theta[i] - (double)alpha * (dbar + (double)beta_outer * mm));
+            m[i] = (float)mm;
+        }
+    }
+}
+
+void orc_diloco_lom_step(const orc_tensor* ts, int32_t nt, int32_t R, float beta_outer, float alpha,
+                         float* theta, const float* const* theta_r, double* const* m_r) {
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+        for (int64_t i = o; i < o + n; ++i) {
+            double acc = 0.0;
+            for (int32_t r = 0; r < R; ++r) {
+                const double d = (double)theta[i] - (double)theta_r[r][i];
+                m_r[r][i] = (double)beta_outer * m_r[r][i] + d;
+                acc += d + (double)beta_outer * m_r[r][i];
+            }
+            theta[i] = (float)((double)theta[i] - (double)alpha * acc / (double)R);
+        }
+    }
+}

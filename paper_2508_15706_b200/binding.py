@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
 )
 PROFILE_SLOTS = 9
 
@@ -71,6 +71,7 @@ def _load():
     L.sl_profile_name.argtypes = [C.c_int32]
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
+    L.sl_diloco_step.argtypes = [P, P, P, P, C.c_float, P]
     L.sl_coded_payload_capacity.argtypes = [P, C.POINTER(C.c_size_t)]
     L.sl_encode_payload.argtypes = [P, P, P, P, P]
     L.sl_decode_payload.argtypes = [P, P, P, P]
@@ -247,6 +248,12 @@ class SparseLoCo:
         _check(_L.sl_outer_step_host(self._h, _dev_ptr(theta_sync, torch.float32), tl,
                                      _dev_ptr(dev_stage, torch.float32), dev_stage.numel(), ea, pa, hp,
                                      _stream()))
+
+    def diloco_step(self, theta_sync, theta_local: List[torch.Tensor], momentum, beta_outer: float) -> None:
+        """Dense baseline (Eq. 1): theta_sync and momentum updated in place."""
+        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
+        _check(_L.sl_diloco_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, _dev_ptr(momentum, torch.float32),
+                                 beta_outer, _stream()))
 
     def coded_payload_capacity(self) -> int:
         v = C.c_size_t()

@@ -1551,6 +1551,71 @@ ixc_decode_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
 }  // namespace
 
 // ================================================================================================
+// Dense baseline: DiLoCo's outer step (Eq. 1), for comparison on the same buffers.
+//   Dbar = (1/R) sum_r (theta - theta_r);  m = beta m + Dbar;  theta = theta - alpha (Dbar + beta m)
+// One CTA per chunk of the table (so exactly the table's elements are touched), 16 elements per
+// thread, all R + 2 streams of a thread's vector in flight together.  fp32: differences and their
+// sum in ascending r, one division by R, two fused multiply-adds.
+// ================================================================================================
+namespace {
+
+struct LocalPtrs {
+    const float* p[kMaxR];
+};
+
+__device__ __forceinline__ float diloco_elem(float th, float acc, float inv_r_num, float beta, float alpha, float& m) {
+    const float dbar = __fdiv_rn(acc, inv_r_num);
+    m = __fmaf_rn(beta, m, dbar);
+    return __fmaf_rn(-alpha, __fmaf_rn(beta, m, dbar), th);
+}
+
+__global__ void __launch_bounds__(kThreads)
+diloco_step_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, float beta, float alpha,
+                   float* __restrict__ theta, LocalPtrs loc, float* __restrict__ mom) {
+    const ChunkDesc cd = chunks[blockIdx.x];
+    const int tid = threadIdx.x;
+    const float fr = (float)n_workers;
+    if (cd.len == kChunk) {
+        const int rs = cd.row_stride ? cd.row_stride : kTile;
+        const long long off0 = cd.base + (long long)(tid >> 4) * rs + (4 * tid & 63), step = 16ll * rs;
+#pragma unroll 1
+        for (int i = 0; i < 4; ++i) {
+            const long long off = off0 + i * step;
+            const float4 th = *reinterpret_cast<const float4*>(theta + off);
+            float4 m = *reinterpret_cast<const float4*>(mom + off);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+            for (int r = 0; r < n_workers; ++r) {
+                const float4 l = __ldcs(reinterpret_cast<const float4*>(loc.p[r] + off));
+                acc.x = __fadd_rn(acc.x, __fsub_rn(th.x, l.x));
+                acc.y = __fadd_rn(acc.y, __fsub_rn(th.y, l.y));
+                acc.z = __fadd_rn(acc.z, __fsub_rn(th.z, l.z));
+                acc.w = __fadd_rn(acc.w, __fsub_rn(th.w, l.w));
+            }
+            float4 o;
+            o.x = diloco_elem(th.x, acc.x, fr, beta, alpha, m.x);
+            o.y = diloco_elem(th.y, acc.y, fr, beta, alpha, m.y);
+            o.z = diloco_elem(th.z, acc.z, fr, beta, alpha, m.z);
+            o.w = diloco_elem(th.w, acc.w, fr, beta, alpha, m.w);
+            *reinterpret_cast<float4*>(theta + off) = o;
+            *reinterpret_cast<float4*>(mom + off) = m;
+        }
+    } else {
+        for (int p = tid; p < cd.len; p += kThreads) {
+            const long long off = cd.base + p;
+            const float th = theta[off];
+            float acc = 0.f;
+            for (int r = 0; r < n_workers; ++r) acc = __fadd_rn(acc, __fsub_rn(th, loc.p[r][off]));
+            float m = mom[off];
+            theta[off] = diloco_elem(th, acc, fr, beta, alpha, m);
+            mom[off] = m;
+        }
+    }
+}
+
+}  // namespace
+
+// ================================================================================================
 // Host side
 // ================================================================================================
 
@@ -2253,6 +2318,26 @@ const char* sl_profile_name(int32_t slot) {
     static const char* names[kProfSlots] = {"ef_topk", "chunk_sum", "tensor_mean", "chunk_var", "tensor_sigma",
                                             "chunk_bins", "tensor_lut", "pack_fix", "decode_avg_apply"};
     return slot >= 0 && slot < kProfSlots ? names[slot] : "";
+}
+
+sl_status sl_diloco_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* momentum,
+                         float beta_outer, void* stream) {
+    if (!c || !theta_sync || !theta_local || !momentum) return SL_ERR_INVALID_ARG;
+    if (!(beta_outer >= 0.0f && beta_outer <= 1.0f)) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync) || misaligned(momentum)) return SL_ERR_ALIGNMENT;
+    LocalPtrs lp;
+    memset(&lp, 0, sizeof(lp));
+    for (int r = 0; r < c->cfg.R; ++r) {
+        if (!theta_local[r]) return SL_ERR_INVALID_ARG;
+        if (misaligned(theta_local[r])) return SL_ERR_ALIGNMENT;
+        lp.p[r] = theta_local[r];
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    diloco_step_kernel<<<(unsigned)c->n_chunks, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->d_chunks, c->cfg.R, beta_outer, c->cfg.outer_lr, theta_sync, lp, momentum);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
 }
 
 sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {
