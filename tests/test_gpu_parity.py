@@ -214,6 +214,30 @@ def test_sl_compress_on_an_aligned_table_matches_outer_step():
             assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+def test_fragment_contexts_equal_one_full_step():
+    """Streaming (the paper's fragment-wise variant) needs nothing new: contexts over disjoint subsets
+    of the tensors, with offsets into the same flat buffers, each take the outer step of their
+    fragment; together they leave theta and the error buffers exactly as one step over all tensors."""
+    from paper_2508_15706_b200.binding import SparseLoCo
+    wl = I.Workload("fragments", ALIGNED, R=3, k=64, recipe="normal", seed=410, outer_lr=0.8)
+    full = _case(wl, e_scale=0.5)
+    frag = _case(wl, e_scale=0.5)
+    full.fill_local(0)
+    frag.fill_local(0)
+    full.step()
+    ids = [[0, 1, 2], [3, 4, 5]]
+    for sub in ids:
+        sl = SparseLoCo([full.shapes[j] for j in sub], [full.offs[j] for j in sub], k=64, R=3, beta=wl.beta,
+                        outer_lr=wl.outer_lr)
+        pays = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=frag.dev) for _ in range(3)]
+        sl.outer_step(frag.theta, frag.local, frag.e, pays)
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
+    assert torch.equal(full.theta, frag.theta)
+    for r in range(3):
+        assert torch.equal(full.e[r], frag.e[r])
+
+
 def test_compress_then_aggregate_equals_outer_step_and_absent_workers():
     import oracle as O
     wl = I.Workload("split", SMALL, R=3, k=64, recipe="normal", seed=51, outer_lr=0.8)
