@@ -214,6 +214,27 @@ def test_sl_compress_on_an_aligned_table_matches_outer_step():
             assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+def test_degenerate_tensor_sizes():
+    """One-element and few-element tensors (k far above the chunk length), a single row shorter than a
+    vector, and a table whose only tensor is a short chunk."""
+    tiny = [I.TensorSpec("one", 1, 1, 0), I.TensorSpec("three", 1, 3, 0), I.TensorSpec("col", 7, 1, 1),
+            I.TensorSpec("w", 64, 64, 1), I.TensorSpec("five", 5, 5, 2)]
+    for k in (1, 64, 256):
+        wl = I.Workload("tiny", tiny, R=2, k=k, recipe="normal", seed=900 + k)
+        c = _case(wl, e_scale=0.5)
+        for step in range(2):
+            c.fill_local(step)
+            snap = c.snapshot(range(len(tiny)))
+            c.step()
+            c.check(snap)
+    wl = I.Workload("lonely", [I.TensorSpec("v", 1, 100, 0)], R=1, k=64, recipe="normal", seed=950)
+    c = _case(wl)
+    c.fill_local(0)
+    snap = c.snapshot([0])
+    c.step()
+    c.check(snap)
+
+
 def test_fragment_contexts_equal_one_full_step():
     """Streaming (the paper's fragment-wise variant) needs nothing new: contexts over disjoint subsets
     of the tensors, with offsets into the same flat buffers, each take the outer step of their
