@@ -527,7 +527,7 @@ void orc_outer_step(const orc_config* cfg, const orc_tensor* ts, int32_t nt, flo
  * App. "Compression of indices": 12 bits per index is the naive cost; the bound is
  * log2 C(C, k) / k bits (8.3 / 6.3 / 5.3 at k = 32 / 128 / 256) and the paper reports 8.9 / 6.6 /
  * 5.6 from a custom scheme of which it names only the ingredients.  The scheme below is this
- * build's own; what is pinned is round-trip exactness, the closed-form length, and that the
+ * library's own; what is pinned is round-trip exactness, the closed-form length, and that the
  * rate on uniformly drawn index sets lies between the bound and the paper's achieved numbers.
  *
  * One chunk, length L, m_sel = min(k, L) ascending indices p_0 < p_1 < ...:

@@ -1926,7 +1926,7 @@ const char* sl_strerror(sl_status s) {
         case SL_OK: return "ok";
         case SL_ERR_INVALID_ARG: return "invalid argument";
         case SL_ERR_ALIGNMENT: return "pointer or offset not 16-byte aligned";
-        case SL_ERR_UNSUPPORTED: return "configuration not supported by this build";
+        case SL_ERR_UNSUPPORTED: return "configuration not supported by this library";
         case SL_ERR_BAD_PAYLOAD: return "malformed payload";
         case SL_ERR_CUDA: return "CUDA error";
         case SL_ERR_NOMEM: return "workspace missing or too small";
