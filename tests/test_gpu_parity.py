@@ -214,6 +214,28 @@ def test_sl_compress_on_an_aligned_table_matches_outer_step():
             assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+def test_tensor_map_table_survives_many_buffers():
+    """Every new buffer pointer gets tensor maps on first use; the table of maps is finite, so a caller
+    that keeps passing fresh buffers makes it start over.  Results must not care."""
+    wl = I.Workload("slots", ALIGNED, R=3, k=64, recipe="normal", seed=430)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    b.sl.set_tile_copies(False)
+    keep = []
+    for step in range(60):   # 3 fresh theta_local buffers per step: 180 pointers > the table's capacity
+        a.fill_local(step % 3)
+        fresh = [x.clone() for x in a.local]
+        keep.append(fresh)   # keep them alive so that the allocator cannot hand the same address out again
+        a.sl.outer_step(a.theta, fresh, a.e, a.payloads)
+        b.fill_local(step % 3)
+        b.step()
+    torch.cuda.synchronize()
+    assert a.sl.device_status() == 0
+    assert torch.equal(a.theta, b.theta)
+    for r in range(3):
+        assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+
+
 def test_degenerate_tensor_sizes():
     """One-element and few-element tensors (k far above the chunk length), a single row shorter than a
     vector, and a table whose only tensor is a short chunk."""
