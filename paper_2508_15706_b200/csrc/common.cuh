@@ -1,0 +1,72 @@
+// Constants, the chunk table and workspace layouts, small helpers shared by all kernels.
+// Part of libsparseloco (one translation unit: included by sparseloco.cu).
+#pragma once
+
+namespace {
+
+constexpr int kChunk = 4096;
+constexpr int kTile = 64;
+constexpr int kThreads = 256;          // threads per CTA of the chunk kernels
+constexpr int kPerThread = kChunk / kThreads;  // 16 elements = 4 x float4
+constexpr int kMaxR = 64;
+constexpr int kMaxK = 256;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kProfSlots = 9;     // kernels of one outer step
+constexpr int kProfMaxSeq = 256;  // recorded sequences kept between two reads
+
+thread_local char g_cuda_err[256] = "";
+
+// One chunk of one tensor: where its elements live in the flat buffers.
+struct ChunkDesc {
+    long long base;    // element offset of in-chunk index 0
+    int row_stride;    // elements between block rows (2-D blocks), 0 for flat runs
+    int len;           // elements in the chunk (4096, or the short tail of a flat tensor)
+    int tensor;        // owning tensor
+    int chunk_in_tensor;
+    long long rec_off; // byte offset of this chunk's record inside a payload
+};
+static_assert(sizeof(ChunkDesc) == 32, "ChunkDesc layout");
+
+struct TensorInfo {
+    long long first_chunk;
+    long long n_chunks;
+    long long n_slots;  // sum over chunks of min(k, len)
+};
+
+struct TStat {  // per (worker, tensor)
+    float mu, sigma, t3;
+    float lut[4];
+    float pad;
+};
+static_assert(sizeof(TStat) == 32, "TStat layout");
+
+struct WorkerPtrs {
+    const float* theta_local[kMaxR];
+    float* e[kMaxR];
+    uint8_t* payload[kMaxR];
+};
+
+struct PayloadPtrs {
+    const uint8_t* p[kMaxR];
+};
+
+struct Workspace {  // device arrays, dimensioned [workers][chunks]...
+    float* val;          // [W][G][kp]
+    uint16_t* idx;       // [W][G][kp]
+    double* psum;        // [W][G]
+    double* pbin;        // [W][G][4]
+    unsigned* pcnt;      // [W][G][4]
+    TStat* tstat;        // [W][T]
+};
+
+__host__ __device__ constexpr int record_index_bytes(int k) { return (12 * k + 7) / 8; }
+__host__ __device__ constexpr int record_stride(int k) {
+    return (record_index_bytes(k) + (2 * k + 7) / 8 + 15) / 16 * 16;
+}
+
+// Element offset (relative to ChunkDesc::base) of in-chunk index p.
+__device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {
+    return row_stride ? (long long)(p >> 6) * row_stride + (p & 63) : (long long)p;
+}
+
+}  // namespace
