@@ -112,7 +112,7 @@ __device__ __forceinline__ ChunkGeo load_geo(const ChunkDesc* d) {
     return g;
 }
 
-template <bool EF, bool PENDING, bool TMA>
+template <bool EF, bool PENDING, bool TMA, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 3)
 ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma) {
@@ -327,7 +327,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         unsigned* bitmap = sm.sel.bitmap[s];
         Picked pk;
         pk.p0 = pk.v0 = pk.p1 = pk.v1 = 0u;
-        bool exact = select_topk(ub, reinterpret_cast<const unsigned*>(tile), cd.len, keff, sm.sel, pk);
+        bool exact = select_topk<WIDE>(ub, reinterpret_cast<const unsigned*>(tile), cd.len, keff, sm.sel, pk);
         if (tid < 128) sm.sel.bitmap[s ^ 1][tid] = 0;  // the other map: its readers passed the barrier above
 
         // refill for unit n + 2.  cp.async variant: the whole stage is consumed (nothing below reads
@@ -374,7 +374,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                 if (have2) tma_load_e(s, d2, r2);
             }
             e_started = true;
-            exact = select_rank(keff, sm.sel, bitmap, pk);
+            exact = select_rank<WIDE>(keff, sm.sel, bitmap, pk);
         }
         if (exact) {
             unsigned tmp[kPerThread];

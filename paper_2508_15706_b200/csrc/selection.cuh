@@ -34,7 +34,8 @@ __device__ __forceinline__ void cp_async_wait() {
 //    rounded down to a multiple of 32.  At least keff values have key >= T.  (In a short chunk
 //    only the ceil(len/512) warps that own elements take part, ceil(keff/that) rounds each.)
 // 2. the 8 warp values cluster around the keff-th largest key, so three splitters between their
-//    minimum and maximum cut the candidates (key >= T, about 2 keff of them) into four classes.
+//    minimum and maximum cut the candidates (key >= T, about 2 keff of them) into four classes
+//    (for k > 64: eight classes, seven equal steps between the extremes and one class above).
 //    Every candidate is appended to its class list; the class counts say which class holds the
 //    cut: classes above it are selected whole, and only that class (some tens of entries) is
 //    ranked, by all-pairs counting on (key, index).
@@ -45,13 +46,22 @@ __device__ __forceinline__ void cp_async_wait() {
 // ------------------------------------------------------------------------------------------------
 constexpr int kFetchWarp = 7;    // fetches the pending lists: the warp with the least selection work
 constexpr int kClassCap = 224;  // entries per class list (<= threads: one thread per entry suffices)
+// For k > 64 the three splitters leave the class around the cut too large (130 entries at k = 123,
+// ranked by all pairs), so larger k use eight classes: seven equal steps from the smallest to the
+// largest warp value and a top class above it.  The same list storage, cut differently: seven
+// lists of kWideLowCap entries and the top class (mostly certain winners, the largest) behind them.
+constexpr int kWideClasses = 8;
+constexpr int kWideLowCap = 88;
+constexpr int kWideTopCap = 256;  // one thread per entry must suffice; 7 * 88 + 256 <= 4 * kClassCap
+static_assert((kWideClasses - 1) * kWideLowCap + kWideTopCap <= 4 * kClassCap, "list storage");
+inline bool wide_classes(int k) { return k > 64; }  // host: which instantiation to launch
 
 struct SelectSmem {
     unsigned lkey[4][kClassCap];  // candidates per class: key
     uint16_t lpos[4][kClassCap];  //                        in-chunk index | sign << 12
     unsigned bitmap[2][128];   // selected positions, double-buffered by unit parity
     unsigned warp_t[8];
-    unsigned cnt[4];
+    __align__(16) unsigned cnt[8];
     unsigned warp_cnt[2][8];
     unsigned n_exact;          // entries the exact search appended
 };
@@ -124,6 +134,7 @@ struct Picked {
 // the thread's own slots are read).  Contains one CTA barrier: every thread of the CTA must call
 // it, and must synchronise again before select_rank().  Returns true when the threshold is 0, in
 // which case nothing was listed and the exact search has to run instead.
+template <bool WIDE>
 __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], const unsigned* __restrict__ tile,
                                             int len, int keff, SelectSmem& sm, Picked& out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -147,10 +158,11 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
             cur = cur == tw ? 0u : cur;  // retire the holder (tagged values are distinct, or all 0)
         }
         if (lane == 0) sm.warp_t[warp] = warp < n_warps ? (tw & ~31u) : 0xFFFFFFFFu;
-        if (tid < 4) sm.cnt[tid] = 0;
+        if (tid < 8) sm.cnt[tid] = 0;
     }
     __syncthreads();
     unsigned T, s1, s2, s3;
+    float wide_scale;  // eight classes: class = min(7, (key - T) * wide_scale), non-decreasing in the key
     {
         const uint4 a = *reinterpret_cast<const uint4*>(&sm.warp_t[0]);
         const uint4 b = *reinterpret_cast<const uint4*>(&sm.warp_t[4]);
@@ -170,7 +182,9 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
         s2 = max(mean, lo);
         s1 = (lo >> 1) + (s2 >> 1);
         s3 = (s2 >> 1) + (hi >> 1);
+        wide_scale = hi > lo ? (float)(kWideClasses - 1) / (float)(hi - lo) : 0.0f;
     }
+    constexpr bool wide = WIDE;
 
     bool exact = T == 0;  // uniform over the CTA
     if (!exact) {
@@ -186,11 +200,20 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
             const int p = owned_index(tid, b);
             const unsigned bits = tile[p];
             const unsigned kq = bits & 0x7FFFFFFFu;
-            const unsigned cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
+            unsigned cls, off, cap;
+            if (wide) {
+                cls = min((unsigned)(kWideClasses - 1), (unsigned)((float)(kq - T) * wide_scale));
+                off = cls * kWideLowCap;
+                cap = cls == kWideClasses - 1 ? kWideTopCap : kWideLowCap;
+            } else {
+                cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
+                off = cls * kClassCap;
+                cap = kClassCap;
+            }
             const unsigned pos = atomicAdd(&sm.cnt[cls], 1u);
-            if (pos < kClassCap) {
-                sm.lkey[cls][pos] = kq;
-                sm.lpos[cls][pos] = (uint16_t)((unsigned)p | ((bits >> 31) << 12));
+            if (pos < cap) {
+                (&sm.lkey[0][0])[off + pos] = kq;
+                (&sm.lpos[0][0])[off + pos] = (uint16_t)((unsigned)p | ((bits >> 31) << 12));
             }
         }
     }
@@ -199,40 +222,81 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
 
 // Second half of the selection, after the barrier that completes the class lists.  Returns true
 // when a list overflowed: nothing was marked and the exact search has to run instead.
+template <bool WIDE>
 __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* bitmap, Picked& out) {
     const int tid = threadIdx.x;
-    const uint4 cn = *reinterpret_cast<const uint4*>(&sm.cnt[0]);
-    // the class holding the cut: the highest class c with count(classes >= c) >= keff
-    unsigned above = 0, cstar = 3, L = cn.w;
-    if (cn.w < (unsigned)keff) {
-        above = cn.w; cstar = 2; L = cn.z;
-        if (above + cn.z < (unsigned)keff) {
-            above += cn.z; cstar = 1; L = cn.y;
-            if (above + cn.y < (unsigned)keff) { above += cn.y; cstar = 0; L = cn.x; }
-        }
-    }
-    if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)kClassCap) return true;  // overflow: exact search
-    const unsigned want = (unsigned)keff - above;  // 1 <= want <= L
-    // classes above the cut are selected whole: `above` (< keff <= 256) entries, one per thread
-    if (tid < (int)above) {
-        unsigned c = 3, j = tid;
-        if (j >= cn.w) {
-            j -= cn.w;
-            c = 2;
-            if (j >= cn.z) {
-                j -= cn.z;
-                c = 1;
+    unsigned above = 0, cstar, L, list_off;
+    const unsigned* __restrict__ lkf = &sm.lkey[0][0];
+    const uint16_t* __restrict__ lpf = &sm.lpos[0][0];
+    if (!WIDE) {
+        const uint4 cn = *reinterpret_cast<const uint4*>(&sm.cnt[0]);
+        // the class holding the cut: the highest class c with count(classes >= c) >= keff
+        cstar = 3;
+        L = cn.w;
+        if (cn.w < (unsigned)keff) {
+            above = cn.w; cstar = 2; L = cn.z;
+            if (above + cn.z < (unsigned)keff) {
+                above += cn.z; cstar = 1; L = cn.y;
+                if (above + cn.y < (unsigned)keff) { above += cn.y; cstar = 0; L = cn.x; }
             }
         }
-        out.p1 = sm.lpos[c][j];
-        out.v1 = sm.lkey[c][j] | ((out.p1 >> 12) << 31);
-        out.p1 &= 0xFFFu;
-        out.mask |= 2u;
-        set_bit(bitmap, out.p1);
+        if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)kClassCap) return true;  // overflow: exact search
+        list_off = cstar * kClassCap;
+        // classes above the cut are selected whole: `above` (< keff <= 256) entries, one per thread
+        if (tid < (int)above) {
+            unsigned c = 3, j = tid;
+            if (j >= cn.w) {
+                j -= cn.w;
+                c = 2;
+                if (j >= cn.z) {
+                    j -= cn.z;
+                    c = 1;
+                }
+            }
+            out.p1 = lpf[c * kClassCap + j];
+            out.v1 = lkf[c * kClassCap + j] | ((out.p1 >> 12) << 31);
+            out.p1 &= 0xFFFu;
+            out.mask |= 2u;
+            set_bit(bitmap, out.p1);
+        }
+    } else {
+        const uint4 c_lo = *reinterpret_cast<const uint4*>(&sm.cnt[0]), c_hi = *reinterpret_cast<const uint4*>(&sm.cnt[4]);
+        const unsigned cn[kWideClasses] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+        bool found = false, overflow = false;
+        cstar = 0;
+        L = 0;
+#pragma unroll
+        for (int c = kWideClasses - 1; c >= 0; --c) {
+            overflow |= cn[c] > (unsigned)(c == kWideClasses - 1 ? kWideTopCap : kWideLowCap);
+            if (!found) {
+                if (above + cn[c] >= (unsigned)keff) {
+                    found = true;
+                    cstar = (unsigned)c;
+                    L = cn[c];
+                } else {
+                    above += cn[c];
+                }
+            }
+        }
+        if (overflow || !found) return true;
+        list_off = cstar * kWideLowCap;
+        if (tid < (int)above) {
+            unsigned c = kWideClasses - 1, j = tid;
+            while (j >= sm.cnt[c]) {  // ends above the cut class because tid < above
+                j -= sm.cnt[c];
+                --c;
+            }
+            out.p1 = lpf[c * kWideLowCap + j];
+            out.v1 = lkf[c * kWideLowCap + j] | ((out.p1 >> 12) << 31);
+            out.p1 &= 0xFFFu;
+            out.mask |= 2u;
+            set_bit(bitmap, out.p1);
+        }
     }
+    const unsigned want = (unsigned)keff - above;  // 1 <= want <= L
     // the cut class: entry i = tid >> sh is ranked by 2^sh adjacent lanes, each over one segment
-    const unsigned* __restrict__ lk = sm.lkey[cstar];
-    const uint16_t* __restrict__ lp = sm.lpos[cstar];
+    const unsigned* __restrict__ lk = lkf + list_off;
+    const uint16_t* __restrict__ lp = lpf + list_off;
     unsigned sh = 0;
     while (sh < 3 && (L << (sh + 1)) <= 32u) ++sh;
     const unsigned i = tid >> sh, seg = tid & ((1u << sh) - 1u);

@@ -236,9 +236,14 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     prof_mark(c, -1, st);
     const unsigned ef_grid = (unsigned)(G < c->ef_ctas ? G : c->ef_ctas);  // persistent CTAs
     const size_t smem = sizeof(PipeSmem);
-#define SL_LAUNCH_EF(EFV, PENDV, TMAV)                                                                          \
-    ef_topk_kernel<EFV, PENDV, TMAV><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta, \
-                                                                      theta_sync, ptrs, ws, ta)
+#define SL_LAUNCH_EF1(EFV, PENDV, TMAV, WIDEV)                                                                        \
+    ef_topk_kernel<EFV, PENDV, TMAV, WIDEV><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta, \
+                                                                             theta_sync, ptrs, ws, ta)
+#define SL_LAUNCH_EF(EFV, PENDV, TMAV)              \
+    do {                                            \
+        if (wide_classes(k)) SL_LAUNCH_EF1(EFV, PENDV, TMAV, true); \
+        else SL_LAUNCH_EF1(EFV, PENDV, TMAV, false); \
+    } while (0)
     if (use_tma) {
         if (!ef) SL_LAUNCH_EF(false, false, true);
         else if (consume) SL_LAUNCH_EF(true, true, true);
@@ -249,6 +254,7 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
         else SL_LAUNCH_EF(true, false, false);
     }
 #undef SL_LAUNCH_EF
+#undef SL_LAUNCH_EF1
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
@@ -484,15 +490,21 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
 #define SL_SMEM_ATTR(...)                                                                                      \
     if (e == cudaSuccess)                                                                                      \
         e = cudaFuncSetAttribute(ef_topk_kernel<__VA_ARGS__>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)
-    SL_SMEM_ATTR(true, false, false);
-    SL_SMEM_ATTR(false, false, false);
-    SL_SMEM_ATTR(true, true, false);
-    SL_SMEM_ATTR(true, false, true);
-    SL_SMEM_ATTR(false, false, true);
-    SL_SMEM_ATTR(true, true, true);
+    SL_SMEM_ATTR(true, false, false, false);
+    SL_SMEM_ATTR(false, false, false, false);
+    SL_SMEM_ATTR(true, true, false, false);
+    SL_SMEM_ATTR(true, false, true, false);
+    SL_SMEM_ATTR(false, false, true, false);
+    SL_SMEM_ATTR(true, true, true, false);
+    SL_SMEM_ATTR(true, false, false, true);
+    SL_SMEM_ATTR(false, false, false, true);
+    SL_SMEM_ATTR(true, true, false, true);
+    SL_SMEM_ATTR(true, false, true, true);
+    SL_SMEM_ATTR(false, false, true, true);
+    SL_SMEM_ATTR(true, true, true, true);
 #undef SL_SMEM_ATTR
     if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true>, kThreads,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true, true>, kThreads,
                                                           sizeof(PipeSmem));
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int));
@@ -985,9 +997,11 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
         SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
         int n_sms = 0, per_sm = 0;
         SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)sizeof(PipeSmem)));
-        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false, false>, kThreads,
+        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(PipeSmem)));
+        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false, false, true>, kThreads,
                                                               sizeof(PipeSmem)));
         su.scratch = ptr;
         su.ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
@@ -1016,8 +1030,12 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     const unsigned ef_grid = (unsigned)(G < su.ef_ctas ? G : su.ef_ctas);
     TmaArgs no_tma;
     memset(&no_tma, 0, sizeof(no_tma));
-    ef_topk_kernel<true, false, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
-                                                                                   theta_sync, ptrs, ws, no_tma);
+    if (wide_classes(k))
+        ef_topk_kernel<true, false, false, true><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
+                                                                                          theta_sync, ptrs, ws, no_tma);
+    else
+        ef_topk_kernel<true, false, false, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
+                                                                                           theta_sync, ptrs, ws, no_tma);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
     tensor_reduce_kernel<0><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);
