@@ -153,9 +153,17 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
         // more than 32 rounds cannot be served by 32 lanes: tw ends as 0 and the exact search takes over
         const int rounds = n_warps == 8 ? (keff + 7) >> 3 : min(33, (keff + n_warps - 1) / n_warps);
         unsigned cur = (m & ~31u) | (unsigned)lane, tw = 0;
-        for (int i = 0; i < rounds; ++i) {
-            tw = __reduce_max_sync(kFull, cur);
-            cur = cur == tw ? 0u : cur;  // retire the holder (tagged values are distinct, or all 0)
+        if (rounds == 8) {  // k = 57..64 on full chunks, the common case: unrolled
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                tw = __reduce_max_sync(kFull, cur);
+                cur = cur == tw ? 0u : cur;
+            }
+        } else {
+            for (int i = 0; i < rounds; ++i) {
+                tw = __reduce_max_sync(kFull, cur);
+                cur = cur == tw ? 0u : cur;  // retire the holder (tagged values are distinct, or all 0)
+            }
         }
         if (lane == 0) sm.warp_t[warp] = warp < n_warps ? (tw & ~31u) : 0xFFFFFFFFu;
         if (tid < 8) sm.cnt[tid] = 0;
