@@ -236,6 +236,29 @@ def test_tensor_map_table_survives_many_buffers():
         assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+@pytest.mark.parametrize("buffers", [1, 2])
+def test_outer_step_from_host_buffers_equals_resident_step(buffers):
+    """sl_outer_step_host (workers' parameters in pinned host memory, staged through one or two device
+    buffers, theta copied back) leaves the same bits as sl_outer_step on resident copies."""
+    wl = I.Workload("host", ALIGNED, R=3, k=64, recipe="normal", seed=440, outer_lr=0.9)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    flat = a.theta.numel()
+    flat4 = (flat + 3) // 4 * 4
+    stage = torch.empty(buffers * flat4, dtype=torch.float32, device=a.dev)
+    theta_host = torch.empty(flat, dtype=torch.float32, pin_memory=True)
+    for step in range(2):
+        a.fill_local(step)
+        b.fill_local(step)
+        hosts = [x.cpu().pin_memory() for x in b.local]
+        a.step()
+        b.sl.outer_step_host(b.theta, hosts, stage, b.e, b.payloads, theta_host)
+        assert b.sl.device_status() == 0
+        assert torch.equal(a.theta, b.theta) and torch.equal(theta_host, b.theta.cpu())
+        for r in range(3):
+            assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+
+
 def test_degenerate_tensor_sizes():
     """One-element and few-element tensors (k far above the chunk length), a single row shorter than a
     vector, and a table whose only tensor is a short chunk."""
