@@ -259,6 +259,32 @@ def test_outer_step_from_host_buffers_equals_resident_step(buffers):
             assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+def test_side_stream_gives_the_same_result():
+    """All work (kernels, tensor-map uploads, memsets) is ordered on the caller's stream: steps issued
+    on a side stream without host synchronisation in between match steps on the default stream."""
+    wl = I.Workload("stream", ALIGNED, R=3, k=64, recipe="normal", seed=450)
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    for c in (a, b):
+        c.sl.set_ef_deferred(True)
+        c.fill_local(0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    for step in range(4):
+        a.sl.outer_step(a.theta, a.local, a.e, a.payloads)
+    with torch.cuda.stream(side):
+        for step in range(4):
+            b.sl.outer_step(b.theta, b.local, b.e, b.payloads)
+        b.sl.ef_flush()
+    a.sl.ef_flush()
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert a.sl.device_status() == 0 and b.sl.device_status() == 0
+    assert torch.equal(a.theta, b.theta)
+    for r in range(3):
+        assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+
+
 def test_degenerate_tensor_sizes():
     """One-element and few-element tensors (k far above the chunk length), a single row shorter than a
     vector, and a table whose only tensor is a short chunk."""
