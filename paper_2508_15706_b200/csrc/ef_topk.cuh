@@ -21,14 +21,25 @@ namespace {
 // the next units ride along three units ahead; before u is formed every warp substitutes the
 // entries that fall into its 512 indices (the lists are sorted, so they form one run).
 // ------------------------------------------------------------------------------------------------
-struct PipeSmem {
-    float theta_l[2][kChunk];
+// Shared memory of one CTA.  The cp.async variant keeps two theta_r stages (every thread refills its
+// own slots two units ahead); the TMA variant needs one (it is free again at the unit's first
+// barrier and refilled for the next unit from there).  With the four-class selection (k <= 64) the
+// TMA variant also takes smaller candidate lists and pending-list slots: 54 KB in all, four CTAs
+// per SM instead of three.
+template <bool TMA, bool WIDE>
+struct PipeSmemT {
+    static constexpr bool kCompact = TMA && !WIDE;
+    static constexpr int kLBuf = TMA ? 1 : 2;
+    static constexpr int kPend = kCompact ? 64 : kMaxK;  // slots of a pending list (k rounded up to 8)
+    static constexpr int kCtasPerSm = kCompact ? 4 : 3;
+    float theta_l[kLBuf][kChunk];
     float e[2][kChunk];  // e on arrival, u after the update
-    SelectSmem sel;
-    __align__(16) float pend_val[3][kMaxK];
-    __align__(16) uint16_t pend_idx[3][kMaxK];
-    unsigned long long full_bar[2];  // TMA variant: the stage's tiles have landed
-    int abort;                       // TMA variant: a bounded wait ran out
+    SelectSmemT<kCompact ? kSmallClassCap : kClassCap> sel;
+    __align__(16) float pend_val[3][kPend];
+    __align__(16) uint16_t pend_idx[3][kPend];
+    unsigned long long l_bar;     // TMA variant: the theta_r block has landed
+    unsigned long long e_bar[2];  // TMA variant: the e block of the stage has landed
+    int abort;                    // TMA variant: a bounded wait ran out
 };
 
 // ---- TMA variant: tile copies through tensor maps, completion on shared-memory barriers ----------
@@ -113,11 +124,12 @@ __device__ __forceinline__ ChunkGeo load_geo(const ChunkDesc* d) {
 }
 
 template <bool EF, bool PENDING, bool TMA, bool WIDE>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, (PipeSmemT<TMA, WIDE>::kCtasPerSm))
 ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma) {
     extern __shared__ __align__(1024) unsigned char dyn_smem[];
-    PipeSmem& sm = *reinterpret_cast<PipeSmem*>(dyn_smem);
+    using Smem = PipeSmemT<TMA, WIDE>;
+    Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // 32-bit counters: chunks x workers < 2^31 is checked on the host
     const int grid = (int)gridDim.x, first = (int)blockIdx.x;
@@ -129,8 +141,9 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         sm.sel.bitmap[1][tid] = 0;
     }
     if (TMA && tid == kTmaThread) {
-        mbar_init(&sm.full_bar[0], 1);
-        mbar_init(&sm.full_bar[1], 1);
+        mbar_init(&sm.l_bar, 1);
+        mbar_init(&sm.e_bar[0], 1);
+        mbar_init(&sm.e_bar[1], 1);
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -166,20 +179,24 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         }
         return d;
     };
-    // arms the stage barrier for one unit and starts its theta_r block (a short chunk moves nothing)
-    auto tma_begin_unit = [&](int s, const ChunkGeo& d, int r) {
-        unsigned long long* bar = &sm.full_bar[s];
+    // theta_r block of a unit into the single buffer (a short chunk moves nothing: the phase just ends)
+    auto tma_load_l = [&](const ChunkGeo& d, int r) {
         if (d.len != kChunk) {
-            mbar_arrive(bar);
+            mbar_arrive(&sm.l_bar);
             return;
         }
-        mbar_arrive_expect_tx(bar, (EF ? 2u : 1u) * kChunk * (unsigned)sizeof(float));
-        tma_load_block(sm.theta_l[s], tma.maps + tma.slot_l[r] * tma.n_classes + d.cls, d.x1, d.x2, bar);
+        mbar_arrive_expect_tx(&sm.l_bar, kChunk * (unsigned)sizeof(float));
+        tma_load_block(sm.theta_l[0], tma.maps + tma.slot_l[r] * tma.n_classes + d.cls, d.x1, d.x2, &sm.l_bar);
     };
-    // the e block of a unit begun earlier
+    // e block of a unit into stage s
     auto tma_load_e = [&](int s, const ChunkGeo& d, int r) {
-        if (!EF || d.len != kChunk) return;
-        tma_load_block(sm.e[s], tma.maps + tma.slot_e[r] * tma.n_classes + d.cls, d.x1, d.x2, &sm.full_bar[s]);
+        if (!EF) return;
+        if (d.len != kChunk) {
+            mbar_arrive(&sm.e_bar[s]);
+            return;
+        }
+        mbar_arrive_expect_tx(&sm.e_bar[s], kChunk * (unsigned)sizeof(float));
+        tma_load_block(sm.e[s], tma.maps + tma.slot_e[r] * tma.n_classes + d.cls, d.x1, d.x2, &sm.e_bar[s]);
     };
     // the fetch warp: the pending list of unit (chunk g, worker r) into ring slot `ring`
     auto issue_pending = [&](int ring, int g, int r) {
@@ -225,12 +242,9 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
     __syncthreads();
     if (TMA) {
         if (tid == kTmaThread) {
-            tma_begin_unit(0, cd, 0);
+            tma_load_l(cd, 0);
             tma_load_e(0, cd, 0);
-            if (n_units > 1) {
-                tma_begin_unit(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
-                tma_load_e(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
-            }
+            if (n_units > 1) tma_load_e(1, n_workers > 1 ? cd : cd1, n_workers > 1 ? 1 : 0);
         }
     } else {
         issue_unit(0, cd, 0);
@@ -256,7 +270,10 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
         float* tile = sm.e[s];
 
         cp_async_wait<1>();  // this unit's copies have landed (only the next unit's may be in flight)
-        if (TMA && !mbar_wait(&sm.full_bar[s], (unsigned)((n >> 1) & 1))) sm.abort = 1;
+        if (TMA) {
+            if (!mbar_wait(&sm.l_bar, (unsigned)(n & 1))) sm.abort = 1;
+            if (EF && !mbar_wait(&sm.e_bar[s], (unsigned)((n >> 1) & 1))) sm.abort = 1;
+        }
 
         if (PENDING && EF) {  // substitute the corrected values of the previous step
             const int ring = n % 3;
@@ -282,7 +299,7 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             for (int i = 0; i < 4; ++i) {
                 const int v = slot0 + 128 * i;
                 const float4 a = ts[i];
-                const float4 l = *reinterpret_cast<const float4*>(&sm.theta_l[s][v]);
+                const float4 l = *reinterpret_cast<const float4*>(&sm.theta_l[TMA ? 0 : s][v]);
                 float4 u;
                 u.x = __fsub_rn(a.x, l.x);
                 u.y = __fsub_rn(a.y, l.y);
@@ -354,7 +371,11 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
                     tma_store_block(tma.maps + tma.slot_e[r] * tma.n_classes + cd.cls, cd.x1, cd.x2, tile);
                     bulk_commit();
                 }
-                if (have2) tma_begin_unit(s, d2, r2);  // the theta_r stage was last read before that barrier
+                if (n + 1 < n_units) {  // the theta_r buffer was last read before that barrier: next unit's block
+                    int c1n, r1n;
+                    ahead(c, r, 1, c1n, r1n);
+                    tma_load_l(c1n == c ? cd : cd1, r1n);
+                }
             }
         } else if (have2) {
             issue_unit(s, d2, r2);
@@ -418,7 +439,9 @@ ef_topk_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_w
             // A wait ran out.  Report it, then give the copies still in flight a bounded time to
             // land before the shared memory they target is released.
             if (tid == 0) atomicExch(tma.status, (int)SL_ERR_TIMEOUT);
-            for (int u = n; u < n + 2 && u < n_units; ++u) mbar_wait(&sm.full_bar[u & 1], (unsigned)((u >> 1) & 1));
+            mbar_wait(&sm.l_bar, (unsigned)(n & 1));
+            if (EF)
+                for (int u = n; u < n + 2 && u < n_units; ++u) mbar_wait(&sm.e_bar[u & 1], (unsigned)((u >> 1) & 1));
         }
         if (tid == kTmaThread) bulk_wait_all();
     }

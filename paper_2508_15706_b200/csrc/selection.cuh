@@ -46,6 +46,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // ------------------------------------------------------------------------------------------------
 constexpr int kFetchWarp = 7;    // fetches the pending lists: the warp with the least selection work
 constexpr int kClassCap = 224;  // entries per class list (<= threads: one thread per entry suffices)
+constexpr int kSmallClassCap = 112;  // ... of the compact variant for k <= 64 (about 110 candidates in all)
 // For k > 64 the three splitters leave the class around the cut too large (130 entries at k = 123,
 // ranked by all pairs), so larger k use eight classes: seven equal steps from the smallest to the
 // largest warp value and a top class above it.  The same list storage, cut differently: seven
@@ -56,9 +57,11 @@ constexpr int kWideTopCap = 256;  // one thread per entry must suffice; 7 * 88 +
 static_assert((kWideClasses - 1) * kWideLowCap + kWideTopCap <= 4 * kClassCap, "list storage");
 inline bool wide_classes(int k) { return k > 64; }  // host: which instantiation to launch
 
-struct SelectSmem {
-    unsigned lkey[4][kClassCap];  // candidates per class: key
-    uint16_t lpos[4][kClassCap];  //                        in-chunk index | sign << 12
+template <int CAP>
+struct SelectSmemT {
+    static constexpr int kCap = CAP;  // entries per class list in the four-class scheme
+    unsigned lkey[4][CAP];  // candidates per class: key
+    uint16_t lpos[4][CAP];  //                        in-chunk index | sign << 12
     unsigned bitmap[2][128];   // selected positions, double-buffered by unit parity
     unsigned warp_t[8];
     __align__(16) unsigned cnt[8];
@@ -80,8 +83,9 @@ __device__ __forceinline__ void set_bit(unsigned* bitmap, unsigned p) { atomicOr
 // elements at or above it are appended to the class lists taken as one array (count in n_exact)
 // and marked in the map.
 // Contains CTA barriers.  Rare path, kept out of line.
+template <class SM>
 __device__ __noinline__ void select_exact_search(const unsigned* ub, bool nonzero, int len, int keff,
-                                                 SelectSmem& sm, unsigned* bitmap) {
+                                                 SM& sm, unsigned* bitmap) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long res = 0;
     if (tid == 0) sm.n_exact = 0;
@@ -134,9 +138,9 @@ struct Picked {
 // the thread's own slots are read).  Contains one CTA barrier: every thread of the CTA must call
 // it, and must synchronise again before select_rank().  Returns true when the threshold is 0, in
 // which case nothing was listed and the exact search has to run instead.
-template <bool WIDE>
+template <bool WIDE, class SM>
 __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], const unsigned* __restrict__ tile,
-                                            int len, int keff, SelectSmem& sm, Picked& out) {
+                                            int len, int keff, SM& sm, Picked& out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     out.mask = 0;
 
@@ -215,8 +219,8 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
                 cap = cls == kWideClasses - 1 ? kWideTopCap : kWideLowCap;
             } else {
                 cls = (kq >= s1 ? 1u : 0u) + (kq >= s2 ? 1u : 0u) + (kq >= s3 ? 1u : 0u);
-                off = cls * kClassCap;
-                cap = kClassCap;
+                off = cls * SM::kCap;
+                cap = SM::kCap;
             }
             const unsigned pos = atomicAdd(&sm.cnt[cls], 1u);
             if (pos < cap) {
@@ -230,8 +234,8 @@ __device__ __forceinline__ bool select_topk(const unsigned (&ub)[kPerThread], co
 
 // Second half of the selection, after the barrier that completes the class lists.  Returns true
 // when a list overflowed: nothing was marked and the exact search has to run instead.
-template <bool WIDE>
-__device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* bitmap, Picked& out) {
+template <bool WIDE, class SM>
+__device__ __forceinline__ bool select_rank(int keff, SM& sm, unsigned* bitmap, Picked& out) {
     const int tid = threadIdx.x;
     unsigned above = 0, cstar, L, list_off;
     const unsigned* __restrict__ lkf = &sm.lkey[0][0];
@@ -248,8 +252,8 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
                 if (above + cn.y < (unsigned)keff) { above += cn.y; cstar = 0; L = cn.x; }
             }
         }
-        if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)kClassCap) return true;  // overflow: exact search
-        list_off = cstar * kClassCap;
+        if (max(max(cn.x, cn.y), max(cn.z, cn.w)) > (unsigned)SM::kCap) return true;  // overflow: exact search
+        list_off = cstar * SM::kCap;
         // classes above the cut are selected whole: `above` (< keff <= 256) entries, one per thread
         if (tid < (int)above) {
             unsigned c = 3, j = tid;
@@ -261,8 +265,8 @@ __device__ __forceinline__ bool select_rank(int keff, SelectSmem& sm, unsigned* 
                     c = 1;
                 }
             }
-            out.p1 = lpf[c * kClassCap + j];
-            out.v1 = lkf[c * kClassCap + j] | ((out.p1 >> 12) << 31);
+            out.p1 = lpf[c * SM::kCap + j];
+            out.v1 = lkf[c * SM::kCap + j] | ((out.p1 >> 12) << 31);
             out.p1 &= 0xFFFu;
             out.mask |= 2u;
             set_bit(bitmap, out.p1);

@@ -56,7 +56,8 @@ struct sl_ctx {
     std::vector<sl_tensor_desc> tensors;
     ChunkDesc* d_chunks;
     TensorInfo* d_tinfo;
-    int ef_ctas;  // resident CTAs of the persistent compression kernel on this device
+    int ef_ctas;  // resident CTAs of the compact compression kernel on this device (informational)
+    int n_sms;
     // tensor-map (TMA) block copies: usable when every full chunk starts on a 64-element boundary
     bool tma_ok, tma_on;
     int n_classes;
@@ -234,11 +235,14 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     }
 
     prof_mark(c, -1, st);
-    const unsigned ef_grid = (unsigned)(G < c->ef_ctas ? G : c->ef_ctas);  // persistent CTAs
-    const size_t smem = sizeof(PipeSmem);
-#define SL_LAUNCH_EF1(EFV, PENDV, TMAV, WIDEV)                                                                        \
-    ef_topk_kernel<EFV, PENDV, TMAV, WIDEV><<<ef_grid, kThreads, smem, st>>>(c->d_chunks, G, workers, k, kp, c->cfg.beta, \
-                                                                             theta_sync, ptrs, ws, ta)
+    // persistent CTAs: as many as fit the device for the variant's shared-memory footprint
+#define SL_LAUNCH_EF1(EFV, PENDV, TMAV, WIDEV)                                                              \
+    do {                                                                                                    \
+        const long long ctas = (long long)c->n_sms * PipeSmemT<TMAV, WIDEV>::kCtasPerSm;                    \
+        ef_topk_kernel<EFV, PENDV, TMAV, WIDEV><<<(unsigned)(G < ctas ? G : ctas), kThreads,                \
+                                                  sizeof(PipeSmemT<TMAV, WIDEV>), st>>>(                    \
+            c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta);                         \
+    } while (0)
 #define SL_LAUNCH_EF(EFV, PENDV, TMAV)              \
     do {                                            \
         if (wide_classes(k)) SL_LAUNCH_EF1(EFV, PENDV, TMAV, true); \
@@ -486,10 +490,10 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     cudaError_t e = cudaGetDevice(&c->device);
     int n_sms = 0, per_sm = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
-    const int smem_bytes = (int)sizeof(PipeSmem);
-#define SL_SMEM_ATTR(...)                                                                                      \
+#define SL_SMEM_ATTR(EFV, PENDV, TMAV, WIDEV)                                                                  \
     if (e == cudaSuccess)                                                                                      \
-        e = cudaFuncSetAttribute(ef_topk_kernel<__VA_ARGS__>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)
+        e = cudaFuncSetAttribute(ef_topk_kernel<EFV, PENDV, TMAV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 (int)sizeof(PipeSmemT<TMAV, WIDEV>))
     SL_SMEM_ATTR(true, false, false, false);
     SL_SMEM_ATTR(false, false, false, false);
     SL_SMEM_ATTR(true, true, false, false);
@@ -503,9 +507,12 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     SL_SMEM_ATTR(false, false, true, true);
     SL_SMEM_ATTR(true, true, true, true);
 #undef SL_SMEM_ATTR
+    // the launch shape counts on the planned residency (the grid must not exceed what is co-resident
+    // only for speed: nothing in the kernel waits on another CTA)
     if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true, true>, kThreads,
-                                                          sizeof(PipeSmem));
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true, false>, kThreads,
+                                                          sizeof(PipeSmemT<true, false>));
+    c->n_sms = n_sms;
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
@@ -998,11 +1005,11 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
         int n_sms = 0, per_sm = 0;
         SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
         SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(PipeSmem)));
+                                     (int)sizeof(PipeSmemT<false, false>)));
         SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(PipeSmem)));
+                                     (int)sizeof(PipeSmemT<false, false>)));
         SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false, false, true>, kThreads,
-                                                              sizeof(PipeSmem)));
+                                                              sizeof(PipeSmemT<false, true>)));
         su.scratch = ptr;
         su.ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
         su.ready = true;
@@ -1031,10 +1038,10 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     TmaArgs no_tma;
     memset(&no_tma, 0, sizeof(no_tma));
     if (wide_classes(k))
-        ef_topk_kernel<true, false, false, true><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
+        ef_topk_kernel<true, false, false, true><<<ef_grid, kThreads, sizeof(PipeSmemT<false, false>), st>>>(d_chunks, G, 1, k, kp, beta,
                                                                                           theta_sync, ptrs, ws, no_tma);
     else
-        ef_topk_kernel<true, false, false, false><<<ef_grid, kThreads, sizeof(PipeSmem), st>>>(d_chunks, G, 1, k, kp, beta,
+        ef_topk_kernel<true, false, false, false><<<ef_grid, kThreads, sizeof(PipeSmemT<false, false>), st>>>(d_chunks, G, 1, k, kp, beta,
                                                                                            theta_sync, ptrs, ws, no_tma);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
