@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "c5_dense_d2048"
 
 # DRAM bytes per ef_topk launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
 # on a smaller case of the same kernel, as bytes per (parameter x worker); see profiles/.
-NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = 12.400  # profiles/ncu_full_c5_layer0_top3_kernels.md
+NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = 12.551  # profiles/ncu_full_c5_layer0_top3_kernels.md
 
 
 def record_stride(k: int) -> int:
