@@ -9,12 +9,18 @@ namespace {
 // ------------------------------------------------------------------------------------------------
 // Kernel 1: u = beta e + (theta - theta_r) written into e, chunk-wise Top-k of u into staging.
 //
-// Persistent CTAs (three per SM).  CTA b takes chunks b, b + grid, ... and, for each, the R workers
-// in turn ("units"), so the chunk of theta_sync is fetched once per chunk and kept in registers.
-// theta_r and e of a unit travel global -> shared as asynchronous 16-byte copies issued two units
-// ahead (two stages); every thread copies exactly the vectors it will consume itself, so no barrier
-// guards their arrival.  u is formed in registers, stored to e with 128-bit stores and kept in the
-// e stage for the selection.  Short tail chunks take plain loads.
+// Persistent CTAs (three or four per SM).  CTA b takes chunks b, b + grid, ... and, for each, the R
+// workers in turn ("units"), so the chunk of theta_sync is fetched once per chunk and kept in
+// registers.  theta_r and e of a unit travel global -> shared ahead of their use:
+//   TMA variant      one tensor-map block copy per 64x64 block, issued by one thread, completion on
+//                    shared-memory barriers with bounded waits; theta_r has one buffer (refilled from
+//                    the unit's first barrier for the next unit), e two stages (filled two units
+//                    ahead); u goes back to e as one block store from its stage;
+//   cp.async variant 16-byte copies issued two units ahead by every thread for exactly the vectors it
+//                    will consume itself, so no barrier guards their arrival; u is stored with
+//                    128-bit stores.
+// u is formed in registers and kept in the e stage for the selection.  Short tail chunks take plain
+// loads and stores.
 //
 // PENDING: the error buffers hold u of the previous step and the corrected values (u - Dhat) of the
 // selected entries wait in the staging arrays (deferred error-feedback subtraction).  The lists of
