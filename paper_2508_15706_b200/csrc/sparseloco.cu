@@ -27,6 +27,7 @@
 #include <string.h>
 
 #include <new>
+#include <mutex>
 #include <vector>
 
 #include "sparseloco.h"
@@ -927,6 +928,7 @@ struct StaticSetup {  // per device: address of the array above, launch shape of
     bool ready;
 };
 StaticSetup g_static_setup[64];
+std::mutex g_static_setup_mutex;  // first calls from several host threads set a device up once
 
 // Chunk table of a single tensor at element offset 0 (same rules as sl_create()).
 __global__ void __launch_bounds__(128)
@@ -999,6 +1001,7 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     SL_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return SL_ERR_UNSUPPORTED;
     StaticSetup& su = g_static_setup[dev];
+    std::lock_guard<std::mutex> lock(g_static_setup_mutex);  // (calls that overlap on the GPU race anyway: see the header)
     if (!su.ready) {  // first call on this device: resolve the array's device address, size the launch
         void* ptr = nullptr;
         SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
