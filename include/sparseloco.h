@@ -125,7 +125,11 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
 /* The whole outer step for R resident workers: sl_compress for r = 0..R-1, then
  * sl_aggregate_apply, with identical results, but free to share work between workers.
  *   theta_local, e, payloads : HOST arrays of R DEVICE pointers.  theta_local entries may alias
- *   each other; e and payload entries must not. */
+ *   each other; e and payload entries must not.
+ * The call only enqueues work, so it can be captured in a CUDA graph and replayed -- after one
+ * ordinary call with the same buffers (descriptors of a buffer are built and uploaded the first time
+ * its pointer is seen) and with the deferred subtraction off (that mode keeps host-side state that a
+ * replay would not advance). */
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
 

@@ -285,6 +285,32 @@ def test_side_stream_gives_the_same_result():
         assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
 
 
+def test_outer_step_in_a_cuda_graph():
+    """No entry point synchronises the host, so a step can be captured in a CUDA graph (after one
+    eager call, which builds the tensor maps of the buffers) and replayed: same bits as eager steps."""
+    wl = I.workload("c1_single_1024")
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    for c in (a, b):
+        c.fill_local(0)
+        c.step()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            a.sl.outer_step(a.theta, a.local, a.e, a.payloads)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        graph.replay()
+        b.sl.outer_step(b.theta, b.local, b.e, b.payloads)
+    torch.cuda.synchronize()
+    assert a.sl.device_status() == 0
+    assert torch.equal(a.theta, b.theta)
+    for r in range(wl.R):
+        assert torch.equal(a.e[r], b.e[r]) and torch.equal(a.payloads[r], b.payloads[r])
+
+
 def test_degenerate_tensor_sizes():
     """One-element and few-element tensors (k far above the chunk length), a single row shorter than a
     vector, and a table whose only tensor is a short chunk."""
