@@ -271,6 +271,27 @@ def run_ours(args) -> dict:
                                        "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
                                        "frac_of_measured_peak": dbytes / (dms * 1e-3) / 1e9 / peak,
                                        "entry_point": "sl_diloco_step", "beta_outer": 0.9}
+    if rank == 0 and world == 1 and not args.no_dense:
+        # the two halves of the step through their own entry points (sl_compress always writes
+        # the error correction in place; one worker per call)
+        if deferred:
+            sl.ef_flush()
+        p0, p1, p2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        sl.compress(theta, locals_r[0], e[0], payloads[0])
+        p0.record(stream)
+        for r in range(wl.R):
+            sl.compress(theta, locals_r[r], e[r], payloads[r])
+        p1.record(stream)
+        for _ in range(3):
+            sl.aggregate_apply(payloads, theta)
+        p2.record(stream)
+        torch.cuda.synchronize()
+        cms, ams = p0.elapsed_time(p1) / wl.R, p1.elapsed_time(p2) / 3
+        result["parts"] = {
+            "sl_compress_ms_per_worker": cms,
+            "sl_compress_gbs": (16 + 2 * record_stride(k) / 4096.0) * N / (cms * 1e-3) / 1e9,
+            "sl_aggregate_apply_ms": ams,
+            "sl_aggregate_apply_gbs": (8 + wl.R * record_stride(k) / 4096.0) * N / (ams * 1e-3) / 1e9}
     if rank == 0 and world == 1 and not args.no_e2e:
         del local, locals_r
         torch.cuda.empty_cache()
@@ -365,8 +386,18 @@ def cpu_baseline(wl, k, budget_s: float) -> dict:
     O.outer_step(cfg, tab, th, lo, e)
     dt = time.time() - t0
     names = ",".join(wl.tensors[j].name for j in ids)
-    return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
-            "sample": f"one outer step, all R={wl.R} workers, tensors [{names}] = {n} params of {wl.numel}"}
+    out = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
+           "sample": f"one outer step, all R={wl.R} workers, tensors [{names}] = {n} params of {wl.numel}"}
+    # the same program on one core, on the smallest tensor of the sample (a few seconds)
+    j1 = min(ids, key=lambda j: wl.tensors[j].numel)
+    cfg, tab, th, lo, e, n1 = make([j1], 0)
+    O.set_threads(1)
+    t0 = time.time()
+    O.outer_step(cfg, tab, th, lo, e)
+    dt1 = time.time() - t0
+    O.set_threads(cores)
+    out["single_thread"] = {"value": n1 / dt1, "seconds": dt1, "sample": f"tensor {wl.tensors[j1].name}, all R={wl.R} workers"}
+    return out
 
 
 def run_reference(args) -> dict:
