@@ -292,6 +292,30 @@ def run_ours(args) -> dict:
             "sl_compress_gbs": (16 + 2 * record_stride(k) / 4096.0) * N / (cms * 1e-3) / 1e9,
             "sl_aggregate_apply_ms": ams,
             "sl_aggregate_apply_gbs": (8 + wl.R * record_stride(k) / 4096.0) * N / (ams * 1e-3) / 1e9}
+    if rank == 0 and world == 1 and args.codec:
+        # entropy-coded index format: one worker's payload of the last step, encode and decode
+        coded = torch.empty(sl.coded_payload_capacity(), dtype=torch.uint8, device=dev)
+        size = torch.zeros(1, dtype=torch.int64, device=dev)
+        back = torch.empty_like(payloads[0])
+        for _ in range(3):
+            sl.encode_payload(payloads[0], coded, size)
+            sl.decode_payload(coded, back)
+        c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        c0.record(stream)
+        for _ in range(10):
+            sl.encode_payload(payloads[0], coded, size)
+        c1.record(stream)
+        for _ in range(10):
+            sl.decode_payload(coded, back)
+        c2.record(stream)
+        torch.cuda.synchronize()
+        chunks, slots = sl.num_chunks()
+        nbytes = int(size.item())
+        code_block = (2 * k + 7) // 8
+        result["index_codec"] = {
+            "payload_bytes": sl.payload_bytes(), "coded_bytes": nbytes, "round_trip_identical": bool(torch.equal(back, payloads[0])),
+            "index_bits_per_value": 8.0 * (nbytes - 16 * len(wl.tensors) - code_block * chunks) / slots,
+            "encode_ms": c0.elapsed_time(c1) / 10, "decode_ms": c1.elapsed_time(c2) / 10}
     if rank == 0 and world == 1 and not args.no_e2e:
         del local, locals_r
         torch.cuda.empty_cache()
@@ -448,6 +472,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense DiLoCo comparator line")
+    ap.add_argument("--codec", action="store_true", help="also time the entropy-coded index format on one payload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")
