@@ -52,6 +52,34 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
     unsigned* recs = reinterpret_cast<unsigned*>(mu_t3 + 2 * 32);          // batch x (stride + 16) bytes
     const int stride = record_stride(k), rwords = stride / 4 + 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kEnt = SPL * WPW;  // entries per thread and batch
+    static_assert(kEnt <= kApplyEntries && WPW <= 4, "entry budget");
+    constexpr int batch = 8 * WPW;
+    // FUSE: the staged (index, value) pairs of this thread's entries in the first batch.  They need
+    // nothing from the chunk table (slots up to k exist for every chunk; those beyond the chunk's
+    // own count are ignored later), so they start before anything else.
+    unsigned pre_p[kEnt];
+    float pre_v[kEnt];
+#pragma unroll
+    for (int e = 0; e < kEnt; ++e) {
+        pre_p[e] = 0u;
+        pre_v[e] = 0.f;
+    }
+    if (FUSE) {
+#pragma unroll
+        for (int wi = 0; wi < WPW; ++wi) {
+            const int rb = warp + 8 * wi;
+            const long long slot_base = ((long long)rb * fa.n_chunks + blockIdx.x) * fa.kp;
+#pragma unroll
+            for (int si = 0; si < SPL; ++si) {
+                const int sl = lane + 32 * si;
+                if (rb < n_workers && sl < k) {
+                    pre_p[wi * SPL + si] = fa.ws.idx[slot_base + sl];
+                    pre_v[wi * SPL + si] = fa.ws.val[slot_base + sl];
+                }
+            }
+        }
+    }
     const ChunkDesc cd = chunks[blockIdx.x];
     const int keff = min(k, cd.len);
     const int code_byte0 = record_index_bytes(k);
@@ -72,20 +100,10 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
     for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
 
     // entry e of a thread: worker warp + 8 (e / SPL), slot lane + 32 (e % SPL)
-    constexpr int kEnt = SPL * WPW;  // entries per thread and batch
-    static_assert(kEnt <= kApplyEntries && WPW <= 4, "entry budget");
-    constexpr int batch = 8 * WPW;
     const int vec_per_rec = stride / 16;
 
     for (int r0 = 0; r0 < n_workers; r0 += batch) {
         const int nb = min(batch, n_workers - r0);
-        unsigned pre_p[kEnt];
-        float pre_v[kEnt];
-#pragma unroll
-        for (int e = 0; e < kEnt; ++e) {
-            pre_p[e] = 0u;
-            pre_v[e] = 0.f;
-        }
         // clear the masks, stage this batch's records and tables (the last barrier of the
         // previous batch's rounds has released both)
 #pragma unroll
@@ -105,7 +123,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
                 recs[tid * rwords + stride / 4] = 0;  // word read past the index block by get12
             }
         } else {
-            // staged (index, value) pairs of this thread's entries: loads in flight across the barrier
+            // staged pairs of the later batches (the first batch's are already on their way)
 #pragma unroll
             for (int wi = 0; wi < WPW; ++wi) {
                 const int rb = warp + 8 * wi;
@@ -113,7 +131,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int
 #pragma unroll
                 for (int si = 0; si < SPL; ++si) {
                     const int sl = lane + 32 * si;
-                    if (rb < nb && sl < keff) {
+                    if (r0 > 0 && rb < nb && sl < keff) {
                         pre_p[wi * SPL + si] = fa.ws.idx[slot_base + sl];
                         pre_v[wi * SPL + si] = fa.ws.val[slot_base + sl];
                     }
