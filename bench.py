@@ -271,6 +271,23 @@ def run_ours(args) -> dict:
                                        "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
                                        "frac_of_measured_peak": dbytes / (dms * 1e-3) / 1e9 / peak,
                                        "entry_point": "sl_diloco_step", "beta_outer": 0.9}
+    if rank == 0 and world == 1 and not args.no_dense and deferred:
+        # the same step with the error correction written in place by every step (the library's
+        # default mode), for comparison with the headline's deferred form
+        sl.ef_flush()
+        sl.set_ef_deferred(False)
+        sl.outer_step(theta, locals_r, e, payloads)
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record(stream)
+        for _ in range(5):
+            sl.outer_step(theta, locals_r, e, payloads)
+        m1.record(stream)
+        torch.cuda.synchronize()
+        mms = m0.elapsed_time(m1) / 5
+        result["materialised_step"] = {"ms_per_step": mms, "params_per_s": N / (mms * 1e-3),
+                                       "note": "sl_outer_step with sl_set_ef_deferred(0): e = u - Dhat written by a "
+                                               "scattered pass in every step"}
+        sl.set_ef_deferred(True)
     if rank == 0 and world == 1 and not args.no_dense:
         # the two halves of the step through their own entry points (sl_compress always writes
         # the error correction in place; one worker per call)
