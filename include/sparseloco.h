@@ -167,13 +167,21 @@ sl_status sl_diloco_step(sl_ctx* ctx, float* theta_sync, const float* const* the
  *                               *dev_coded_bytes (DEVICE uint64, 8-byte aligned).  Uses the lent
  *                               workspace as scratch (NOMEM without one) and must not overlap a
  *                               compression on another stream.
- *   sl_decode_payload         : coded -> payload (sl_payload_bytes() bytes, fully overwritten).  A
- *                               corrupted stream yields a wrong but well-bounded record, never an
- *                               out-of-range access; run sl_validate_payload on the result. */
+ *   sl_decode_payload         : coded -> payload (sl_payload_bytes() bytes, fully overwritten).
+ *                               coded_bytes (host value) = bytes of `coded` that may be read: the size
+ *                               sl_encode_payload reported, or 0 for the full capacity; it must cover
+ *                               the tables, code blocks and directory (else INVALID_ARG).  No read
+ *                               goes past it: a directory entry beyond it is clamped and a stream
+ *                               that runs out reads as zero bits, so a corrupted input yields a
+ *                               wrong but well-formed-sized record, never an out-of-range access.
+ *                               Such an input (also a directory that does not ascend) records
+ *                               SL_ERR_BAD_PAYLOAD in the device status word (sl_device_status); run
+ *                               sl_validate_payload on the result as well. */
 sl_status sl_coded_payload_capacity(const sl_ctx* ctx, size_t* bytes);
 sl_status sl_encode_payload(sl_ctx* ctx, const uint8_t* payload, uint8_t* coded, uint64_t* dev_coded_bytes,
                             void* cuda_stream);
-sl_status sl_decode_payload(sl_ctx* ctx, const uint8_t* coded, uint8_t* payload, void* cuda_stream);
+sl_status sl_decode_payload(sl_ctx* ctx, const uint8_t* coded, size_t coded_bytes, uint8_t* payload,
+                            void* cuda_stream);
 
 /* How the compression kernel moves the 64x64 blocks of theta_r and e (no counterpart in the paper).
  * 1: one tensor-map (TMA) block copy per block and direction, completion on shared-memory barriers --

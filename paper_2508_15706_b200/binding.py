@@ -74,7 +74,7 @@ def _load():
     L.sl_diloco_step.argtypes = [P, P, P, P, C.c_float, P]
     L.sl_coded_payload_capacity.argtypes = [P, C.POINTER(C.c_size_t)]
     L.sl_encode_payload.argtypes = [P, P, P, P, P]
-    L.sl_decode_payload.argtypes = [P, P, P, P]
+    L.sl_decode_payload.argtypes = [P, P, C.c_size_t, P, P]
     L.sl_set_tile_copies.argtypes = [P, C.c_int32]
     L.sl_device_status.argtypes = [P, P]
     L.sl_static_scratch_bytes.restype = C.c_size_t
@@ -266,8 +266,11 @@ class SparseLoCo:
         _check(_L.sl_encode_payload(self._h, _dev_ptr(payload, torch.uint8), _dev_ptr(coded, torch.uint8),
                                     _dev_ptr(coded_bytes), _stream()))
 
-    def decode_payload(self, coded, payload) -> None:
-        _check(_L.sl_decode_payload(self._h, _dev_ptr(coded, torch.uint8), _dev_ptr(payload, torch.uint8), _stream()))
+    def decode_payload(self, coded, payload, coded_bytes: int = 0) -> None:
+        """Entropy-coded payload -> 12-bit payload.  `coded_bytes` = readable bytes of `coded`
+        (0: the tensor's size); a damaged input shows in device_status() as SL_ERR_BAD_PAYLOAD."""
+        _check(_L.sl_decode_payload(self._h, _dev_ptr(coded, torch.uint8), coded_bytes or coded.numel(),
+                                    _dev_ptr(payload, torch.uint8), _stream()))
 
     def set_tile_copies(self, use_tensor_maps: bool) -> None:
         _check(_L.sl_set_tile_copies(self._h, int(use_tensor_maps)))

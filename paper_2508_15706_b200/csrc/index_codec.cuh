@@ -162,19 +162,31 @@ ixc_write_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
 }
 
 // K4: coded payload -> 12-bit records.  One thread per group of 16 chunks (one directory entry).
+// `stream_bits` = bits of the index stream that the caller's buffer holds: a read position taken from
+// the directory is clamped to it and a bit past it reads as 0, so a corrupted directory or stream
+// never makes the kernel touch memory outside the coded buffer; either case (and a directory that
+// does not ascend) is recorded as SL_ERR_BAD_PAYLOAD in `status`.
 __global__ void __launch_bounds__(128)
 ixc_decode_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_tensors, int k,
                   const uint8_t* __restrict__ coded, unsigned long long dir_off, unsigned long long stream_off,
-                  uint8_t* __restrict__ payload) {
+                  unsigned long long stream_bits, uint8_t* __restrict__ payload, int* __restrict__ status) {
     const long long grp = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (grp < 4ll * n_tensors)
         reinterpret_cast<unsigned*>(payload)[grp] = reinterpret_cast<const unsigned*>(coded)[grp];
     const long long g0 = grp * kIxcGroup;
     if (g0 >= n_chunks) return;
     const unsigned* stream = reinterpret_cast<const unsigned*>(coded + stream_off);
-    unsigned long long pos = reinterpret_cast<const unsigned*>(coded + dir_off)[grp];
+    const unsigned* dir = reinterpret_cast<const unsigned*>(coded + dir_off);
+    unsigned long long pos = dir[grp];
+    bool bad = pos > stream_bits;
+    if (g0 + kIxcGroup < n_chunks) bad |= dir[grp + 1] < pos;
+    if (pos > stream_bits) pos = stream_bits;
     const int cb = (2 * k + 7) / 8, ib = (12 * k + 7) / 8, stride = record_stride(k);
     auto get1 = [&]() -> unsigned {
+        if (pos >= stream_bits) {
+            bad = true;
+            return 0u;
+        }
         const unsigned bit = (stream[pos >> 5] >> (pos & 31)) & 1u;
         ++pos;
         return bit;
@@ -213,6 +225,7 @@ ixc_decode_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
         for (int i = 0; i < cb; ++i) recb[ib + i] = csrc[i];
         for (byte = ib + cb; byte < stride; ++byte) recb[byte] = 0;
     }
+    if (bad) atomicExch(status, (int)SL_ERR_BAD_PAYLOAD);
 }
 
 }  // namespace

@@ -2,8 +2,8 @@
 // file) over the kernels in the .cuh files beside it (one translation unit).
 //
 // Kernel sequence of one outer step (all on the caller's stream, no host synchronisation):
-//   ef_topk.cuh      ef_topk_kernel           pseudo-gradient + error feedback + chunk-wise Top-k
-//                                             (Eq. 2 line 1, Sec. 3.3); selection.cuh holds the Top-k
+//   ef_select.cuh    ef_select_kernel         pseudo-gradient + error feedback + chunk-wise Top-k
+//                                             (Eq. 2 line 1, Sec. 3.3), one warp per (chunk, worker)
 //   quantiser.cuh    chunk_sum_kernel<0>      per-chunk fp64 sum of the selected values   (Sec. 4: mean)
 //                    tensor_reduce_kernel<0>  grouped fp64 sum per (worker, tensor) -> mu
 //                    chunk_sum_kernel<1>      per-chunk fp64 sum of squared centred values
@@ -33,8 +33,7 @@
 #include "sparseloco.h"
 
 #include "common.cuh"
-#include "selection.cuh"
-#include "ef_topk.cuh"
+#include "ef_select.cuh"
 #include "quantiser.cuh"
 #include "pack.cuh"
 #include "apply.cuh"
@@ -67,6 +66,10 @@ struct sl_ctx {
     std::vector<CUtensorMap> h_maps;    // host copy the device array is filled from
     std::vector<const void*> slot_ptr;  // buffer described by each slot
     bool slots_cleared;                 // the slot table was emptied during the current assignment
+    bool maps_fresh;                    // maps were (re)written since the last compression launch
+    bool upload_pending;                // ... and that upload has no event yet
+    cudaEvent_t upload_event;           // recorded after the last upload, on upload_stream
+    cudaStream_t upload_stream;
     int* d_status;                      // device status word (SL_OK or what a kernel recorded)
     // entropy-coded payload: byte offsets of the directory and the index stream, worst-case size
     size_t ixc_dir_off, ixc_stream_off, ixc_capacity;
@@ -88,7 +91,7 @@ struct sl_ctx {
 
 namespace {
 
-constexpr int kMapSlots = 2 * kMaxR + 2;  // buffers with tensor maps at one time: theta_local and e of every worker
+constexpr int kMapSlots = 2 * kMaxR + 2;  // buffers with tensor maps at one time: theta, theta_local and e of every worker
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
 typedef CUresult (*TmaEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -175,7 +178,27 @@ int tma_map_slot(sl_ctx* c, const void* ptr, cudaStream_t st) {
                         sizeof(CUtensorMap) * c->n_classes, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return -1;
     c->slot_ptr.push_back(ptr);
+    c->maps_fresh = true;     // the next launch fences before its first copy through a rewritten map
+    c->upload_pending = true; // ... and other streams must be ordered after this upload
     return slot;
+}
+
+// Tensor maps are uploaded on the stream of the call that first sees a buffer.  A later call on another
+// stream finds the slot by pointer alone, so it is ordered after the last upload through an event.
+sl_status order_after_map_uploads(sl_ctx* c, cudaStream_t st) {
+    if (c->upload_pending) {
+        if (!c->upload_event) SL_CUDA(cudaEventCreateWithFlags(&c->upload_event, cudaEventDisableTiming));
+        SL_CUDA(cudaEventRecord(c->upload_event, st));
+        c->upload_stream = st;
+        c->upload_pending = false;
+    } else if (c->upload_event && st != c->upload_stream) {
+        // (not while `st` is being captured into a graph: the event belongs to no capture; the header
+        // asks for one ordinary call with the same buffers before a capture, which is what orders it)
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        SL_CUDA(cudaStreamIsCapturing(st, &cap));
+        if (cap == cudaStreamCaptureStatusNone) SL_CUDA(cudaStreamWaitEvent(st, c->upload_event, 0));
+    }
+    return SL_OK;
 }
 
 sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
@@ -216,16 +239,18 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     // tile copies through tensor maps when the table allows it and every buffer got its maps
     TmaArgs ta;
     memset(&ta, 0, sizeof(ta));
+    ta.status = c->d_status;
     bool use_tma = c->tma_on;
     if (use_tma) {
         ta.maps = c->d_maps;
         ta.n_classes = c->n_classes;
-        ta.status = c->d_status;
         for (int q = 0; q < c->n_classes; ++q) ta.class_rs[q] = c->class_rs[q];
         for (int pass = 0; pass < 2 && use_tma; ++pass) {
             // if the slot table fills up half-way, it is emptied and the assignment starts over: one
-            // call needs at most 2 R slots, which an empty table holds
+            // call needs at most 2 R + 1 slots, which an empty table holds
             c->slots_cleared = false;
+            ta.slot_s = tma_map_slot(c, theta_sync, st);
+            use_tma = ta.slot_s >= 0;
             for (int r = 0; r < workers && use_tma; ++r) {
                 ta.slot_l[r] = tma_map_slot(c, ptrs.theta_local[r], st);
                 ta.slot_e[r] = ef ? tma_map_slot(c, ptrs.e[r], st) : 0;
@@ -233,33 +258,28 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
             }
             if (!c->slots_cleared) break;
         }
+        if (use_tma) {
+            sl_status s = order_after_map_uploads(c, st);
+            if (s != SL_OK) return s;
+            ta.fresh = c->maps_fresh ? 1 : 0;
+            c->maps_fresh = false;
+        }
     }
 
     prof_mark(c, -1, st);
-    // persistent CTAs: as many as fit the device for the variant's shared-memory footprint
-#define SL_LAUNCH_EF1(EFV, PENDV, TMAV, WIDEV)                                                              \
-    do {                                                                                                    \
-        const long long ctas = (long long)c->n_sms * PipeSmemT<TMAV, WIDEV>::kCtasPerSm;                    \
-        ef_topk_kernel<EFV, PENDV, TMAV, WIDEV><<<(unsigned)(G < ctas ? G : ctas), kThreads,                \
-                                                  sizeof(PipeSmemT<TMAV, WIDEV>), st>>>(                    \
-            c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta);                         \
-    } while (0)
-#define SL_LAUNCH_EF(EFV, PENDV, TMAV)              \
-    do {                                            \
-        if (wide_classes(k)) SL_LAUNCH_EF1(EFV, PENDV, TMAV, true); \
-        else SL_LAUNCH_EF1(EFV, PENDV, TMAV, false); \
-    } while (0)
-    if (use_tma) {
-        if (!ef) SL_LAUNCH_EF(false, false, true);
-        else if (consume) SL_LAUNCH_EF(true, true, true);
-        else SL_LAUNCH_EF(true, false, true);
-    } else {
-        if (!ef) SL_LAUNCH_EF(false, false, false);
-        else if (consume) SL_LAUNCH_EF(true, true, false);
-        else SL_LAUNCH_EF(true, false, false);
+    {   // one persistent CTA per SM
+        const unsigned grid = (unsigned)(G < c->n_sms ? G : c->n_sms);
+        const int tm = use_tma ? 1 : 0;
+        if (!ef)
+            ef_select_kernel<false, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
+                                                                                       c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
+        else if (consume)
+            ef_select_kernel<true, true><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
+                                                                                     c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
+        else
+            ef_select_kernel<true, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
+                                                                                      c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
     }
-#undef SL_LAUNCH_EF
-#undef SL_LAUNCH_EF1
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
@@ -395,6 +415,9 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->ef_ctas = 0;
     c->tma_ok = c->tma_on = false;
     c->slots_cleared = false;
+    c->maps_fresh = c->upload_pending = false;
+    c->upload_event = nullptr;
+    c->upload_stream = nullptr;
     c->n_classes = 0;
     c->d_maps = nullptr;
     c->d_status = nullptr;
@@ -491,28 +514,13 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     cudaError_t e = cudaGetDevice(&c->device);
     int n_sms = 0, per_sm = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
-#define SL_SMEM_ATTR(EFV, PENDV, TMAV, WIDEV)                                                                  \
-    if (e == cudaSuccess)                                                                                      \
-        e = cudaFuncSetAttribute(ef_topk_kernel<EFV, PENDV, TMAV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                 (int)sizeof(PipeSmemT<TMAV, WIDEV>))
-    SL_SMEM_ATTR(true, false, false, false);
-    SL_SMEM_ATTR(false, false, false, false);
-    SL_SMEM_ATTR(true, true, false, false);
-    SL_SMEM_ATTR(true, false, true, false);
-    SL_SMEM_ATTR(false, false, true, false);
-    SL_SMEM_ATTR(true, true, true, false);
-    SL_SMEM_ATTR(true, false, false, true);
-    SL_SMEM_ATTR(false, false, false, true);
-    SL_SMEM_ATTR(true, true, false, true);
-    SL_SMEM_ATTR(true, false, true, true);
-    SL_SMEM_ATTR(false, false, true, true);
-    SL_SMEM_ATTR(true, true, true, true);
-#undef SL_SMEM_ATTR
-    // the launch shape counts on the planned residency (the grid must not exceed what is co-resident
-    // only for speed: nothing in the kernel waits on another CTA)
     if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, true, true, false>, kThreads,
-                                                          sizeof(PipeSmemT<true, false>));
+        e = cudaFuncSetAttribute(ef_select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_select_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
+    per_sm = 1;
     c->n_sms = n_sms;
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int));
@@ -547,6 +555,7 @@ sl_status sl_destroy(sl_ctx* c) {
     cudaFree(c->d_tinfo);
     cudaFree(c->d_status);
     cudaFree(c->d_maps);
+    if (c->upload_event) cudaEventDestroy(c->upload_event);
     for (auto& ev : c->prof_events) cudaEventDestroy(ev);
     if (c->host_path_ready) {
         cudaStreamDestroy(c->copy_stream);
@@ -819,15 +828,21 @@ sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, u
     return SL_OK;
 }
 
-sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, uint8_t* payload, void* stream) {
+sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, size_t coded_bytes, uint8_t* payload, void* stream) {
     if (!c || !coded || !payload) return SL_ERR_INVALID_ARG;
     if (misaligned(coded) || misaligned(payload)) return SL_ERR_ALIGNMENT;
+    if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
+    // what the buffer is said to hold bounds every read; it must at least reach the index stream
+    if (coded_bytes == 0 || coded_bytes > c->ixc_capacity) coded_bytes = c->ixc_capacity;
+    if (coded_bytes < c->ixc_stream_off) return SL_ERR_INVALID_ARG;
+    const unsigned long long stream_bits = (unsigned long long)((coded_bytes - c->ixc_stream_off) / 4 * 4) * 8ull;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     const long long groups = (c->n_chunks + kIxcGroup - 1) / kIxcGroup;
     const long long items = groups > 4ll * c->n_tensors ? groups : 4ll * c->n_tensors;
     ixc_decode_kernel<<<blocks_for(items, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        c->d_chunks, c->n_chunks, c->n_tensors, c->cfg.k, coded, c->ixc_dir_off, c->ixc_stream_off, payload);
+        c->d_chunks, c->n_chunks, c->n_tensors, c->cfg.k, coded, c->ixc_dir_off, c->ixc_stream_off, stream_bits,
+        payload, c->d_status);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -924,6 +939,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 struct StaticSetup {  // per device: address of the array above, launch shape of the persistent kernel
     void* scratch;
+    int* status;  // where the kernel would record a bounded wait that ran out: the array's last 256 bytes
     int ef_ctas;
     bool ready;
 };
@@ -995,7 +1011,7 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     const size_t off_pcnt = off_pbin + up256(WG * 4 * sizeof(double));
     const size_t off_tstat = off_pcnt + up256(WG * 4 * sizeof(unsigned));
     const size_t need = off_tstat + up256(sizeof(TStat));
-    if (need > kStaticScratchBytes) return SL_ERR_TOO_LARGE;  // the fixed scratch cannot hold this tensor
+    if (need > kStaticScratchBytes - 256) return SL_ERR_TOO_LARGE;  // the fixed scratch cannot hold this tensor
 
     int dev = -1;
     SL_CUDA(cudaGetDevice(&dev));
@@ -1005,16 +1021,13 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     if (!su.ready) {  // first call on this device: resolve the array's device address, size the launch
         void* ptr = nullptr;
         SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
-        int n_sms = 0, per_sm = 0;
+        int n_sms = 0;
         SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(PipeSmemT<false, false>)));
-        SL_CUDA(cudaFuncSetAttribute(ef_topk_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(PipeSmemT<false, false>)));
-        SL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ef_topk_kernel<true, false, false, true>, kThreads,
-                                                              sizeof(PipeSmemT<false, true>)));
+        SL_CUDA(cudaFuncSetAttribute(ef_select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(SelSmem)));
         su.scratch = ptr;
-        su.ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
+        su.status = reinterpret_cast<int*>(static_cast<char*>(ptr) + kStaticScratchBytes - 256);
+        su.ef_ctas = n_sms;
         su.ready = true;
     }
     char* base = static_cast<char*>(su.scratch);
@@ -1038,14 +1051,11 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     // by an earlier call (of any size) is ever consumed and nothing has to be cleared.
     build_single_tensor_table_kernel<<<blocks_for(G, 128), 128, 0, st>>>(rows, cols, k, G, d_chunks, d_tinfo);
     const unsigned ef_grid = (unsigned)(G < su.ef_ctas ? G : su.ef_ctas);
-    TmaArgs no_tma;
+    TmaArgs no_tma;  // plain loads and stores: nothing has to be encoded or uploaded for the caller's buffers
     memset(&no_tma, 0, sizeof(no_tma));
-    if (wide_classes(k))
-        ef_topk_kernel<true, false, false, true><<<ef_grid, kThreads, sizeof(PipeSmemT<false, false>), st>>>(d_chunks, G, 1, k, kp, beta,
-                                                                                          theta_sync, ptrs, ws, no_tma);
-    else
-        ef_topk_kernel<true, false, false, false><<<ef_grid, kThreads, sizeof(PipeSmemT<false, false>), st>>>(d_chunks, G, 1, k, kp, beta,
-                                                                                           theta_sync, ptrs, ws, no_tma);
+    no_tma.status = su.status;
+    ef_select_kernel<true, false><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync, ptrs,
+                                                                              ws, no_tma, 0);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
     tensor_reduce_kernel<0><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);

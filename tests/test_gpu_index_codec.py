@@ -74,3 +74,68 @@ def test_full_size_round_trip_and_rate():
     index_bits = 8 * (n - 16 * T - 16 * chunks) / slots   # code blocks are 16 bytes per chunk at k = 64
     assert index_bits < 8.0, index_bits                   # 12 in the plain format; 7.36 is the bound at k = 64
     assert n < 0.72 * c.sl.payload_bytes()
+
+
+def test_damaged_coded_payloads_stay_inside_the_buffer():
+    """A coded payload damaged on the host -- directory entries far beyond the stream, a directory
+    that goes backwards, a stream of all ones, a truncated buffer -- is decoded without reading past
+    the bytes the caller declared (the decoder clamps every position to them) and the damage is
+    reported: SL_ERR_BAD_PAYLOAD in the status word and / or a record sl_validate_payload rejects.
+    The coded buffer is a slice that ends exactly at the declared size, inside a larger allocation
+    filled with a canary, so the bytes behind it are known and the output must not depend on them."""
+    wl = I.Workload("ixc_bad", [I.TensorSpec("w", 512, 512, 0), I.TensorSpec("v", 1, 5000, 0)], R=1, k=64,
+                    recipe="normal", seed=5)
+    c = _case(wl, e_scale=0.5)
+    c.fill_local(0)
+    c.step()
+    cap = c.sl.coded_payload_capacity()
+    good = torch.zeros(cap, dtype=torch.uint8, device=c.dev)
+    size = torch.zeros(1, dtype=torch.int64, device=c.dev)
+    c.sl.encode_payload(c.payloads[0], good, size)
+    torch.cuda.synchronize()
+    n = int(size.item())
+    chunks, _ = c.sl.num_chunks()
+    T = len(c.shapes)
+    dir_off = (16 * T + 16 * chunks + 3) // 4 * 4
+    n_dir = (chunks + 15) // 16
+    stream_off = dir_off + 4 * n_dir
+    status = torch.zeros(1, dtype=torch.int32, device=c.dev)
+
+    def run(mutate, declared):
+        host = good[:n].cpu().numpy().copy()
+        mutate(host)
+        arena = torch.full((cap + 4096,), 0xEE, dtype=torch.uint8, device=c.dev)
+        arena[:declared] = torch.from_numpy(host[:declared]).to(c.dev)
+        outs = []
+        for canary in (0xEE, 0x11):  # whatever lies behind the declared bytes must not matter
+            arena[declared:] = canary
+            back = torch.full_like(c.payloads[0], 0xA5)
+            c.sl.decode_payload(arena, back, coded_bytes=declared)
+            dev_status = c.sl.device_status()
+            c.sl.validate_payload(back, status)
+            torch.cuda.synchronize()
+            outs.append((back.cpu().numpy().copy(), dev_status, int(status.item())))
+        assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1:] == outs[1][1:]
+        return outs[0]
+
+    # untouched: round trip, nothing reported
+    back, st, val = run(lambda h: None, n)
+    assert st == 0 and val == 0 and np.array_equal(back, c.payloads[0].cpu().numpy())
+
+    def far_directory(h):
+        h[dir_off + 4:dir_off + 8] = np.frombuffer(np.uint32(0xFFFFFF00).tobytes(), np.uint8)
+    back, st, val = run(far_directory, n)
+    assert st == 4
+
+    def backwards_directory(h):
+        h[dir_off + 8:dir_off + 12] = 0
+    back, st, val = run(backwards_directory, n)
+    assert st == 4
+
+    def all_ones(h):
+        h[stream_off:] = 0xFF
+    back, st, val = run(all_ones, n)
+    assert st == 4 or val == 4
+
+    back, st, val = run(lambda h: None, stream_off + 16)  # truncated: most of the stream is missing
+    assert st == 4
