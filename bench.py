@@ -124,9 +124,36 @@ def pick_distinct_locals(torch, wl, k: int, flat: int, payload_bytes: int, works
     free, _total = torch.cuda.mem_get_info()
     fixed = (1 + wl.R) * 4 * flat + wl.R * payload_bytes + workspace_bytes + (6 << 30)
     for D in [wl.R] + [d for d in (32, 16, 8, 4, 2, 1) if d < wl.R]:
-        if fixed + D * 4 * flat <= free:
+        shifted = 0 if D == wl.R else 4 * ALIAS_SHIFT * ((wl.R + D - 1) // D - 1)
+        if fixed + D * (4 * flat + shifted) <= free:
             return D
     raise RuntimeError(f"workload {wl.name} does not fit: need {fixed + 4 * flat} bytes, {free} free")
+
+
+ALIAS_SHIFT = 1 << 26  # elements (268 MB) between the views of two workers that share a theta_local buffer
+
+
+def make_locals(torch, I, wl, theta, D: int, shift: int):
+    """theta_local of every worker when only D < R distinct buffers fit.  Worker r reads buffer r % D
+    through a view that starts (r // D) * shift elements into it (the buffers are that much longer,
+    the tail filled with noise of theta's scale), so two workers that share a buffer read addresses
+    268 MB apart for the same chunk: every one of the R reads of a chunk comes from HBM, as it would
+    with R distinct buffers.  With shift = 0 the workers read identical views and the second read of
+    a chunk can be served from L2.  Returns (storage, views)."""
+    flat = theta.numel()
+    extra = shift * ((wl.R + D - 1) // D - 1)
+    storage, views = [], []
+    for d in range(D):
+        buf = torch.empty(flat + extra, dtype=torch.float32, device=theta.device)
+        I.theta_local(wl, theta, d, 0, out=buf)
+        if extra:
+            g = torch.Generator(device=theta.device).manual_seed(77_000 + d)
+            buf[flat:].normal_(0.0, 0.02, generator=g)
+        storage.append(buf)
+    for r in range(wl.R):
+        o = (r // D) * shift
+        views.append(storage[r % D][o:o + flat])
+    return storage, views
 
 
 def run_ours(args) -> dict:
@@ -160,16 +187,14 @@ def run_ours(args) -> dict:
     sl.set_ef_deferred(deferred)
     if args.tile_copies != "auto":
         sl.set_tile_copies(args.tile_copies == "tma")
-    D = pick_distinct_locals(torch, wl, k, flat, sl.payload_bytes(), sl.workspace_bytes())
+    D = args.distinct_locals or pick_distinct_locals(torch, wl, k, flat, sl.payload_bytes(), sl.workspace_bytes())
+    shift = args.alias_shift if D < wl.R else 0
     ws = torch.empty(sl.workspace_bytes(), dtype=torch.uint8, device=dev)
     sl.set_workspace(ws)
     theta = I.theta_sync(wl, dev)
-    local = []
-    for d in range(D):
-        local.append(I.theta_local(wl, theta, d, 0))
+    local, locals_r = make_locals(torch, I, wl, theta, D, shift)
     e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(wl.R)]
     payloads = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(wl.R)]
-    locals_r = [local[r % D] for r in range(wl.R)]
     torch.cuda.synchronize()
 
     def barrier():
@@ -231,7 +256,11 @@ def run_ours(args) -> dict:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "params": N, "tensors": len(wl.tensors), "R": wl.R, "k": k, "H": wl.H,
                    "chunk": 4096, "beta": wl.beta, "outer_lr": wl.outer_lr,
-                   "distinct_theta_local_buffers": D, "tile_copies": args.tile_copies,
+                   "distinct_theta_local_buffers": D,
+                   "theta_local_sharing": ("none" if D == wl.R else
+                                           f"worker r reads buffer r % {D} through a view shifted by (r // {D}) x {shift} elements"
+                                           if shift else f"worker r reads buffer r % {D} (identical views: L2 can serve re-reads)"),
+                   "tile_copies": args.tile_copies,
                    "ef_subtract": args.ef_subtract + (" (each step substitutes the previous step's corrected values "
                                                       "while streaming e; a final flush is inside the timed region)"
                                                       if deferred else ""),
@@ -339,12 +368,109 @@ def run_ours(args) -> dict:
         result["e2e"] = run_e2e(torch, I, sl, wl, theta, e, payloads, flat, N, args)
     elif not args.no_e2e:
         result["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_alias_check and wl.name == DEFAULT_WORKLOAD:
+        # everything of the main workload goes before the check allocates its own
+        del sl, ws, theta, e, payloads
+        local = locals_r = None
+        torch.cuda.empty_cache()
+        result["theta_local_sharing_check"] = sharing_check(torch, I, dev, peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, k, budget_s=args.cpu_budget)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     return result if rank == 0 else None
+
+
+def time_compression_kernel(torch, sl, theta, locals_r, e, payloads, steps: int = 4) -> float:
+    """Average milliseconds of the compression kernel over `steps` outer steps (CUDA events recorded by
+    the library around the kernel on the launch stream), after two warm-up steps."""
+    for _ in range(2):
+        sl.outer_step(theta, locals_r, e, payloads)
+    torch.cuda.synchronize()
+    sl.profile_enable(True)
+    for _ in range(steps):
+        sl.outer_step(theta, locals_r, e, payloads)
+    torch.cuda.synchronize()
+    ms, n = sl.profile_read()["ef_topk"]
+    sl.profile_enable(False)
+    return ms / max(n, 1)
+
+
+def sharing_check(torch, I, dev, peak: float) -> dict:
+    """What sharing theta_local buffers between workers does to the compression kernel's rate.
+    (a) half the depth of the 2B config (12 layers), where R = 16 distinct buffers fit: the kernel
+        timed with 16 distinct buffers, with 8 buffers read through shifted views (the headline's
+        arrangement) and with 8 buffers read through identical views;
+    (b) the full 2B config with R = 8 workers and 8 distinct buffers (nothing shared)."""
+    from paper_2508_15706_b200.binding import SparseLoCo
+    out = {}
+
+    def build(wl):
+        shapes = [(t.rows, t.cols) for t in wl.tensors]
+        sl = SparseLoCo(shapes, I.offsets(wl.tensors), k=wl.k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr,
+                        alloc_workspace=False)
+        sl.set_ef_deferred(True)
+        ws = torch.empty(sl.workspace_bytes(), dtype=torch.uint8, device=dev)
+        sl.set_workspace(ws)
+        theta = I.theta_sync(wl, dev)
+        e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(wl.R)]
+        payloads = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(wl.R)]
+        return sl, ws, theta, e, payloads
+
+    wl = I.workload("c5_l12")
+    N = wl.numel
+    sl, ws, theta, e, payloads = build(wl)
+    bytes_launch = ef_topk_bytes_per_param(wl.R) * N
+    storage, views = make_locals(torch, I, wl, theta, wl.R, 0)
+    rows = {}
+    ms = time_compression_kernel(torch, sl, theta, views, e, payloads)
+    rows["16_distinct"] = ms
+    # the first 8 buffers again, shared: the extra tail the shifted views need comes from buffer d + 8
+    # (any fp32 content of theta's scale serves), so nothing is re-allocated
+    shift = ALIAS_SHIFT
+    shifted = None
+    try:
+        storage8, shifted = make_locals(torch, I, wl, theta, 8, shift)
+    except torch.cuda.OutOfMemoryError:
+        storage8 = None
+    if shifted is not None:
+        sl.ef_flush()
+        rows["8_shared_shifted_views"] = time_compression_kernel(torch, sl, theta, shifted, e, payloads)
+        del storage8, shifted
+    sl.ef_flush()
+    rows["8_shared_identical_views"] = time_compression_kernel(torch, sl, theta, [views[r % 8] for r in range(wl.R)],
+                                                               e, payloads)
+    out["c5_l12"] = {"params": N, "R": wl.R, "algorithmic_gb_per_launch": bytes_launch / 1e9,
+                     "ms": rows, "gbs": {k_: bytes_launch / (v * 1e-3) / 1e9 for k_, v in rows.items()},
+                     "frac_of_measured_peak": {k_: bytes_launch / (v * 1e-3) / 1e9 / peak for k_, v in rows.items()}}
+    sl.ef_flush()
+    del sl, ws, theta, e, payloads, storage, views
+    torch.cuda.empty_cache()
+
+    import dataclasses
+    wl = dataclasses.replace(I.workload(DEFAULT_WORKLOAD), R=8)
+    N = wl.numel
+    sl, ws, theta, e, payloads = build(wl)
+    storage, views = make_locals(torch, I, wl, theta, wl.R, 0)
+    ms = time_compression_kernel(torch, sl, theta, views, e, payloads)
+    b8 = ef_topk_bytes_per_param(wl.R) * N
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(torch.cuda.current_stream())
+    for _ in range(4):
+        sl.outer_step(theta, views, e, payloads)
+    sl.ef_flush()
+    t1.record(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    step_ms = t0.elapsed_time(t1) / 4
+    out["c5_dense_d2048_R8_unshared"] = {
+        "params": N, "R": 8, "distinct_theta_local_buffers": 8, "compression_kernel_ms": ms,
+        "compression_kernel_gbs": b8 / (ms * 1e-3) / 1e9, "frac_of_measured_peak": b8 / (ms * 1e-3) / 1e9 / peak,
+        "ms_per_step": step_ms, "params_per_s": N / (step_ms * 1e-3),
+        "step_gbs": algorithmic_bytes_per_param(8, wl.k) * N / (step_ms * 1e-3) / 1e9}
+    del sl, ws, theta, e, payloads, storage, views
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_e2e(torch, I, sl, wl, theta, e, payloads, flat, N, args) -> dict:
@@ -486,6 +612,12 @@ def main():
     ap.add_argument("--tile-copies", default="auto", choices=["auto", "tma", "threads"],
                     help="how the compression kernel moves 64x64 blocks: tensor-map block copies (the library's "
                          "default when the table allows) or per-thread 16-byte asynchronous copies")
+    ap.add_argument("--distinct-locals", type=int, default=0,
+                    help="distinct theta_local buffers (default: as many as fit, at most R)")
+    ap.add_argument("--alias-shift", type=int, default=ALIAS_SHIFT,
+                    help="element shift between the views of workers sharing a theta_local buffer (0: identical views)")
+    ap.add_argument("--no-alias-check", action="store_true",
+                    help="skip the measurement of what sharing theta_local buffers does to the kernel's rate")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense DiLoCo comparator line")

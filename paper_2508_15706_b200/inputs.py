@@ -108,6 +108,9 @@ def workload(name: str) -> Workload:
     if name == "c5_dense_d2048":
         return Workload(name, dense_transformer(2048, 24, 8192, 32000), R=16, k=64, H=30,
                         outer_lr=0.8, recipe="normal", seed=5)
+    if name == "c5_l12":  # half the depth of c5_dense_d2048: 16 distinct theta_local AND 16 e buffers fit one GPU
+        return Workload(name, dense_transformer(2048, 12, 8192, 32000), R=16, k=64, H=30,
+                        outer_lr=0.8, recipe="normal", seed=5)
     if name == "c5_layer0":  # one decoder layer of c5_dense_d2048: small enough to profile
         full = dense_transformer(2048, 24, 8192, 32000)
         return Workload(name, [t for t in full if t.layer == 0], R=16, k=64, H=30,
