@@ -1,4 +1,4 @@
-// Decode + average + outer update (optionally fused with the packing step).
+// Decode + average + outer update (optionally fused with the packing step), one warp per chunk.
 // Part of libsparseloco (one translation unit: included by sparseloco.cu).
 #pragma once
 #include "common.cuh"
@@ -7,239 +7,247 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------------
-// Decode + average + outer update.  One CTA per chunk.  Every (worker, slot) entry of the chunk is
-// decoded by its own thread and ORs its worker's bit into a per-position mask in shared memory.
-// The mask gives the entry its rank among the workers that selected the same position (bits
-// below its own), and the entries are added into a 4096-float shared tile in rounds: rank 0
-// first, then rank 1, ... with a barrier in between.  Every position thus receives its values in
-// ascending worker order (reproducible bits), one writer per position and round, and the number
-// of rounds is the largest number of workers that meet at one position (3 or 4 at R = 16).  Then
-// every thread applies theta = fma(-alpha/D, sum, theta) to its own 16 positions.
-// Workers are taken in batches of at most 32 (one mask bit each, 8 entries per thread).
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned get12(const unsigned* rec, int s) {
-    const int bit = 12 * s;
-    return __funnelshift_r(rec[bit >> 5], rec[(bit >> 5) + 1], bit & 31) & 0xFFFu;
-}
-__device__ __forceinline__ unsigned get2(const unsigned* rec, int code_byte0, int s) {
-    const int bit = code_byte0 * 8 + 2 * s;
-    return (rec[bit >> 5] >> (bit & 31)) & 3u;
-}
-
-constexpr int kApplyEntries = 8;  // most entries per thread and batch
-
+// Decode + average + outer update (Eq. 2 lines 3-4).  Persistent CTAs of four warps, eight per SM;
+// a CTA takes whole chunks (b, b + grid, ...) and owns a 4096-float sum tile in shared memory.  For a
+// chunk it
+//   1. starts the loads of the chunk's theta (8 x 128 bits per thread, in registers until step 4),
+//   2. decodes the workers in batches of 16, warp w the workers 4 w .. 4 w + 3 of the batch: a lane holds
+//      the slot pairs (2 m, 2 m + 1), m = lane + 32 j, of a worker and turns them into (index, table value),
+//   3. adds them into the tile in ascending worker order: the warps take turns (a CTA barrier between
+//      two warps, a warp barrier between two workers of a warp).  A worker's indices are distinct, so
+//      every position receives its values in worker order (reproducible bits) without atomics,
+//   4. applies theta = fma(-alpha/D, sum, theta) to its 32 positions, clears the tile on the way and
+//      stores the vectors that received anything.
+//
 // FUSE 0: the entries come from the payload records (sl_aggregate_apply).  FUSE 1 / 2: the whole outer
 // step is running and the records do not exist yet: the entries come from the staging arrays, get
-// their codes here, and the kernel also writes the records and the error correction, i.e. it does
-// what pack_fix_kernel<1> / <2> does, saving that kernel's pass and the re-read of the records.
+// their codes here, and the kernel also writes the records and the error correction (e[index] =
+// value - table[code] for FUSE 1; the same value back into the staging array for FUSE 2, the deferred
+// form), i.e. it does what pack_fix_kernel<1> / <2> does, saving that kernel's pass.
+//
+// A slot pair is 24 bits of the index block (bytes 3 m .. 3 m + 2) and one nibble of the code block, so
+// a lane assembles its part of a record with byte stores into the CTA's record buffer and the finished
+// records leave as 16-byte vectors.
+// ------------------------------------------------------------------------------------------------
 struct FuseArgs {
     Workspace ws;
     long long n_chunks;
     int n_tensors, kp;
 };
 
-// SPL = slots per lane: ceil(k / 32) rounded up to 1, 2, 4 or 8; WPW = workers per warp and batch (1, 2 or
-// 4, SPL * WPW <= 8): a thread holds SPL * WPW entries and a batch is 8 * WPW workers
-template <int SPL, int WPW, int FUSE>
-__global__ void __launch_bounds__(kThreads, 4)
-decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale,
+constexpr int kApplyWarps = 4;
+constexpr int kApplyThreads = 32 * kApplyWarps;
+constexpr int kApplyCtasPerSm = 8;
+constexpr int kApplyBatch = 16;                  // workers decoded between two rounds of ordered additions
+constexpr int kApplyPerWarp = kApplyBatch / kApplyWarps;
+constexpr int kApplyTile = kChunk + kApplyThreads;  // the sum tile + one dump slot per thread for entries that do not count
+
+__host__ __device__ constexpr size_t apply_smem_bytes(int k) {
+    return (size_t)kApplyTile * sizeof(float) + (size_t)kApplyBatch * (record_stride(k) + 32);
+}
+
+// PPL = slot pairs per lane: ceil(k / 64) rounded up to 1, 2 or 4
+template <int PPL, int FUSE>
+__global__ void __launch_bounds__(kApplyThreads, kApplyCtasPerSm)
+decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, float scale,
                         PayloadPtrs pl, float* __restrict__ theta_sync, FuseArgs fa, WorkerPtrs ptrs) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    float* acc = reinterpret_cast<float*>(dyn);                            // 4096 sums
-    unsigned* wmask = reinterpret_cast<unsigned*>(acc + kChunk);           // 4096 worker masks
-    float* luts = reinterpret_cast<float*>(wmask + kChunk);                // 32 x 4
-    float* mu_t3 = luts + 4 * 32;                                          // 32 x 2 (FUSE: mean, 3 sigma)
-    unsigned* recs = reinterpret_cast<unsigned*>(mu_t3 + 2 * 32);          // batch x (stride + 16) bytes
-    const int stride = record_stride(k), rwords = stride / 4 + 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int kEnt = SPL * WPW;  // entries per thread and batch
-    static_assert(kEnt <= kApplyEntries && WPW <= 4, "entry budget");
-    constexpr int batch = 8 * WPW;
-    // FUSE: the staged (index, value) pairs of this thread's entries in the first batch.  They need
-    // nothing from the chunk table (slots up to k exist for every chunk; those beyond the chunk's
-    // own count are ignored later), so they start before anything else.
-    unsigned pre_p[kEnt];
-    float pre_v[kEnt];
+    const int stride = record_stride(k), ib = record_index_bytes(k);
+    float* acc = reinterpret_cast<float*>(dyn);
+    uint8_t* recs = dyn + (size_t)kApplyTile * sizeof(float);
+    // per worker of the batch: mean, 3 sigma, 0, present | the four table entries
+    float4* tabs = reinterpret_cast<float4*>(recs + (size_t)kApplyBatch * stride);
+    constexpr int WB = kApplyPerWarp;
+    const unsigned dump = (unsigned)(kChunk + tid);  // where an entry that does not count adds its 0
+    // per-worker strides of the staging arrays, in index pairs / value pairs (kp is a multiple of 8)
+    const long long wstride = FUSE ? fa.n_chunks * (long long)fa.kp / 2 : 0;
+
+    for (int i = tid; i < kApplyTile / 4; i += kApplyThreads) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+
+    for (long long g = blockIdx.x; g < n_chunks; g += gridDim.x) {
+        const ChunkDesc cd = chunks[g];
+        const int keff = min(k, cd.len);
+        const bool full = cd.len == kChunk;
+        const int rs = cd.row_stride ? cd.row_stride : kTile;
+        float* __restrict__ th = theta_sync + cd.base;
+        // thread t owns in-chunk indices 512 i + 4 t + j: block row 8 i + t / 16, column 4 (t % 16)
+        float* __restrict__ th_vec = th + (long long)(tid >> 4) * rs + 4 * (tid & 15);
+        const long long vec_step = 8ll * rs;
+        float4 a[8];
+        if (full) {
 #pragma unroll
-    for (int e = 0; e < kEnt; ++e) {
-        pre_p[e] = 0u;
-        pre_v[e] = 0.f;
-    }
-    if (FUSE) {
+            for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(th_vec + i * vec_step);
+        }
+        // which of this lane's slots exist in this chunk (the same for every worker)
+        bool in0[PPL], in1[PPL];
 #pragma unroll
-        for (int wi = 0; wi < WPW; ++wi) {
-            const int rb = warp + 8 * wi;
-            const long long slot_base = ((long long)rb * fa.n_chunks + blockIdx.x) * fa.kp;
+        for (int j = 0; j < PPL; ++j) {
+            const int m = lane + 32 * j;
+            in0[j] = 2 * m < keff;
+            in1[j] = 2 * m + 1 < keff;
+        }
+        const unsigned* idx_pairs = FUSE ? reinterpret_cast<const unsigned*>(fa.ws.idx + g * fa.kp) : nullptr;
+        float2* val_pairs = FUSE ? reinterpret_cast<float2*>(fa.ws.val + g * fa.kp) : nullptr;
+        const TStat* tstat = FUSE ? fa.ws.tstat + cd.tensor : nullptr;
+
+        for (int r0 = 0; r0 < n_workers; r0 += kApplyBatch) {
+            const int nb = min(kApplyBatch, n_workers - r0);
+            if (FUSE) {  // the records of this batch start as zeros (unused slots and padding stay zero)
+                for (int v = tid; v < nb * (stride / 16); v += kApplyThreads) reinterpret_cast<uint4*>(recs)[v] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            if (tid < kApplyBatch) {  // what decodes worker r0 + tid: one load per thread, read back by all below
+                float4 h = make_float4(0.f, 0.f, 0.f, 0.f), t = h;
+                if (tid < nb) {
+                    const int r = r0 + tid;
+                    if (FUSE) {
+                        const float4* st = reinterpret_cast<const float4*>(tstat + (long long)r * fa.n_tensors);
+                        const float4 s0 = st[0], s1 = st[1];  // mu, sigma, 3 sigma, table[0] | table[1..3], pad
+                        h = make_float4(s0.x, s0.z, 0.f, 1.f);
+                        t = make_float4(s0.w, s1.x, s1.y, s1.z);
+                    } else if (pl.p[r]) {
+                        h.w = 1.f;
+                        t = __ldg(reinterpret_cast<const float4*>(pl.p[r] + 16ll * cd.tensor));
+                    }
+                }
+                tabs[2 * tid] = h;
+                tabs[2 * tid + 1] = t;
+            }
+            // ---- A. this warp's workers of the batch (any order): pos = index pair, val = value pair / codes
+            const int w0 = WB * warp;
+            unsigned pos[WB][PPL];
+            float2 val[WB][PPL];
 #pragma unroll
-            for (int si = 0; si < SPL; ++si) {
-                const int sl = lane + 32 * si;
-                if (rb < n_workers && sl < k) {
-                    pre_p[wi * SPL + si] = fa.ws.idx[slot_base + sl];
-                    pre_v[wi * SPL + si] = fa.ws.val[slot_base + sl];
+            for (int q = 0; q < WB; ++q) {
+                const int r = r0 + w0 + q;
+#pragma unroll
+                for (int j = 0; j < PPL; ++j) {
+                    const int m = lane + 32 * j;
+                    pos[q][j] = 0u;
+                    val[q][j] = make_float2(0.f, 0.f);
+                    if (w0 + q < nb && in0[j]) {
+                        if (FUSE) {
+                            pos[q][j] = idx_pairs[r * wstride + m];
+                            val[q][j] = val_pairs[r * wstride + m];
+                        } else if (pl.p[r]) {
+                            // 24 bits at byte 3 m of the record, from the aligned words around it (the second
+                            // word may belong to the code block or the padding: inside the record either way)
+                            const uint8_t* rec = pl.p[r] + cd.rec_off;
+                            const int w = (3 * m) >> 2, sh = ((3 * m) & 3) * 8;
+                            const unsigned lo = __ldg(reinterpret_cast<const unsigned*>(rec) + w);
+                            const unsigned hi = sh > 8 ? __ldg(reinterpret_cast<const unsigned*>(rec) + w + 1) : 0u;
+                            const unsigned x = __funnelshift_r(lo, hi, sh) & 0xFFFFFFu;
+                            const unsigned nib = (__ldg(rec + ib + (m >> 1)) >> ((m & 1) * 4)) & 0xFu;
+                            pos[q][j] = (x & 0xFFFu) | ((x >> 12) << 16);
+                            val[q][j] = make_float2(__uint_as_float(nib & 3u), __uint_as_float(nib >> 2));  // the codes
+                        }
+                    }
+                }
+            }
+            __syncthreads();  // tables and zeroed records are in place
+#pragma unroll
+            for (int q = 0; q < WB; ++q) {
+                const int r = r0 + w0 + q;
+                const float4 hd = tabs[2 * (w0 + q)], lut = tabs[2 * (w0 + q) + 1];
+                const bool have = hd.w != 0.f;  // false beyond the batch and for an absent worker
+                const float mu = hd.x, t3 = hd.y;
+                uint8_t* rec = recs + (size_t)(w0 + q) * stride;
+#pragma unroll
+                for (int j = 0; j < PPL; ++j) {
+                    const int m = lane + 32 * j;
+                    unsigned p0 = pos[q][j] & 0xFFFFu, p1 = pos[q][j] >> 16;
+                    const bool ok0 = have && in0[j], ok1 = have && in1[j];
+                    unsigned c0, c1;
+                    if (FUSE) {
+                        c0 = (unsigned)quant_code(val[q][j].x, mu, t3);
+                        c1 = (unsigned)quant_code(val[q][j].y, mu, t3);
+                    } else {
+                        c0 = __float_as_uint(val[q][j].x);
+                        c1 = __float_as_uint(val[q][j].y);
+                    }
+                    const float l0 = c0 == 0 ? lut.x : c0 == 1 ? lut.y : c0 == 2 ? lut.z : lut.w;
+                    const float l1 = c1 == 0 ? lut.x : c1 == 1 ? lut.y : c1 == 2 ? lut.z : lut.w;
+                    if (FUSE) {
+                        const float f0 = __fsub_rn(val[q][j].x, l0), f1 = __fsub_rn(val[q][j].y, l1);
+                        if (FUSE == 1) {
+                            if (ok0 && p0 < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p0)] = f0;
+                            if (ok1 && p1 < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p1)] = f1;
+                        } else if (ok0) {
+                            // (slot 2 m + 1 exists in the array even when it is beyond keff: kp is even)
+                            val_pairs[r * wstride + m] = make_float2(f0, f1);
+                        }
+                        // this lane's three bytes of the index block and its nibble of the code block
+                        const unsigned x = (ok0 ? p0 : 0u) | ((ok1 ? p1 : 0u) << 12);
+                        const unsigned nib = (ok0 ? c0 : 0u) | ((ok1 ? c1 : 0u) << 2);
+                        const unsigned other = __shfl_xor_sync(kFull, nib, 1);
+                        if (ok0) {
+#pragma unroll
+                            for (int bb = 0; bb < 3; ++bb)
+                                if (3 * m + bb < ib) rec[3 * m + bb] = (uint8_t)(x >> (8 * bb));
+                            if (!(lane & 1)) rec[ib + (m >> 1)] = (uint8_t)(nib | (other << 4));
+                        }
+                    }
+                    // what step B adds where: entries that do not count add 0 to the thread's dump slot
+                    const bool use0 = ok0 && p0 < (unsigned)cd.len, use1 = ok1 && p1 < (unsigned)cd.len;
+                    p0 = use0 ? p0 : dump;
+                    p1 = use1 ? p1 : dump;
+                    pos[q][j] = p0 | (p1 << 16);
+                    val[q][j] = make_float2(use0 ? l0 : 0.0f, use1 ? l1 : 0.0f);
+                }
+            }
+            // ---- B. ascending worker order: the warps take turns, a warp's workers go one after the other
+            // (a worker's positions are distinct; the barriers separate workers)
+            for (int turn = 0; turn * WB < nb; ++turn) {
+                if (warp == turn) {
+#pragma unroll
+                    for (int q = 0; q < WB; ++q) {
+#pragma unroll
+                        for (int j = 0; j < PPL; ++j) {
+                            const unsigned p0 = pos[q][j] & 0xFFFFu, p1 = pos[q][j] >> 16;
+                            acc[p0] = __fadd_rn(acc[p0], val[q][j].x);
+                            acc[p1] = __fadd_rn(acc[p1], val[q][j].y);
+                        }
+                        __syncwarp();
+                    }
+                }
+                __syncthreads();
+            }
+            if (FUSE) {  // the records of the batch are complete (written before the barriers above): out they go
+                const int vpr = stride / 16;
+                for (int v = tid; v < nb * vpr; v += kApplyThreads) {
+                    const int rb = v / vpr, w = v - rb * vpr;
+                    reinterpret_cast<uint4*>(ptrs.payload[r0 + rb] + cd.rec_off)[w] = reinterpret_cast<const uint4*>(recs)[v];
                 }
             }
         }
-    }
-    const ChunkDesc cd = chunks[blockIdx.x];
-    const int keff = min(k, cd.len);
-    const int code_byte0 = record_index_bytes(k);
-    float* __restrict__ th = theta_sync + cd.base;
 
-    // theta loads first (in flight while the records are decoded);
-    // vector i of this thread (in-chunk indices 1024 i + 4 tid ..+3) sits at th_vec + i * vec_step
-    float4 a[4];
-    const int rs = cd.row_stride ? cd.row_stride : kTile;
-    float* __restrict__ th_vec = th + (long long)(tid >> 4) * rs + (4 * tid & 63);
-    const long long vec_step = 16ll * rs;
-    const bool full = cd.len == kChunk;
-    if (full) {
+        if (full) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(th_vec + i * vec_step);
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(acc + 1024 * i + 4 * tid) = make_float4(0.f, 0.f, 0.f, 0.f);
-
-    // entry e of a thread: worker warp + 8 (e / SPL), slot lane + 32 (e % SPL)
-    const int vec_per_rec = stride / 16;
-
-    for (int r0 = 0; r0 < n_workers; r0 += batch) {
-        const int nb = min(batch, n_workers - r0);
-        // clear the masks, stage this batch's records and tables (the last barrier of the
-        // previous batch's rounds has released both)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(wmask + 1024 * i + 4 * tid) = make_uint4(0u, 0u, 0u, 0u);
-        if (FUSE == 0) {
-            for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
-                const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
-                const uint8_t* src = pl.p[r0 + rb];
-                if (src) {
-                    const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + cd.rec_off) + w);
-                    *reinterpret_cast<uint4*>(recs + rb * rwords + 4 * w) = x;
+            for (int i = 0; i < 8; ++i) {
+                float* av = acc + 512 * i + 4 * tid;
+                const float4 sv = *reinterpret_cast<const float4*>(av);
+                // a vector that received nothing keeps its bits; with scale < 0 so does one whose sums are
+                // all +0 (fma(scale, +0, x) = x + -0 = x), and neither needs its store
+                const bool untouched = scale < 0.0f && (__float_as_uint(sv.x) | __float_as_uint(sv.y) |
+                                                        __float_as_uint(sv.z) | __float_as_uint(sv.w)) == 0u;
+                if (!untouched) {
+                    float4 o;
+                    o.x = __fmaf_rn(scale, sv.x, a[i].x);
+                    o.y = __fmaf_rn(scale, sv.y, a[i].y);
+                    o.z = __fmaf_rn(scale, sv.z, a[i].z);
+                    o.w = __fmaf_rn(scale, sv.w, a[i].w);
+                    *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
+                    *reinterpret_cast<float4*>(av) = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-            }
-            if (tid < nb) {
-                const uint8_t* src = pl.p[r0 + tid];
-                if (src) *reinterpret_cast<float4*>(luts + 4 * tid) = __ldg(reinterpret_cast<const float4*>(src + 16ll * cd.tensor));
-                recs[tid * rwords + stride / 4] = 0;  // word read past the index block by get12
             }
         } else {
-            // staged pairs of the later batches (the first batch's are already on their way)
-#pragma unroll
-            for (int wi = 0; wi < WPW; ++wi) {
-                const int rb = warp + 8 * wi;
-                const long long slot_base = ((long long)(r0 + rb) * fa.n_chunks + blockIdx.x) * fa.kp;
-#pragma unroll
-                for (int si = 0; si < SPL; ++si) {
-                    const int sl = lane + 32 * si;
-                    if (r0 > 0 && rb < nb && sl < keff) {
-                        pre_p[wi * SPL + si] = fa.ws.idx[slot_base + sl];
-                        pre_v[wi * SPL + si] = fa.ws.val[slot_base + sl];
-                    }
-                }
-            }
-            for (int w = tid; w < nb * rwords; w += kThreads) recs[w] = 0;  // the records are assembled here
-            if (tid < nb) {
-                const TStat st = fa.ws.tstat[(long long)(r0 + tid) * fa.n_tensors + cd.tensor];
-                *reinterpret_cast<float4*>(luts + 4 * tid) = make_float4(st.lut[0], st.lut[1], st.lut[2], st.lut[3]);
-                mu_t3[2 * tid] = st.mu;
-                mu_t3[2 * tid + 1] = st.t3;
+            for (int p = tid; p < cd.len; p += kApplyThreads) {  // (nothing was added at or beyond the chunk's length)
+                th[p] = __fmaf_rn(scale, acc[p], th[p]);
+                acc[p] = 0.0f;
             }
         }
-        __syncthreads();
-
-        unsigned ent_p[kEnt];  // position | worker bit number << 12; 0xFFFFFFFF = no entry
-        float ent_v[kEnt];
-#pragma unroll
-        for (int e = 0; e < kEnt; ++e) {
-            ent_p[e] = 0xFFFFFFFFu;
-            ent_v[e] = 0.f;
-        }
-#pragma unroll
-        for (int wi = 0; wi < WPW; ++wi) {
-            const int rb = warp + 8 * wi;
-            if (rb < nb && pl.p[r0 + rb]) {  // uniform over the warp
-                unsigned* rec = recs + rb * rwords;
-                const long long slot_base = FUSE ? ((long long)(r0 + rb) * fa.n_chunks + blockIdx.x) * fa.kp : 0;
-#pragma unroll
-                for (int si = 0; si < SPL; ++si) {
-                    const int sl = lane + 32 * si;
-                    if (sl < keff) {
-                        unsigned p, code;
-                        if (FUSE == 0) {
-                            p = get12(rec, sl);
-                            code = get2(rec, code_byte0, sl);
-                        } else {
-                            p = pre_p[wi * SPL + si];
-                            const float v = pre_v[wi * SPL + si];
-                            code = (unsigned)quant_code(v, mu_t3[2 * rb], mu_t3[2 * rb + 1]);
-                            const int bit = 12 * sl;
-                            atomicOr(&rec[bit >> 5], p << (bit & 31));
-                            if ((bit & 31) > 20) atomicOr(&rec[(bit >> 5) + 1], p >> (32 - (bit & 31)));
-                            const int cbit = code_byte0 * 8 + 2 * sl;
-                            atomicOr(&rec[cbit >> 5], code << (cbit & 31));
-                            const float fixed = __fsub_rn(v, luts[4 * rb + code]);
-                            if (FUSE == 1 && p < (unsigned)cd.len)
-                                ptrs.e[r0 + rb][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = fixed;
-                            if (FUSE == 2) fa.ws.val[slot_base + sl] = fixed;
-                        }
-                        if (p < (unsigned)cd.len) {
-                            ent_v[wi * SPL + si] = luts[4 * rb + code];
-                            ent_p[wi * SPL + si] = p | ((unsigned)rb << 12);
-                            atomicOr(&wmask[p], 1u << rb);
-                        }
-                    }
-                }
-            }
-        }
-        __syncthreads();
-        if (FUSE) {  // the records are complete: out they go
-            for (int v = tid; v < nb * vec_per_rec; v += kThreads) {
-                const int rb = v / vec_per_rec, w = v - rb * vec_per_rec;
-                reinterpret_cast<uint4*>(ptrs.payload[r0 + rb] + cd.rec_off)[w] =
-                    *reinterpret_cast<const uint4*>(recs + rb * rwords + 4 * w);
-            }
-        }
-        // rank of every entry among the workers at its position; round 0
-        int my_max = 0;
-#pragma unroll
-        for (int e = 0; e < kEnt; ++e) {
-            if (ent_p[e] != 0xFFFFFFFFu) {
-                const unsigned p = ent_p[e] & 0xFFFu, rb = ent_p[e] >> 12;
-                const unsigned wm = wmask[p];
-                const int rank = __popc(wm & ((1u << rb) - 1u));
-                my_max = max(my_max, __popc(wm));
-                if (rank == 0) {
-                    acc[p] = __fadd_rn(acc[p], ent_v[e]);
-                    ent_p[e] = 0xFFFFFFFFu;
-                } else {
-                    ent_p[e] = p | ((unsigned)rank << 12);  // from here on: position | rank << 12
-                }
-            }
-        }
-        for (int t = 1; __syncthreads_or(my_max > t); ++t) {
-#pragma unroll
-            for (int e = 0; e < kEnt; ++e) {
-                if (ent_p[e] != 0xFFFFFFFFu && (int)(ent_p[e] >> 12) == t) {
-                    const unsigned p = ent_p[e] & 0xFFFu;
-                    acc[p] = __fadd_rn(acc[p], ent_v[e]);
-                }
-            }
-        }
-    }
-
-    if (full) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 sv = *reinterpret_cast<const float4*>(acc + 1024 * i + 4 * tid);
-            float4 o;
-            o.x = __fmaf_rn(scale, sv.x, a[i].x);
-            o.y = __fmaf_rn(scale, sv.y, a[i].y);
-            o.z = __fmaf_rn(scale, sv.z, a[i].z);
-            o.w = __fmaf_rn(scale, sv.w, a[i].w);
-            *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
-        }
-    } else {
-        for (int p = tid; p < cd.len; p += kThreads) th[p] = __fmaf_rn(scale, acc[p], th[p]);
+        // (the next chunk's first additions come after several CTA barriers: the cleared tile is seen by all)
     }
 }
 

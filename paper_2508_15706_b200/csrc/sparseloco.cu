@@ -319,10 +319,8 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const int R = c->cfg.R;
     const double D = c->cfg.divide_by_present ? (double)present : (double)R;
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
-    const int stride = record_stride(c->cfg.k);
-    const int nb = R < 32 ? R : 32;  // the kernel never stages more than 32 records at once
-    const size_t smem = (size_t)kChunk * 8 + 32 * 24 + (size_t)nb * (stride + 16);
-    const int spl = (c->cfg.k + 31) / 32;
+    const size_t smem = apply_smem_bytes(c->cfg.k);
+    const int ppl = (c->cfg.k + 63) / 64;
     FuseArgs fa;
     memset(&fa, 0, sizeof(fa));
     WorkerPtrs wp;
@@ -334,27 +332,19 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
         fa.kp = c->kp;
         wp = *fuse_ptrs;
     }
-#define SL_APPLY2(SPLV, WPWV)                                                                                   \
+    // persistent CTAs: as many as are resident at once
+    const long long resident = (long long)c->n_sms * kApplyCtasPerSm;
+    const unsigned grid = (unsigned)(c->n_chunks < resident ? c->n_chunks : resident);
+#define SL_APPLY(PPLV)                                                                                          \
     do {                                                                                                        \
-        auto kern = fuse == 0 ? decode_avg_apply_kernel<SPLV, WPWV, 0>                                          \
-                  : fuse == 1 ? decode_avg_apply_kernel<SPLV, WPWV, 1> : decode_avg_apply_kernel<SPLV, WPWV, 2>; \
-        if (smem > 48 * 1024)                                                                                   \
-            SL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
-        kern<<<(unsigned)c->n_chunks, kThreads, smem, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
+        auto kern = fuse == 0 ? decode_avg_apply_kernel<PPLV, 0>                                                \
+                  : fuse == 1 ? decode_avg_apply_kernel<PPLV, 1> : decode_avg_apply_kernel<PPLV, 2>;            \
+        kern<<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
     } while (0)
-    // workers per warp: as few as cover min(R, 32) workers in one batch, within 8 entries per thread
-#define SL_APPLY(SPLV, MAXW)                                             \
-    do {                                                                 \
-        if (R <= 8 || MAXW == 1) SL_APPLY2(SPLV, 1);                      \
-        else if (R <= 16 || MAXW == 2) SL_APPLY2(SPLV, (MAXW >= 2 ? 2 : 1)); \
-        else SL_APPLY2(SPLV, (MAXW >= 4 ? 4 : MAXW));                     \
-    } while (0)
-    if (spl <= 1) SL_APPLY(1, 4);
-    else if (spl <= 2) SL_APPLY(2, 4);
-    else if (spl <= 4) SL_APPLY(4, 2);
-    else SL_APPLY(8, 1);
+    if (ppl <= 1) SL_APPLY(1);
+    else if (ppl <= 2) SL_APPLY(2);
+    else SL_APPLY(4);
 #undef SL_APPLY
-#undef SL_APPLY2
     prof_mark(c, 8, st);
     if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
     SL_CUDA(cudaGetLastError());
@@ -521,6 +511,16 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(ef_select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
     per_sm = 1;
+    {   // the apply kernel's shared memory depends on k alone: sized once
+        const int asz = (int)apply_smem_bytes(cfg->k);
+#define SL_APPLY_ATTR(PPLV, FUSEV)                                                                                     \
+    if (e == cudaSuccess)                                                                                              \
+        e = cudaFuncSetAttribute(decode_avg_apply_kernel<PPLV, FUSEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, asz)
+        SL_APPLY_ATTR(1, 0); SL_APPLY_ATTR(1, 1); SL_APPLY_ATTR(1, 2);
+        SL_APPLY_ATTR(2, 0); SL_APPLY_ATTR(2, 1); SL_APPLY_ATTR(2, 2);
+        SL_APPLY_ATTR(4, 0); SL_APPLY_ATTR(4, 1); SL_APPLY_ATTR(4, 2);
+#undef SL_APPLY_ATTR
+    }
     c->n_sms = n_sms;
     c->ef_ctas = n_sms * (per_sm > 0 ? per_sm : 1);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int));
