@@ -51,7 +51,7 @@ typedef enum {
     SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, bits != 2, ...) */
     SL_ERR_BAD_PAYLOAD = 4, /* reported through the device status word of sl_validate_payload */
     SL_ERR_CUDA = 5,        /* a CUDA runtime call failed; see sl_last_cuda_error() */
-    SL_ERR_NOMEM = 6,       /* workspace missing or too small */
+    SL_ERR_NOMEM = 6,       /* workspace missing or too small; host allocation failed */
     SL_ERR_TOO_LARGE = 7,   /* problem exceeds a fixed built-in capacity */
     SL_ERR_TIMEOUT = 8      /* a bounded wait inside a kernel ran out; reported by sl_device_status() */
 } sl_status;
@@ -82,7 +82,9 @@ typedef struct sl_ctx sl_ctx;
 
 /* Build a context for a tensor table on the current CUDA device.  Allocates the device chunk
  * table (32 bytes per chunk) -- the only allocation the library ever makes -- and synchronises.
- * `tensors` is a host array.  Errors: INVALID_ARG, ALIGNMENT (offset % 4), UNSUPPORTED, CUDA. */
+ * `tensors` is a host array; the element ranges [offset, offset + rows * cols) must not overlap.
+ * Errors: INVALID_ARG (also overlapping tensors), ALIGNMENT (offset % 4), UNSUPPORTED, TOO_LARGE
+ * (cols >= 2^31, a tensor of more than 2^40 elements), NOMEM (host allocation failed), CUDA. */
 sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t n_tensors,
                     sl_ctx** out);
 sl_status sl_destroy(sl_ctx* ctx);

@@ -26,8 +26,10 @@
 #include <stdio.h>
 #include <string.h>
 
-#include <new>
+#include <algorithm>
 #include <mutex>
+#include <new>
+#include <utility>
 #include <vector>
 
 #include "sparseloco.h"
@@ -395,8 +397,20 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile || cfg->quant_bits != 2) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
 
+    {   // element ranges: no overflow, no two tensors sharing an element (kernels of different chunks would race)
+        std::vector<std::pair<long long, long long>> span((size_t)n_tensors);
+        for (int j = 0; j < n_tensors; ++j) {
+            const sl_tensor_desc& t = tensors[j];
+            if (t.rows < 1 || t.cols < 1 || t.offset < 0) return SL_ERR_INVALID_ARG;
+            if (t.cols > 0x7FFFFFFFll || t.rows > (1ll << 40) / t.cols || t.offset > (1ll << 46)) return SL_ERR_TOO_LARGE;
+            span[(size_t)j] = {(long long)t.offset, (long long)t.offset + t.rows * t.cols};
+        }
+        std::sort(span.begin(), span.end());
+        for (int j = 1; j < n_tensors; ++j)
+            if (span[(size_t)j].first < span[(size_t)j - 1].second) return SL_ERR_INVALID_ARG;
+    }
     sl_ctx* c = new (std::nothrow) sl_ctx();
-    if (!c) return SL_ERR_INVALID_ARG;
+    if (!c) return SL_ERR_NOMEM;
     c->cfg = *cfg;
     c->n_tensors = n_tensors;
     c->kp = (cfg->k + 7) / 8 * 8;

@@ -25,12 +25,34 @@ def oracle_threads() -> int:
     return n
 
 
+GUARD_BYTES = 4096   # on either side of every buffer the kernels write
+CANARY = 0xC5
+
+
+class Guarded:
+    """A device buffer with a band of known bytes before and after it.  The kernels get the middle;
+    `intact()` tells whether anything wrote outside it (the stand-in for a memory checker)."""
+
+    def __init__(self, numel: int, dtype, device, extra_bytes: int = 0):
+        item = torch.empty((), dtype=dtype).element_size()
+        self.n_bytes = numel * item
+        total = GUARD_BYTES + (self.n_bytes + extra_bytes + 255) // 256 * 256 + GUARD_BYTES
+        self.raw = torch.full((total,), CANARY, dtype=torch.uint8, device=device)
+        self.view = self.raw[GUARD_BYTES:GUARD_BYTES + self.n_bytes].view(dtype)
+        self.tail_from = GUARD_BYTES + self.n_bytes + extra_bytes
+
+    def intact(self) -> bool:
+        return bool((self.raw[:GUARD_BYTES] == CANARY).all()) and bool((self.raw[self.tail_from:] == CANARY).all())
+
+
 class DeviceCase:
     """Device-resident buffers of one workload: theta_sync, D distinct theta_local buffers
-    (worker r reads buffer r % D), R error buffers, R payloads."""
+    (worker r reads buffer r % D, through a view shifted by (r // D) * alias_shift elements, as
+    bench.py arranges them), R error buffers, R payloads, the workspace.  Everything the kernels
+    write sits between guard bands, which check() and step() verify."""
 
     def __init__(self, wl: I.Workload, k: Optional[int] = None, distinct_local: Optional[int] = None,
-                 e_scale: float = 0.0, device=None):
+                 e_scale: float = 0.0, device=None, alias_shift: int = 0):
         from paper_2508_15706_b200.binding import SparseLoCo
         self.wl = wl
         self.k = wl.k if k is None else k
@@ -38,13 +60,40 @@ class DeviceCase:
         self.offs = I.offsets(wl.tensors)
         self.shapes = [(t.rows, t.cols) for t in wl.tensors]
         self.D = wl.R if distinct_local is None else distinct_local
+        self.alias_shift = alias_shift if self.D < wl.R else 0
         self.sl = SparseLoCo(self.shapes, self.offs, k=self.k, R=wl.R, H=wl.H, beta=wl.beta,
-                             outer_lr=wl.outer_lr)
-        self.theta = I.theta_sync(wl, self.dev)
-        self.local = [torch.empty_like(self.theta) for _ in range(self.D)]
-        self.e = [I.initial_error(wl, r, self.dev, scale=e_scale) for r in range(wl.R)]
-        self.payloads = [torch.zeros(self.sl.payload_bytes(), dtype=torch.uint8, device=self.dev)
-                         for _ in range(wl.R)]
+                             outer_lr=wl.outer_lr, alloc_workspace=False)
+        flat = I.flat_numel(wl.tensors)
+        self.flat = flat
+        self.guarded: List[Guarded] = []
+
+        def guarded(numel, dtype):
+            g = Guarded(numel, dtype, self.dev)
+            self.guarded.append(g)
+            return g.view
+
+        self.theta = guarded(flat, torch.float32)
+        self.theta.zero_()
+        I.theta_sync(wl, self.dev, out=self.theta)
+        extra = self.alias_shift * ((wl.R + self.D - 1) // self.D - 1)
+        self.local = [torch.empty(flat + extra, dtype=torch.float32, device=self.dev) for _ in range(self.D)]
+        if extra:
+            for d, buf in enumerate(self.local):
+                g = torch.Generator(device=self.dev).manual_seed(77_000 + d)
+                buf[flat:].normal_(0.0, 0.02, generator=g)
+        self.e = []
+        for r in range(wl.R):
+            buf = guarded(flat, torch.float32)
+            buf.zero_()
+            I.initial_error(wl, r, self.dev, scale=e_scale, out=buf)
+            self.e.append(buf)
+        self.payloads = []
+        for _ in range(wl.R):
+            buf = guarded(self.sl.payload_bytes(), torch.uint8)
+            buf.zero_()
+            self.payloads.append(buf)
+        self.ws = guarded(self.sl.workspace_bytes(), torch.uint8)
+        self.sl.set_workspace(self.ws)
         self.cfg = O.Config(k=self.k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr)
         # payload geometry, from the oracle's definitions
         self.rec_off, self.n_chunks = [], []
@@ -63,25 +112,31 @@ class DeviceCase:
             I.theta_local(self.wl, self.theta, d, step, out=self.local[d])
 
     def local_of(self, r: int) -> torch.Tensor:
-        return self.local[r % self.D]
+        o = (r // self.D) * self.alias_shift
+        return self.local[r % self.D][o:o + self.flat]
 
-    def snapshot(self, tensor_ids: Sequence[int]) -> Dict[int, dict]:
+    def guards_intact(self) -> bool:
+        return all(g.intact() for g in self.guarded)
+
+    def snapshot(self, tensor_ids: Sequence[int], spare: Optional[torch.Tensor] = None) -> Dict[int, dict]:
         """CPU copies of theta_sync / theta_local / e slices of the given tensors (pre-step)."""
         snap = {}
-        e_cpu = self.error_slices(tensor_ids)
-        for j in tensor_ids:
+        for j in tensor_ids:  # parameters first: `spare` may be one of the theta_local buffers
             t, off = self.wl.tensors[j], self.offs[j]
             sl = slice(off, off + t.numel)
             snap[j] = {
                 "theta": self.theta[sl].cpu().numpy().copy(),
                 "local": [self.local_of(r)[sl].cpu().numpy().copy() for r in range(self.wl.R)],
-                "e": [e_cpu[r][j] for r in range(self.wl.R)],
             }
+        e_cpu = self.error_slices(tensor_ids, spare=spare)
+        for j in tensor_ids:
+            snap[j]["e"] = [e_cpu[r][j] for r in range(self.wl.R)]
         return snap
 
     def step(self) -> None:
         self.sl.outer_step(self.theta, [self.local_of(r) for r in range(self.wl.R)], self.e, self.payloads)
         assert self.sl.device_status() == 0, "a kernel recorded a device-side error"
+        assert self.guards_intact(), "a kernel wrote outside one of its output buffers"
 
     def tensor_payload(self, r: int, j: int) -> np.ndarray:
         p = self.payloads[r]
@@ -98,28 +153,32 @@ class DeviceCase:
         self.sl.ef_flush(copies, keep_pending=True)
         return copies
 
-    def error_slices(self, tensor_ids: Sequence[int]) -> List[Dict[int, np.ndarray]]:
+    def error_slices(self, tensor_ids: Sequence[int], spare: Optional[torch.Tensor] = None) -> List[Dict[int, np.ndarray]]:
         """CPU copies of the true error of the given tensors, per worker.  Large cases materialise
-        one worker at a time into a single spare buffer."""
+        one worker at a time into a single spare buffer (`spare`, at least a flat buffer long, or a
+        fresh allocation)."""
         def cut(buf):
             return {j: buf[self.offs[j]:self.offs[j] + self.wl.tensors[j].numel].cpu().numpy().copy()
                     for j in tensor_ids}
         if not self.sl.ef_pending():
             return [cut(x) for x in self.e]
         out = []
-        spare = torch.empty_like(self.e[0])
+        own = spare is None
+        spare = torch.empty_like(self.e[0]) if own else spare[:self.flat]
         for r in range(self.wl.R):
             spare.copy_(self.e[r])
             self.sl.ef_flush([spare if q == r else None for q in range(self.wl.R)], keep_pending=True)
             torch.cuda.synchronize()
             out.append(cut(spare))
-        del spare
+        if own:
+            del spare
         return out
 
-    def check(self, snap: Dict[int, dict], ef_enabled: bool = True, present: Optional[List[bool]] = None) -> dict:
+    def check(self, snap: Dict[int, dict], ef_enabled: bool = True, present: Optional[List[bool]] = None,
+              spare: Optional[torch.Tensor] = None) -> dict:
         """Run the oracle on the snapshot tensors and compare with the device state after step()."""
         torch.cuda.synchronize()
-        e_cpu = self.error_slices(list(snap.keys()))
+        e_cpu = self.error_slices(list(snap.keys()), spare=spare)
         R = self.wl.R
         worst = 0.0
         report = {"tensors": 0, "payload_bytes": 0, "theta_max_err_over_rms": 0.0}

@@ -474,3 +474,25 @@ def test_argument_errors():
     assert ei.value.status == B.SL_ERR_ALIGNMENT
     sl.outer_step(th, [th, th], e, pay)
     torch.cuda.synchronize()
+
+
+def test_read_stats_matches_the_oracle_statistics():
+    """sl_read_stats: per (worker, tensor) mean, sigma, 3 sigma and the four table entries of the last
+    compression, bit for bit those of the oracle's quantiser (Sec. 4), for every worker slot; a tensor
+    of more than 64 chunks takes the second summation group."""
+    import oracle as O
+    tensors = [I.TensorSpec("a", 128, 192, 0), I.TensorSpec("big", 576, 640, 0), I.TensorSpec("norm", 1, 768, 1),
+               I.TensorSpec("flat", 1, 4096 * 2 + 100, 1)]
+    wl = I.Workload("stats", tensors, R=3, k=64, recipe="student_t4", seed=91)
+    c = _case(wl, e_scale=0.5)
+    c.fill_local(0)
+    snap = c.snapshot(range(len(tensors)))
+    c.step()
+    cfg = O.Config(k=wl.k, R=wl.R, beta=wl.beta, outer_lr=wl.outer_lr)
+    for r in range(wl.R):
+        got = c.sl.read_stats(r, len(tensors)).cpu().numpy()
+        for j, t in enumerate(tensors):
+            out = O.compress(cfg, O.Table([(t.rows, t.cols)]), snap[j]["theta"], snap[j]["local"][r], snap[j]["e"][r].copy())
+            mu, sigma, lut = out.stats[0, 0], out.stats[0, 1], out.stats[0, 2:6]
+            want = np.array([mu, sigma, np.float32(3.0) * sigma, *lut, 0.0], np.float32)
+            assert np.array_equal(got[j].view(np.uint32), want.view(np.uint32)), (r, t.name, got[j], want)

@@ -4,11 +4,14 @@ allocator's device-wide synchronisation).  Its scratch is a fixed 4 MiB array in
 so the call needs no context and no workspace.
 
 The check: on the same inputs it must leave exactly the bytes that the ordinary entry point,
-sl_compress() on a context holding that single tensor, leaves -- payload and error buffer
-bit-exact (the bar of the other GPU tests) -- on two calls in a row that carry the error buffer
-over, for a blocked matrix, a flat vector with a short tail, and a smaller call after a larger one
-(the shared scratch keeps the previous call's contents, which must not leak into the next).
+sl_compress() on a context holding that single tensor, leaves, and that the CPU oracle computes
+-- payload and error buffer bit-exact (the bar of the other GPU tests) -- on two calls in a row
+that carry the error buffer over, for a blocked matrix, a flat vector with a short tail, a smaller
+call after a larger one (the shared scratch keeps the previous call's contents, which must not
+leak into the next), and two tensors that nearly fill the scratch.
 Oversized tensors must be refused.  This file is collected last on purpose."""
+import os
+
 import pytest
 import torch
 
@@ -29,11 +32,24 @@ def _pair(rows, cols, k, seed):
     return B, wl, theta, sl, n_pay, dev
 
 
-@pytest.mark.parametrize("rows,cols,k", [(128, 192, 64), (1, 4096 * 3 + 1234, 41), (64, 64, 123)])
+# the last two fill most of the 4 MiB scratch (about 8,700 chunks at k = 64): a blocked matrix of 7,920
+# chunks and a flat vector of 8,001 chunks with a short tail, 124 and 126 summation groups
+SHAPES = [(128, 192, 64), (1, 4096 * 3 + 1234, 41), (64, 64, 123), (5632, 5760, 64), (1, 4096 * 8000 + 77, 64)]
+
+
+@pytest.mark.parametrize("rows,cols,k", SHAPES)
 def test_static_scratch_entry_point_matches_sl_compress(rows, cols, k):
+    """Against sl_compress() on the same inputs, and both against the CPU oracle (Alg. 1, the worker's
+    compression block): payload bytes and error buffer bit for bit."""
+    import numpy as np
+    import oracle as O
+    O.set_threads(os.cpu_count() or 1)
     B, wl, theta, sl, n_pay, dev = _pair(rows, cols, k, seed=500 + k)
     e_ref = I.initial_error(wl, 0, dev, scale=0.5)
     e_new = e_ref.clone()
+    e_orc = e_ref.cpu().numpy().copy()
+    cfg = O.Config(k=k, R=1, beta=wl.beta)
+    tab = O.Table([(rows, cols)])
     for step in range(2):  # two calls in a row, error feedback carried from the first into the second
         local = I.theta_local(wl, theta, 0, step)
         pay_ref = torch.zeros(n_pay, dtype=torch.uint8, device=dev)
@@ -43,6 +59,10 @@ def test_static_scratch_entry_point_matches_sl_compress(rows, cols, k):
         torch.cuda.synchronize()
         assert torch.equal(pay_new, pay_ref), f"payload differs at step {step}"
         assert torch.equal(e_new.view(torch.int32), e_ref.view(torch.int32)), f"error buffer differs at step {step}"
+        out = O.compress(cfg, tab, theta.cpu().numpy(), local.cpu().numpy(), e_orc)
+        assert np.array_equal(pay_new.cpu().numpy(), out.payload), f"payload differs from the oracle at step {step}"
+        assert np.array_equal(e_new.cpu().numpy().view(np.uint32), e_orc.view(np.uint32)), \
+            f"error buffer differs from the oracle at step {step}"
 
 
 def test_static_scratch_rejects_what_does_not_fit_and_bad_arguments():
