@@ -473,6 +473,72 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
     return out
 
 
+def run_worker_per_gpu(args) -> dict:
+    """--mode worker-per-gpu: one worker per rank (R = number of ranks): sl_compress on the rank's own
+    theta_local and e, an NCCL all-gather of the payloads into local memory, sl_aggregate_apply on the
+    rank's theta replica.  value = params / max-over-ranks step time (every rank updates the same
+    params with R = N workers); per-GPU work is fixed as N grows."""
+    import torch
+    import torch.distributed as dist
+    from paper_2508_15706_b200 import inputs as I
+    from paper_2508_15706_b200.binding import SparseLoCo
+    from paper_2508_15706_b200.worker_step import WorkerStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    import dataclasses
+    wl = dataclasses.replace(I.workload(args.workload), R=world)
+    k = args.k or wl.k
+    shapes = [(t.rows, t.cols) for t in wl.tensors]
+    sl = SparseLoCo(shapes, I.offsets(wl.tensors), k=k, R=world, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr)
+    theta = I.theta_sync(wl, dev)
+    local = I.theta_local(wl, theta, rank, 0)
+    e = I.initial_error(wl, rank, dev, scale=0.5)
+    coded = args.wire == "coded"
+    ws = WorkerStep(sl, sl.payload_bytes(), world, rank, dev, coded=coded,
+                    coded_capacity=sl.coded_payload_capacity() if coded else 0)
+    for _ in range(args.warmup):
+        ws.step(theta, local, e)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        ws.step(theta, local, e)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms_max = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    clocks = sampler.stop(t0, t1)
+    N = wl.numel
+    wire = int(ws.exchange.meta[:, 1].max())
+    out = {"metric": METRIC, "value": N * args.steps / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": wl.name, "params": N, "R": world, "k": k, "mode": "worker-per-gpu",
+                      "exchange": "all-gather of payloads (torch.distributed, NCCL) into local memory",
+                      "wire_format": args.wire, "wire_bytes_per_worker": wire, "plain_payload_bytes": sl.payload_bytes(),
+                      "l2": "inputs larger than L2"},
+           "clocks": clocks, "gpu_launches": (9 + (3 + world if coded else 0)) * args.steps}
+    if world > 1:
+        dist.destroy_process_group()
+    return out if rank == 0 else None
+
+
 def run_e2e(torch, I, sl, wl, theta, e, payloads, flat, N, args) -> dict:
     """The same step through the host-buffer entry point: every worker's parameters start in pinned
     host memory and cross to the device inside the timed region; the updated theta_sync is read back."""
@@ -588,7 +654,7 @@ def run_reference(args) -> dict:
     names = ",".join(wl.tensors[j].name for j in ids)
     sample = f"each step = one outer step, all R={wl.R} workers, tensors [{names}] = {n} params of {wl.numel}"
     return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
-            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", str(args.gpus))), "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.numel, "R": wl.R, "k": k, "H": wl.H, "chunk": 4096},
@@ -618,6 +684,11 @@ def main():
                     help="element shift between the views of workers sharing a theta_local buffer (0: identical views)")
     ap.add_argument("--no-alias-check", action="store_true",
                     help="skip the measurement of what sharing theta_local buffers does to the kernel's rate")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "worker-per-gpu"],
+                    help="replicas: every rank runs the whole R-worker step on its own GPU (the headline); "
+                         "worker-per-gpu: one worker per rank, payloads all-gathered (R = number of ranks)")
+    ap.add_argument("--wire", default="plain", choices=["plain", "coded"],
+                    help="worker-per-gpu: what travels, the 12-bit payload or its entropy-coded form")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense DiLoCo comparator line")
@@ -627,9 +698,36 @@ def main():
     ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    out = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
+    if args.impl == "reference":
+        out = run_reference(args)
+    elif args.mode == "worker-per-gpu":
+        out = run_worker_per_gpu(args)
+    else:
+        out = run_ours(args)
     if out is not None:
         print(json.dumps(out))
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this command line, one per GPU,
+    with the environment a launcher would set (rendezvous on 127.0.0.1), and pass on what they print
+    (rank 0 alone prints the JSON line).  Returns the first non-zero exit code."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable] + sys.argv, env=env))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
 
 
 if __name__ == "__main__":
