@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "c5_dense_d2048"
 
 # DRAM bytes per ef_topk launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
 # on a smaller case of the same kernel, as bytes per (parameter x worker); see profiles/.
-NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER = 12.551  # profiles/ncu_full_c5_layer0_top3_kernels.md
+NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER = 12.551  # profiles/ncu_full_c5_layer0_top3_kernels.md
 
 
 def record_stride(k: int) -> int:
@@ -48,7 +48,7 @@ def algorithmic_bytes_per_param(R: int, k: int) -> float:
     return R * 12 + 4 + 8 + R * 2 * record_stride(k) / 4096.0
 
 
-def ef_topk_bytes_per_param(R: int) -> float:
+def ef_select_bytes_per_param(R: int) -> float:
     return R * 12 + 4
 
 
@@ -232,9 +232,9 @@ def run_ours(args) -> dict:
 
     # roofline of the dominant kernel, timed live with CUDA events inside the timed region
     top = max(prof.items(), key=lambda kv: kv[1][0])
-    ef_ms, ef_n = prof["ef_topk"]
+    ef_ms, ef_n = prof["ef_select"]
     ef_avg_ms = ef_ms / max(ef_n, 1)
-    ef_bytes = ef_topk_bytes_per_param(wl.R) * N
+    ef_bytes = ef_select_bytes_per_param(wl.R) * N
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -244,8 +244,8 @@ def run_ours(args) -> dict:
     peak_src = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
     achieved = ef_bytes / (ef_avg_ms * 1e-3) / 1e9
     traffic = None
-    if NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER is not None:
-        traffic = NCU_EF_TOPK_DRAM_BYTES_PER_PARAM_WORKER * N * wl.R
+    if NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER is not None:
+        traffic = NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER * N * wl.R
     step_bytes = algorithmic_bytes_per_param(wl.R, k) * N
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
     kernel_ms = {name: round(v[0] / max(v[1], 1), 4) for name, v in prof.items()}
@@ -268,7 +268,7 @@ def run_ours(args) -> dict:
                    "multi_gpu": "replicas only (no data-path collective)"},
         "clocks": clocks,
         "gpu_launches": 8 * args.steps + (1 if deferred else 0),
-        "roofline": {"bound": "hbm", "kernel": "ef_topk", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "ef_select", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": ef_bytes, "avg_launch_ms": ef_avg_ms,
                      "dominant_by_time": top[0]},
@@ -392,7 +392,7 @@ def time_compression_kernel(torch, sl, theta, locals_r, e, payloads, steps: int 
     for _ in range(steps):
         sl.outer_step(theta, locals_r, e, payloads)
     torch.cuda.synchronize()
-    ms, n = sl.profile_read()["ef_topk"]
+    ms, n = sl.profile_read()["ef_select"]
     sl.profile_enable(False)
     return ms / max(n, 1)
 
@@ -421,7 +421,7 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
     wl = I.workload("c5_l12")
     N = wl.numel
     sl, ws, theta, e, payloads = build(wl)
-    bytes_launch = ef_topk_bytes_per_param(wl.R) * N
+    bytes_launch = ef_select_bytes_per_param(wl.R) * N
     storage, views = make_locals(torch, I, wl, theta, wl.R, 0)
     rows = {}
     ms = time_compression_kernel(torch, sl, theta, views, e, payloads)
@@ -454,7 +454,7 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
     sl, ws, theta, e, payloads = build(wl)
     storage, views = make_locals(torch, I, wl, theta, wl.R, 0)
     ms = time_compression_kernel(torch, sl, theta, views, e, payloads)
-    b8 = ef_topk_bytes_per_param(wl.R) * N
+    b8 = ef_select_bytes_per_param(wl.R) * N
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record(torch.cuda.current_stream())
     for _ in range(4):

@@ -784,7 +784,7 @@ sl_status sl_profile_read(sl_ctx* c, float* ms_total, int64_t* launches) {
 }
 
 const char* sl_profile_name(int32_t slot) {
-    static const char* names[kProfSlots] = {"ef_topk", "chunk_sum", "tensor_mean", "chunk_var", "tensor_sigma",
+    static const char* names[kProfSlots] = {"ef_select", "chunk_sum", "tensor_mean", "chunk_var", "tensor_sigma",
                                             "chunk_bins", "tensor_lut", "pack_fix", "decode_avg_apply"};
     return slot >= 0 && slot < kProfSlots ? names[slot] : "";
 }
