@@ -22,8 +22,8 @@ namespace {
 // Lane l of a warp owns in-chunk indices p = 128 i + 4 l + j (i = 0..31, j = 0..3), register 4 i + j.
 //
 // Selection (exact: magnitude = float bits without the sign, ties to the lower index):
-//  A. 8 group maxima per lane (16 values each); M = the largest.
-//  B. a threshold T by bisection over the 256 group maxima: at least keff groups, hence at least keff
+//  A. 8 group maxima per lane (16 values each; 32 of 4 values each for k > 128); M = the largest.
+//  B. a threshold T by bisection over the group maxima: at least keff groups, hence at least keff
 //     elements, reach T, and only a few more do (about 1.15 keff elements).
 //  C. every element with key >= T is a candidate; the lanes list the candidates' positions in shared
 //     memory.
@@ -33,8 +33,8 @@ namespace {
 //     resolved by a second bisection over positions.
 //  F. selected candidates set their bit in a 4096-bit map; its prefix popcount is the slot of each
 //     (ascending in-chunk index) and the holder writes (index, value) to the staging arrays.
-// All-zero chunks, thresholds of zero, more candidates than the list holds and k > 256 take an exact
-// bitwise search over all 4096 keys instead (select_slow).
+// All-zero chunks, thresholds of zero and more candidates than the list holds take an exact bitwise
+// search over all 4096 keys instead (select_slow).
 //
 // Chunks that cannot travel as tensor-map blocks (short tails, tables whose blocks do not start on a
 // 64-element boundary, tile copies switched off) are read and written with plain loads and stores by
@@ -115,7 +115,7 @@ constexpr int kSelThreads = 32 * (kSelWarps + 1);    // + the producer warp
 constexpr int kThetaRing = 3;                        // blocks of theta in flight or in use
 constexpr int kUnitSlots = 5;                        // units in flight or in use
 constexpr int kCandCap = 384;                        // candidate positions a warp can list
-constexpr int kGroups = 256;                         // group maxima per chunk (16 elements each)
+constexpr int kSelNarrowMaxK = 128;                  // largest k served by the groups-of-16 kernel
 
 struct SelSmem {
     float theta_s[kThetaRing][kChunk];
@@ -360,49 +360,62 @@ __device__ __forceinline__ void rank_and_emit(const uint16_t* __restrict__ cand,
     }
 }
 
-// Steps A-F on the warp's registers.  `u` = this lane's 128 values (0 at indices >= len).
-template <bool GLOBAL>
-__device__ __forceinline__ void select_unit(const float (&u)[128], const USource& src, int len, int keff,
-                                            unsigned* bitmap, uint16_t* cand, uint16_t* __restrict__ out_idx,
-                                            float* __restrict__ out_val) {
-    const int lane = threadIdx.x & 31;
+// Steps A and B: GN group maxima per lane (groups of 128 / GN of the lane's values, 32 GN per chunk) and a
+// threshold T that at least keff of them reach, and not many more; T = 0 when there is none (all-zero
+// or mostly-zero chunk, maxima that are all NaN, keff beyond the number of groups).  `probe` = a key
+// that fewer than keff groups reach: a good first guess for the element-level cut.
+template <int GN>
+__device__ __forceinline__ void group_threshold(const float (&u)[128], int keff, unsigned& T, unsigned& probe) {
+    constexpr int GS = 128 / GN;
     // A. group maxima (on floats: a NaN is skipped, which can only lower the threshold)
-    unsigned kg[8];
+    unsigned kg[GN];
     float mall = 0.0f;
 #pragma unroll
-    for (int g = 0; g < 8; ++g) {
+    for (int g = 0; g < GN; ++g) {
         float m = 0.0f;
 #pragma unroll
-        for (int q = 16 * g; q < 16 * g + 16; q += 2) m = fmaxf(m, fmaxf(fabsf(u[q]), fabsf(u[q + 1])));
+        for (int q = GS * g; q < GS * g + GS; q += 2) m = fmaxf(m, fmaxf(fabsf(u[q]), fabsf(u[q + 1])));
         kg[g] = __float_as_uint(m);
         mall = fmaxf(mall, m);
     }
     const unsigned M = __reduce_max_sync(kFull, __float_as_uint(mall));
-
-    // B. threshold: count(group maxima >= T) >= keff, and not many more
-    unsigned T = 0, probe = 0;
-    if (M != 0u && keff <= kGroups) {
-        unsigned lo = 0, hi = M + 1u, c_lo = kGroups;  // count(>= lo) = c_lo >= keff > count(>= hi)
-        const unsigned enough = (unsigned)keff + max(2u, (unsigned)keff >> 3);
-        unsigned x = M > (2u << 23) ? M - (2u << 23) : (M >> 1);  // first guess: a quarter of the largest magnitude
-        for (int it = 0; it < 40; ++it) {
-            unsigned c = 0;
+    // B. bisection over the keys of the group maxima
+    T = 0;
+    probe = 0;
+    if (M == 0u || keff > 32 * GN) return;
+    unsigned lo = 0, hi = M + 1u, c_lo = 32 * GN;  // count(>= lo) = c_lo >= keff > count(>= hi)
+    const unsigned enough = (unsigned)keff + max(2u, (unsigned)keff >> 3);
+    unsigned x = M > (2u << 23) ? M - (2u << 23) : (M >> 1);  // first guess: a quarter of the largest magnitude
+    for (int it = 0; it < 40; ++it) {
+        unsigned c = 0;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) c += kg[g] >= x ? 1u : 0u;
-            c = __reduce_add_sync(kFull, c);
-            if (c >= (unsigned)keff) {
-                lo = x;
-                c_lo = c;
-            } else {
-                hi = x;
-            }
-            if ((lo != 0u && c_lo <= enough) || hi - lo <= 1) break;
-            x = lo + ((hi - lo) >> 1);
+        for (int g = 0; g < GN; ++g) c += kg[g] >= x ? 1u : 0u;
+        c = __reduce_add_sync(kFull, c);
+        if (c >= (unsigned)keff) {
+            lo = x;
+            c_lo = c;
+        } else {
+            hi = x;
         }
-        T = lo;
-        probe = hi;  // fewer than keff groups reach it: a good first guess for the element-level cut
+        if ((lo != 0u && c_lo <= enough) || hi - lo <= 1) break;
+        x = lo + ((hi - lo) >> 1);
     }
-    if (T == 0u) {  // zero chunk, mostly-zero chunk, NaN-only maxima, k > 256: exact search over everything
+    T = lo;
+    probe = hi;
+}
+
+// Steps A-F on the warp's registers.  `u` = this lane's 128 values (0 at indices >= len).
+template <bool GLOBAL, bool WIDE>
+__device__ __forceinline__ void select_unit(const float (&u)[128], const USource& src, int len, int keff,
+                                            unsigned* bitmap, uint16_t* cand, uint16_t* __restrict__ out_idx,
+                                            float* __restrict__ out_val) {
+    const int lane = threadIdx.x & 31;
+    // groups of 16 values up to k = 128 (about 1.15 k candidates); beyond that a threshold taken from 256
+    // group maxima lets too many elements through, and groups of 4 take over (WIDE: a kernel of its own,
+    // so that the common case carries neither the code nor the registers of the other)
+    unsigned T, probe;
+    group_threshold<WIDE ? 32 : 8>(u, keff, T, probe);
+    if (T == 0u) {  // no usable threshold: exact search over everything
         select_slow<GLOBAL>(src, len, keff, bitmap, out_idx, out_val);
         return;
     }
@@ -441,7 +454,7 @@ __device__ __forceinline__ void select_unit(const float (&u)[128], const USource
     else rank_and_emit<kCandCap / 32, GLOBAL>(cand, n_c, T, probe, src, keff, bitmap, out_idx, out_val);
 }
 
-template <bool EF, bool PENDING>
+template <bool EF, bool PENDING, bool WIDE>
 __global__ void __launch_bounds__(kSelThreads, 1)
 ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                  const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma, int use_tma) {
@@ -694,7 +707,7 @@ ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
             src.rs = kTile;
         }
         const long long slot_base = ((long long)r * n_chunks + g) * kp;
-        select_unit<EF>(u, src, cd.len, keff, bitmap, cand, ws.idx + slot_base, ws.val + slot_base);
+        select_unit<EF, WIDE>(u, src, cd.len, keff, bitmap, cand, ws.idx + slot_base, ws.val + slot_base);
         __syncwarp();  // the map and the list are free again
         if (!EF && lane == 0) mbar_arrive(&sm.empty_u[s]);
     }

@@ -272,15 +272,19 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     {   // one persistent CTA per SM
         const unsigned grid = (unsigned)(G < c->n_sms ? G : c->n_sms);
         const int tm = use_tma ? 1 : 0;
-        if (!ef)
-            ef_select_kernel<false, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
-                                                                                       c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
-        else if (consume)
-            ef_select_kernel<true, true><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
-                                                                                     c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
-        else
-            ef_select_kernel<true, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(c->d_chunks, G, workers, k, kp,
-                                                                                      c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
+#define SL_LAUNCH_SELECT(EFV, PENDV)                                                                                  \
+    do {                                                                                                             \
+        if (k > kSelNarrowMaxK)                                                                                      \
+            ef_select_kernel<EFV, PENDV, true><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                          \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
+        else                                                                                                         \
+            ef_select_kernel<EFV, PENDV, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                         \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
+    } while (0)
+        if (!ef) SL_LAUNCH_SELECT(false, false);
+        else if (consume) SL_LAUNCH_SELECT(true, true);
+        else SL_LAUNCH_SELECT(true, false);
+#undef SL_LAUNCH_SELECT
     }
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
@@ -518,12 +522,13 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     cudaError_t e = cudaGetDevice(&c->device);
     int n_sms = 0, per_sm = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_select_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(ef_select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelSmem));
+#define SL_SELECT_ATTR(EFV, PENDV, WIDEV)                                                                            \
+    if (e == cudaSuccess)                                                                                            \
+        e = cudaFuncSetAttribute(ef_select_kernel<EFV, PENDV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
+                                 (int)sizeof(SelSmem))
+    SL_SELECT_ATTR(true, false, false); SL_SELECT_ATTR(true, true, false); SL_SELECT_ATTR(false, false, false);
+    SL_SELECT_ATTR(true, false, true); SL_SELECT_ATTR(true, true, true); SL_SELECT_ATTR(false, false, true);
+#undef SL_SELECT_ATTR
     per_sm = 1;
     {   // the apply kernel's shared memory depends on k alone: sized once
         const int asz = (int)apply_smem_bytes(cfg->k);
@@ -1037,7 +1042,9 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
         SL_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
         int n_sms = 0;
         SL_CUDA(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-        SL_CUDA(cudaFuncSetAttribute(ef_select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SL_CUDA(cudaFuncSetAttribute(ef_select_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(SelSmem)));
+        SL_CUDA(cudaFuncSetAttribute(ef_select_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)sizeof(SelSmem)));
         su.scratch = ptr;
         su.status = reinterpret_cast<int*>(static_cast<char*>(ptr) + kStaticScratchBytes - 256);
@@ -1068,8 +1075,12 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     TmaArgs no_tma;  // plain loads and stores: nothing has to be encoded or uploaded for the caller's buffers
     memset(&no_tma, 0, sizeof(no_tma));
     no_tma.status = su.status;
-    ef_select_kernel<true, false><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync, ptrs,
-                                                                              ws, no_tma, 0);
+    if (k > kSelNarrowMaxK)
+        ef_select_kernel<true, false, true><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
+                                                                                        ptrs, ws, no_tma, 0);
+    else
+        ef_select_kernel<true, false, false><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
+                                                                                         ptrs, ws, no_tma, 0);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);
     tensor_reduce_kernel<0><<<1, 128, 0, st>>>(d_tinfo, G, 1, 1, ws, ptrs);
