@@ -91,6 +91,9 @@ def lib():
         L.orc_outer_step.argtypes = [P, P, C.c_int32, P, P, P, P]
         L.orc_diloco_step.argtypes = [P, C.c_int32, C.c_int32, C.c_float, C.c_float, P, P, P]
         L.orc_diloco_lom_step.argtypes = [P, C.c_int32, C.c_int32, C.c_float, C.c_float, P, P, P]
+        L.orc_lom_step.argtypes = [P, P, C.c_int32, C.c_float, C.c_int32, P, P, P]
+        L.orc_diloco_topk_step.argtypes = [P, P, C.c_int32, C.c_float, P, P, P, P]
+        L.orc_lom_topk_step.argtypes = [P, P, C.c_int32, C.c_float, P, P, P, P]
         L.orc_ixc_encode_chunk.argtypes = [P, C.c_int32, C.c_int32, P, P]
         L.orc_ixc_decode_chunk.argtypes = [P, P, C.c_int32, C.c_int32, P]
         L.orc_ixc_encode_payload.argtypes = [P, P, C.c_int32, P, P]
@@ -345,3 +348,33 @@ def diloco_lom_step(tab: Table, theta: np.ndarray, theta_r: List[np.ndarray], m_
     arr = _ptr_array([_chk(a, np.float32) for a in theta_r])
     marr = _ptr_array([_chk(a, np.float64) for a in m_r])
     lib().orc_diloco_lom_step(tab.arr, tab.n, len(theta_r), beta_outer, alpha, _ptr(theta), arr, marr)
+
+
+# ---------------------------------------------------------------- Top-k / local-momentum variants (Alg. 2-4)
+
+def lom_step(cfg: Config, tab: Table, theta: np.ndarray, theta_r: List[np.ndarray], m_r: List[np.ndarray],
+             mu: float, sub_k: bool = False) -> None:
+    """Alg. 2 (DiLoCo-LOM; with sub_k: DiLoCo-LOM-Sub-k) in place on theta and the fp32 momenta m_r."""
+    c = cfg.c()
+    lib().orc_lom_step(C.byref(c), tab.arr, tab.n, mu, int(sub_k), _ptr(_chk(theta, np.float32)),
+                       _ptr_array([_chk(a, np.float32) for a in theta_r]),
+                       _ptr_array([_chk(a, np.float32) for a in m_r]))
+
+
+def diloco_topk_step(cfg: Config, tab: Table, theta: np.ndarray, theta_r: List[np.ndarray],
+                     e: Optional[List[np.ndarray]], m: np.ndarray, mu: float) -> None:
+    """Alg. 3 (DiLoCo + Top-k, error feedback when e is given) in place on theta, m and the e_r."""
+    c = cfg.c()
+    ea = _ptr_array([_chk(a, np.float32) for a in e]) if e is not None else None
+    lib().orc_diloco_topk_step(C.byref(c), tab.arr, tab.n, mu, _ptr(_chk(theta, np.float32)),
+                               _ptr_array([_chk(a, np.float32) for a in theta_r]), ea, _ptr(_chk(m, np.float32)))
+
+
+def lom_topk_step(cfg: Config, tab: Table, theta: np.ndarray, theta_r: List[np.ndarray], m_r: List[np.ndarray],
+                  e: Optional[List[np.ndarray]], mu: float) -> None:
+    """Alg. 4 (DiLoCo-LOM + Top-k, error feedback when e is given) in place on theta, the m_r and the e_r."""
+    c = cfg.c()
+    ea = _ptr_array([_chk(a, np.float32) for a in e]) if e is not None else None
+    lib().orc_lom_topk_step(C.byref(c), tab.arr, tab.n, mu, _ptr(_chk(theta, np.float32)),
+                            _ptr_array([_chk(a, np.float32) for a in theta_r]),
+                            _ptr_array([_chk(a, np.float32) for a in m_r]), ea)

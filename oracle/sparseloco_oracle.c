@@ -729,3 +729,161 @@ void orc_diloco_lom_step(const orc_tensor* ts, int32_t nt, int32_t R, float beta
         }
     }
 }
+
+/* ================================================================ the paper's Top-k / LOM variants
+ *
+ * App. "Exact algorithmic description of DiLoCo variants", Alg. 2-4 (Sec. 3.2 for LOM and Sub-k).
+ * No quantiser: Top-k keeps the selected values as they are.  All Top-k operations are chunk-wise with
+ * the chunking and tie rule of the main path.  Precision: what a worker keeps between steps (m_r, e_r)
+ * and what its selection is taken on are fp32, formed by single-rounded operations in the algorithm's
+ * order -- d = theta - theta_r; m_r = fma(mu, m_r, d); Nesterov direction nd = fma(mu, m_r, d);
+ * u = fma(rho, e_r, .) -- because the selection depends on their bits; everything across workers (the
+ * average, the global momentum, the parameter update) is evaluated in fp64 and rounded once.
+ */
+
+/* Chunk-wise Top-k of a flat buffer u (tensor j at ts[j].offset): for every chunk the selected
+ * element positions (inside the flat buffer) and values, appended to pos / val; returns the count. */
+static int64_t topk_of_flat(const orc_config* cfg, const orc_tensor* ts, int32_t nt, const float* u,
+                            int64_t* pos, float* val) {
+    const int32_t k = cfg->k, C = cfg->chunk_elems;
+    int64_t w = 0;
+    float* cu = (float*)malloc(sizeof(float) * (size_t)C);
+    int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)(k > 0 ? k : 1));
+    for (int32_t j = 0; j < nt; ++j) {
+        const orc_tensor* t = &ts[j];
+        const int64_t nc = orc_num_chunks(cfg, t);
+        for (int64_t ch = 0; ch < nc; ++ch) {
+            const int32_t L = (int32_t)orc_chunk_len(cfg, t, ch);
+            for (int32_t p = 0; p < L; ++p) cu[p] = u[t->offset + orc_chunk_pos(cfg, t, ch, p)];
+            const int32_t m = orc_topk_chunk(cu, L, k, idx);
+            for (int32_t s = 0; s < m; ++s, ++w) {
+                pos[w] = t->offset + orc_chunk_pos(cfg, t, ch, idx[s]);
+                val[w] = cu[idx[s]];
+            }
+        }
+    }
+    free(cu);
+    free(idx);
+    return w;
+}
+
+/* Alg. 2: DiLoCo-LOM, and DiLoCo-LOM-Sub-k when sub_k != 0.  theta and the local momenta m_r (fp32)
+ * are updated in place; alpha = cfg->outer_lr, k = cfg->k. */
+void orc_lom_step(const orc_config* cfg, const orc_tensor* ts, int32_t nt, float mu, int32_t sub_k,
+                  float* theta, const float* const* theta_r, float* const* m_r) {
+    const int32_t R = cfg->R;
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+        for (int64_t i = o; i < o + n; ++i) {
+            double acc = 0.0;
+            for (int32_t r = 0; r < R; ++r) {
+                const float d = theta[i] - theta_r[r][i];
+                const float m = fmaf(mu, m_r[r][i], d); /* local momentum */
+                m_r[r][i] = m;
+                acc += (double)fmaf(mu, m, d); /* local Nesterov direction */
+            }
+            theta[i] = (float)((double)theta[i] - (double)cfg->outer_lr * acc / (double)R);
+        }
+    }
+    if (sub_k) { /* m_r <- m_r - Top-k(m_r): the selected entries become zero */
+        const int64_t slots = orc_total_slots(cfg, ts, nt);
+        int64_t* pos = (int64_t*)malloc(sizeof(int64_t) * (size_t)(slots ? slots : 1));
+        float* val = (float*)malloc(sizeof(float) * (size_t)(slots ? slots : 1));
+        for (int32_t r = 0; r < R; ++r) {
+            const int64_t w = topk_of_flat(cfg, ts, nt, m_r[r], pos, val);
+            for (int64_t s = 0; s < w; ++s) m_r[r][pos[s]] = m_r[r][pos[s]] - val[s];
+        }
+        free(pos);
+        free(val);
+    }
+}
+
+/* Alg. 3: DiLoCo + Top-k, with error feedback when e != NULL (decay rho = cfg->beta).  theta, the
+ * global momentum m and the e_r are updated in place. */
+void orc_diloco_topk_step(const orc_config* cfg, const orc_tensor* ts, int32_t nt, float mu,
+                          float* theta, const float* const* theta_r, float* const* e, float* m) {
+    const int32_t R = cfg->R;
+    int64_t flat = 0;
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t end = ts[j].offset + ts[j].rows * ts[j].cols;
+        if (end > flat) flat = end;
+    }
+    const int64_t slots = orc_total_slots(cfg, ts, nt);
+    double* acc = (double*)calloc((size_t)flat, sizeof(double));
+    float* u = (float*)calloc((size_t)flat, sizeof(float));
+    int64_t* pos = (int64_t*)malloc(sizeof(int64_t) * (size_t)(slots ? slots : 1));
+    float* val = (float*)malloc(sizeof(float) * (size_t)(slots ? slots : 1));
+    for (int32_t r = 0; r < R; ++r) {
+        for (int32_t j = 0; j < nt; ++j) {
+            const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+            for (int64_t i = o; i < o + n; ++i) {
+                const float d = theta[i] - theta_r[r][i];
+                u[i] = e ? fmaf(cfg->beta, e[r][i], d) : d;
+            }
+        }
+        const int64_t w = topk_of_flat(cfg, ts, nt, u, pos, val);
+        if (e) { /* e_r = u - Dhat */
+            for (int32_t j = 0; j < nt; ++j) {
+                const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+                for (int64_t i = o; i < o + n; ++i) e[r][i] = u[i];
+            }
+            for (int64_t s = 0; s < w; ++s) e[r][pos[s]] = u[pos[s]] - val[s];
+        }
+        for (int64_t s = 0; s < w; ++s) acc[pos[s]] += (double)val[s];
+    }
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+        for (int64_t i = o; i < o + n; ++i) {
+            const double dbar = acc[i] / (double)R;
+            const double mm = (double)mu * (double)m[i] + dbar;
+            theta[i] = (float)((double)theta[i] - (double)cfg->outer_lr * (dbar + (double)mu * mm));
+            m[i] = (float)mm;
+        }
+    }
+    free(acc); free(u); free(pos); free(val);
+}
+
+/* Alg. 4: DiLoCo-LOM + Top-k, with error feedback when e != NULL.  theta, the local momenta m_r and
+ * the e_r are updated in place. */
+void orc_lom_topk_step(const orc_config* cfg, const orc_tensor* ts, int32_t nt, float mu,
+                       float* theta, const float* const* theta_r, float* const* m_r, float* const* e) {
+    const int32_t R = cfg->R;
+    int64_t flat = 0;
+    for (int32_t j = 0; j < nt; ++j) {
+        const int64_t end = ts[j].offset + ts[j].rows * ts[j].cols;
+        if (end > flat) flat = end;
+    }
+    const int64_t slots = orc_total_slots(cfg, ts, nt);
+    double* acc = (double*)calloc((size_t)flat, sizeof(double));
+    uint8_t* hit = (uint8_t*)calloc((size_t)flat, 1);
+    float* u = (float*)calloc((size_t)flat, sizeof(float));
+    int64_t* pos = (int64_t*)malloc(sizeof(int64_t) * (size_t)(slots ? slots : 1));
+    float* val = (float*)malloc(sizeof(float) * (size_t)(slots ? slots : 1));
+    for (int32_t r = 0; r < R; ++r) {
+        for (int32_t j = 0; j < nt; ++j) {
+            const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+            for (int64_t i = o; i < o + n; ++i) {
+                const float d = theta[i] - theta_r[r][i];
+                const float mm = fmaf(mu, m_r[r][i], d);
+                m_r[r][i] = mm;
+                const float nd = fmaf(mu, mm, d);
+                u[i] = e ? fmaf(cfg->beta, e[r][i], nd) : nd;
+            }
+        }
+        const int64_t w = topk_of_flat(cfg, ts, nt, u, pos, val);
+        if (e) {
+            for (int32_t j = 0; j < nt; ++j) {
+                const int64_t n = ts[j].rows * ts[j].cols, o = ts[j].offset;
+                for (int64_t i = o; i < o + n; ++i) e[r][i] = u[i];
+            }
+            for (int64_t s = 0; s < w; ++s) e[r][pos[s]] = u[pos[s]] - val[s];
+        }
+        for (int64_t s = 0; s < w; ++s) {
+            acc[pos[s]] += (double)val[s];
+            hit[pos[s]] = 1;
+        }
+    }
+    for (int64_t i = 0; i < flat; ++i)
+        if (hit[i]) theta[i] = (float)((double)theta[i] - (double)cfg->outer_lr * acc[i] / (double)R);
+    free(acc); free(hit); free(u); free(pos); free(val);
+}
