@@ -144,6 +144,34 @@ sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* thet
 sl_status sl_diloco_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local, float* momentum,
                          float beta_outer, void* cuda_stream);
 
+/* The paper's Top-k and local-outer-momentum variants on the same buffers (Sec. 3.2; appendix "Exact
+ * algorithmic description of DiLoCo variants", Alg. 2-4).  None of them quantises: Top-k keeps the
+ * selected values as they are, chunk-wise with the chunking and tie rule above, k = the context's k.
+ * alpha = the context's outer_lr, the error-feedback decay rho = the context's beta, mu = the outer
+ * momentum coefficient (0 <= mu <= 1).  What a worker keeps (m_r, e_r) and what it selects on are fp32,
+ * formed by single-rounded operations in the algorithm's order: d = theta - theta_r; m_r = fma(mu, m_r,
+ * d); nd_r = fma(mu, m_r, d); u_r = fma(rho, e_r, .).  Averages are fp32 sums in ascending r divided by
+ * R.  All pointer tables are HOST arrays of R DEVICE pointers; buffers are flat fp32 and only the
+ * elements of the tensor table are touched.  The Top-k steps use the lent workspace (NOMEM without
+ * one); waiting values of a deferred subtraction are written out first.
+ *
+ *   sl_lom_step         Alg. 2, DiLoCo-LOM: m_r and theta updated in place, theta = theta - alpha mean_r
+ *                       nd_r.  sub_k != 0: DiLoCo-LOM-Sub-k, afterwards m_r = m_r - Top-k(m_r), i.e. the k
+ *                       largest entries of every chunk of m_r become +0.
+ *   sl_diloco_topk_step Alg. 3, DiLoCo + Top-k: u_r = theta - theta_r, or fma(rho, e_r, theta - theta_r)
+ *                       when e is given (then e_r = u_r - Top-k(u_r) in place); D = mean_r Top-k(u_r);
+ *                       momentum = fma(mu, momentum, D); theta = theta - alpha (D + mu momentum).
+ *   sl_lom_topk_step    Alg. 4, DiLoCo-LOM + Top-k: m_r and nd_r as in Alg. 2, u_r = nd_r or fma(rho, e_r,
+ *                       nd_r); theta = theta - alpha mean_r Top-k(u_r).  theta_local is CONSUMED: on return
+ *                       buffer r holds nd_r (the entries must be distinct buffers).
+ * Errors: INVALID_ARG (NULL, mu outside [0, 1], aliased state buffers), ALIGNMENT, NOMEM, CUDA. */
+sl_status sl_lom_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local, float* const* m_r,
+                      float mu, int32_t sub_k, void* cuda_stream);
+sl_status sl_diloco_topk_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local, float* const* e,
+                              float* momentum, float mu, void* cuda_stream);
+sl_status sl_lom_topk_step(sl_ctx* ctx, float* theta_sync, float* const* theta_local, float* const* m_r,
+                           float* const* e, float mu, void* cuda_stream);
+
 /* Entropy-coded indices for the wire (App. "Compression of indices": 12 bits per index is the naive
  * cost, log2 C(4096, k) / k the bound, 8.9 / 6.6 / 5.6 bits at k = 32 / 128 / 256 what the paper
  * reports from a scheme it does not describe).  The coding below is this library's own and reaches

@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name",
+    "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step",
 )
 PROFILE_SLOTS = 9
 
@@ -72,6 +72,9 @@ def _load():
     L.sl_profile_name.restype = C.c_char_p
     L.sl_validate_payload.argtypes = [P, P, P, P]
     L.sl_diloco_step.argtypes = [P, P, P, P, C.c_float, P]
+    L.sl_lom_step.argtypes = [P, P, P, P, C.c_float, C.c_int32, P]
+    L.sl_diloco_topk_step.argtypes = [P, P, P, P, P, C.c_float, P]
+    L.sl_lom_topk_step.argtypes = [P, P, P, P, P, C.c_float, P]
     L.sl_coded_payload_capacity.argtypes = [P, C.POINTER(C.c_size_t)]
     L.sl_encode_payload.argtypes = [P, P, P, P, P]
     L.sl_decode_payload.argtypes = [P, P, C.c_size_t, P, P]
@@ -254,6 +257,28 @@ class SparseLoCo:
         tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
         _check(_L.sl_diloco_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, _dev_ptr(momentum, torch.float32),
                                  beta_outer, _stream()))
+
+    # -- the paper's Top-k / local-momentum variants (Alg. 2-4 of its appendix), no quantiser
+    def lom_step(self, theta_sync, theta_local: List[torch.Tensor], m_r: List[torch.Tensor], mu: float,
+                 sub_k: bool = False) -> None:
+        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
+        ma = _ptr_array([_dev_ptr(t, torch.float32) for t in m_r])
+        _check(_L.sl_lom_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, ma, mu, int(sub_k), _stream()))
+
+    def diloco_topk_step(self, theta_sync, theta_local: List[torch.Tensor], e: Optional[List[torch.Tensor]],
+                         momentum, mu: float) -> None:
+        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
+        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        _check(_L.sl_diloco_topk_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, ea,
+                                      _dev_ptr(momentum, torch.float32), mu, _stream()))
+
+    def lom_topk_step(self, theta_sync, theta_local: List[torch.Tensor], m_r: List[torch.Tensor],
+                      e: Optional[List[torch.Tensor]], mu: float) -> None:
+        """theta_local is consumed: on return buffer r holds worker r's Nesterov direction."""
+        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
+        ma = _ptr_array([_dev_ptr(t, torch.float32) for t in m_r])
+        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        _check(_L.sl_lom_topk_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, ma, ea, mu, _stream()))
 
     def coded_payload_capacity(self) -> int:
         v = C.c_size_t()

@@ -19,6 +19,11 @@ namespace {
 //   4. applies theta = fma(-alpha/D, sum, theta) to its 32 positions, clears the tile on the way and
 //      stores the vectors that received anything.
 //
+// FUSE 3 / 4 serve the paper's Top-k baselines, which have no quantiser (appendix on DiLoCo variants):
+// the staged values are added as they are and nothing is packed; FUSE 3 applies theta = fma(-alpha/R,
+// sum, theta) (Alg. 4), FUSE 4 the Nesterov outer step on the average, m = fma(mu, m, avg), theta =
+// fma(-alpha, fma(mu, m, avg), theta), for every element (Alg. 3: the momentum moves everywhere).
+//
 // FUSE 0: the entries come from the payload records (sl_aggregate_apply).  FUSE 1 / 2: the whole outer
 // step is running and the records do not exist yet: the entries come from the staging arrays, get
 // their codes here, and the kernel also writes the records and the error correction (e[index] =
@@ -33,6 +38,9 @@ struct FuseArgs {
     Workspace ws;
     long long n_chunks;
     int n_tensors, kp;
+    // FUSE 4 only: the global outer momentum and its coefficient, alpha and the divisor
+    float* momentum;
+    float mu, alpha, divisor;
 };
 
 constexpr int kApplyWarps = 4;
@@ -59,6 +67,8 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     // per worker of the batch: mean, 3 sigma, 0, present | the four table entries
     float4* tabs = reinterpret_cast<float4*>(recs + (size_t)kApplyBatch * stride);
     constexpr int WB = kApplyPerWarp;
+    constexpr bool PACK = FUSE == 1 || FUSE == 2;  // quantise, write records and the error correction
+    constexpr bool RAW = FUSE >= 3;                // staged values travel unquantised
     const unsigned dump = (unsigned)(kChunk + tid);  // where an entry that does not count adds its 0
     // per-worker strides of the staging arrays, in index pairs / value pairs (kp is a multiple of 8)
     const long long wstride = FUSE ? fa.n_chunks * (long long)fa.kp / 2 : 0;
@@ -94,14 +104,16 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
 
         for (int r0 = 0; r0 < n_workers; r0 += kApplyBatch) {
             const int nb = min(kApplyBatch, n_workers - r0);
-            if (FUSE) {  // the records of this batch start as zeros (unused slots and padding stay zero)
+            if (PACK) {  // the records of this batch start as zeros (unused slots and padding stay zero)
                 for (int v = tid; v < nb * (stride / 16); v += kApplyThreads) reinterpret_cast<uint4*>(recs)[v] = make_uint4(0u, 0u, 0u, 0u);
             }
             if (tid < kApplyBatch) {  // what decodes worker r0 + tid: one load per thread, read back by all below
                 float4 h = make_float4(0.f, 0.f, 0.f, 0.f), t = h;
                 if (tid < nb) {
                     const int r = r0 + tid;
-                    if (FUSE) {
+                    if (RAW) {
+                        h.w = 1.f;
+                    } else if (FUSE) {
                         const float4* st = reinterpret_cast<const float4*>(tstat + (long long)r * fa.n_tensors);
                         const float4 s0 = st[0], s1 = st[1];  // mu, sigma, 3 sigma, table[0] | table[1..3], pad
                         h = make_float4(s0.x, s0.z, 0.f, 1.f);
@@ -158,17 +170,17 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     const int m = lane + 32 * j;
                     unsigned p0 = pos[q][j] & 0xFFFFu, p1 = pos[q][j] >> 16;
                     const bool ok0 = have && in0[j], ok1 = have && in1[j];
-                    unsigned c0, c1;
-                    if (FUSE) {
+                    unsigned c0 = 0, c1 = 0;
+                    if (PACK) {
                         c0 = (unsigned)quant_code(val[q][j].x, mu, t3);
                         c1 = (unsigned)quant_code(val[q][j].y, mu, t3);
-                    } else {
+                    } else if (!RAW) {
                         c0 = __float_as_uint(val[q][j].x);
                         c1 = __float_as_uint(val[q][j].y);
                     }
-                    const float l0 = c0 == 0 ? lut.x : c0 == 1 ? lut.y : c0 == 2 ? lut.z : lut.w;
-                    const float l1 = c1 == 0 ? lut.x : c1 == 1 ? lut.y : c1 == 2 ? lut.z : lut.w;
-                    if (FUSE) {
+                    const float l0 = RAW ? val[q][j].x : c0 == 0 ? lut.x : c0 == 1 ? lut.y : c0 == 2 ? lut.z : lut.w;
+                    const float l1 = RAW ? val[q][j].y : c1 == 0 ? lut.x : c1 == 1 ? lut.y : c1 == 2 ? lut.z : lut.w;
+                    if (PACK) {
                         const float f0 = __fsub_rn(val[q][j].x, l0), f1 = __fsub_rn(val[q][j].y, l1);
                         if (FUSE == 1) {
                             if (ok0 && p0 < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p0)] = f0;
@@ -213,7 +225,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                 }
                 __syncthreads();
             }
-            if (FUSE) {  // the records of the batch are complete (written before the barriers above): out they go
+            if (PACK) {  // the records of the batch are complete (written before the barriers above): out they go
                 const int vpr = stride / 16;
                 for (int v = tid; v < nb * vpr; v += kApplyThreads) {
                     const int rb = v / vpr, w = v - rb * vpr;
@@ -222,7 +234,37 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
             }
         }
 
-        if (full) {
+        if (FUSE == 4) {  // Nesterov outer step on the average: every element moves
+            float* __restrict__ mo = fa.momentum + cd.base;
+            if (full) {
+                float* __restrict__ mo_vec = mo + (long long)(tid >> 4) * rs + 4 * (tid & 15);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float* av = acc + 512 * i + 4 * tid;
+                    const float4 sv = *reinterpret_cast<const float4*>(av);
+                    float4 m = *reinterpret_cast<const float4*>(mo_vec + i * vec_step), o;
+                    const float dx = __fdiv_rn(sv.x, fa.divisor), dy = __fdiv_rn(sv.y, fa.divisor);
+                    const float dz = __fdiv_rn(sv.z, fa.divisor), dw = __fdiv_rn(sv.w, fa.divisor);
+                    m.x = __fmaf_rn(fa.mu, m.x, dx); m.y = __fmaf_rn(fa.mu, m.y, dy);
+                    m.z = __fmaf_rn(fa.mu, m.z, dz); m.w = __fmaf_rn(fa.mu, m.w, dw);
+                    o.x = __fmaf_rn(-fa.alpha, __fmaf_rn(fa.mu, m.x, dx), a[i].x);
+                    o.y = __fmaf_rn(-fa.alpha, __fmaf_rn(fa.mu, m.y, dy), a[i].y);
+                    o.z = __fmaf_rn(-fa.alpha, __fmaf_rn(fa.mu, m.z, dz), a[i].z);
+                    o.w = __fmaf_rn(-fa.alpha, __fmaf_rn(fa.mu, m.w, dw), a[i].w);
+                    *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
+                    *reinterpret_cast<float4*>(mo_vec + i * vec_step) = m;
+                    *reinterpret_cast<float4*>(av) = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            } else {
+                for (int p = tid; p < cd.len; p += kApplyThreads) {
+                    const float d = __fdiv_rn(acc[p], fa.divisor);
+                    const float m = __fmaf_rn(fa.mu, mo[p], d);
+                    th[p] = __fmaf_rn(-fa.alpha, __fmaf_rn(fa.mu, m, d), th[p]);
+                    mo[p] = m;
+                    acc[p] = 0.0f;
+                }
+            }
+        } else if (full) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 float* av = acc + 512 * i + 4 * tid;

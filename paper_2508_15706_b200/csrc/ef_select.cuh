@@ -454,7 +454,9 @@ __device__ __forceinline__ void select_unit(const float (&u)[128], const USource
     else rank_and_emit<kCandCap / 32, GLOBAL>(cand, n_c, T, probe, src, keff, bitmap, out_idx, out_val);
 }
 
-template <bool EF, bool PENDING, bool WIDE>
+// DELTA: the "theta_r" buffers hold the vector to compress itself (a local Nesterov direction, a
+// momentum: the Top-k baselines of Alg. 2 and 4) instead of parameters to subtract from theta.
+template <bool EF, bool PENDING, bool WIDE, bool DELTA = false>
 __global__ void __launch_bounds__(kSelThreads, 1)
 ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                  const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma, int use_tma) {
@@ -516,8 +518,12 @@ ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
                     for (int q = 1; q < tma.n_classes; ++q) cls = tma.class_rs[q] == rs ? q : cls;
                     x2 = (int)(d.base / rs);
                     x1 = (int)(d.base - (long long)x2 * rs) >> 6;
-                    mbar_arrive_expect_tx(&sm.full_s[b], kChunk * (unsigned)sizeof(float));
-                    tma_load_block(sm.theta_s[b], tma.maps + tma.slot_s * tma.n_classes + cls, x1, x2, &sm.full_s[b]);
+                    if (DELTA) {  // nothing is subtracted from theta: its block is not needed
+                        mbar_arrive(&sm.full_s[b]);
+                    } else {
+                        mbar_arrive_expect_tx(&sm.full_s[b], kChunk * (unsigned)sizeof(float));
+                        tma_load_block(sm.theta_s[b], tma.maps + tma.slot_s * tma.n_classes + cls, x1, x2, &sm.full_s[b]);
+                    }
                 } else {
                     mbar_arrive(&sm.full_s[b]);
                 }
@@ -624,13 +630,15 @@ ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const int v = 128 * i + 4 * lane;
-                const float4 a = *reinterpret_cast<const float4*>(&tsm[v]);
                 const float4 l = *reinterpret_cast<const float4*>(&tlm[v]);
-                float4 x;
-                x.x = __fsub_rn(a.x, l.x);
-                x.y = __fsub_rn(a.y, l.y);
-                x.z = __fsub_rn(a.z, l.z);
-                x.w = __fsub_rn(a.w, l.w);
+                float4 x = l;
+                if (!DELTA) {
+                    const float4 a = *reinterpret_cast<const float4*>(&tsm[v]);
+                    x.x = __fsub_rn(a.x, l.x);
+                    x.y = __fsub_rn(a.y, l.y);
+                    x.z = __fsub_rn(a.z, l.z);
+                    x.w = __fsub_rn(a.w, l.w);
+                }
                 if (EF) {
                     const float4 ev = *reinterpret_cast<const float4*>(&em[v]);
                     x.x = __fmaf_rn(beta, ev.x, x.x);
@@ -655,12 +663,15 @@ ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
                 const long long off = chunk_elem_offset(cd.row_stride, p0);
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (p0 + 4 <= cd.len) {
-                    const float4 a = *reinterpret_cast<const float4*>(tsp + off);
                     const float4 l = *reinterpret_cast<const float4*>(tlp + off);
-                    x.x = __fsub_rn(a.x, l.x);
-                    x.y = __fsub_rn(a.y, l.y);
-                    x.z = __fsub_rn(a.z, l.z);
-                    x.w = __fsub_rn(a.w, l.w);
+                    x = l;
+                    if (!DELTA) {
+                        const float4 a = *reinterpret_cast<const float4*>(tsp + off);
+                        x.x = __fsub_rn(a.x, l.x);
+                        x.y = __fsub_rn(a.y, l.y);
+                        x.z = __fsub_rn(a.z, l.z);
+                        x.w = __fsub_rn(a.w, l.w);
+                    }
                     if (EF) {
                         const float4 ev = *reinterpret_cast<const float4*>(er + off);
                         x.x = __fmaf_rn(beta, ev.x, x.x);
@@ -674,7 +685,7 @@ ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (p0 + j < cd.len) {
-                            t[j] = __fsub_rn(tsp[off + j], tlp[off + j]);
+                            t[j] = DELTA ? tlp[off + j] : __fsub_rn(tsp[off + j], tlp[off + j]);
                             if (EF) {
                                 t[j] = __fmaf_rn(beta, er[off + j], t[j]);
                                 er[off + j] = t[j];

@@ -54,7 +54,10 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
 }
 
 // Writes the corrected values waiting in the staging arrays into the error buffers (deferred
-// subtraction made good).  One warp per (worker, chunk).
+// subtraction made good).  One warp per (worker, chunk).  ZERO: writes +0 at the staged positions
+// instead (Top-k without a quantiser sends the selected values exactly, so what stays behind there,
+// u - Top-k(u), is zero: Alg. 2-4 of the appendix on DiLoCo variants).
+template <bool ZERO>
 __global__ void __launch_bounds__(128)
 ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, Workspace ws,
                 WorkerPtrs ptrs) {
@@ -69,7 +72,8 @@ ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const long long slot_base = ((long long)r * n_chunks + g) * kp;
     for (int s = lane; s < keff; s += 32) {
         const unsigned p = ws.idx[slot_base + s];
-        if (p < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = ws.val[slot_base + s];
+        if (p < (unsigned)cd.len)
+            ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = ZERO ? 0.0f : ws.val[slot_base + s];
     }
 }
 

@@ -206,8 +206,83 @@ sl_status order_after_map_uploads(sl_ctx* c, cudaStream_t st) {
 sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
     const int R = c->cfg.R;
     const Workspace ws = carve(c, R);
-    ef_flush_kernel<<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp, ws,
-                                                                    ptrs);
+    ef_flush_kernel<false><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
+                                                                           ws, ptrs);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+// The waiting values of a deferred subtraction go into the buffers of the step that left them.
+sl_status flush_pending(sl_ctx* c, cudaStream_t st) {
+    if (!c->pending) return SL_OK;
+    WorkerPtrs fp;
+    memset(&fp, 0, sizeof(fp));
+    for (int r = 0; r < c->cfg.R; ++r) fp.e[r] = c->pending_e[r];
+    sl_status s = launch_flush(c, fp, st);
+    if (s == SL_OK) c->pending = false;
+    return s;
+}
+
+// Kernel 1 for `workers` workers: u (from theta - theta_r, or with `delta` from the vectors in the
+// theta_local slots themselves), error feedback when `ef`, chunk-wise Top-k into the staging arrays.
+// `consume`: substitute the waiting values of a deferred subtraction on the way.
+sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const WorkerPtrs& ptrs, cudaStream_t st,
+                        bool ef, bool consume, bool delta) {
+    const Workspace ws = carve(c, workers);
+    const long long G = c->n_chunks;
+    const int k = c->cfg.k, kp = c->kp;
+    // tile copies through tensor maps when the table allows it and every buffer got its maps
+    TmaArgs ta;
+    memset(&ta, 0, sizeof(ta));
+    ta.status = c->d_status;
+    bool use_tma = c->tma_on;
+    if (use_tma) {
+        ta.maps = c->d_maps;
+        ta.n_classes = c->n_classes;
+        for (int q = 0; q < c->n_classes; ++q) ta.class_rs[q] = c->class_rs[q];
+        for (int pass = 0; pass < 2 && use_tma; ++pass) {
+            // if the slot table fills up half-way, it is emptied and the assignment starts over: one
+            // call needs at most 2 R + 1 slots, which an empty table holds
+            c->slots_cleared = false;
+            ta.slot_s = delta ? 0 : tma_map_slot(c, theta_sync, st);
+            use_tma = ta.slot_s >= 0;
+            for (int r = 0; r < workers && use_tma; ++r) {
+                ta.slot_l[r] = tma_map_slot(c, ptrs.theta_local[r], st);
+                ta.slot_e[r] = ef ? tma_map_slot(c, ptrs.e[r], st) : 0;
+                use_tma = ta.slot_l[r] >= 0 && ta.slot_e[r] >= 0;
+            }
+            if (!c->slots_cleared) break;
+        }
+        if (use_tma) {
+            sl_status s = order_after_map_uploads(c, st);
+            if (s != SL_OK) return s;
+            ta.fresh = c->maps_fresh ? 1 : 0;
+            c->maps_fresh = false;
+        }
+    }
+    // one persistent CTA per SM
+    const unsigned grid = (unsigned)(G < c->n_sms ? G : c->n_sms);
+    const int tm = use_tma ? 1 : 0;
+#define SL_LAUNCH_SELECT(EFV, PENDV, DELTAV)                                                                         \
+    do {                                                                                                             \
+        if (k > kSelNarrowMaxK)                                                                                      \
+            ef_select_kernel<EFV, PENDV, true, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                  \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
+        else                                                                                                         \
+            ef_select_kernel<EFV, PENDV, false, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                 \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
+    } while (0)
+    if (delta) {
+        if (ef) SL_LAUNCH_SELECT(true, false, true);
+        else SL_LAUNCH_SELECT(false, false, true);
+    } else if (!ef) {
+        SL_LAUNCH_SELECT(false, false, false);
+    } else if (consume) {
+        SL_LAUNCH_SELECT(true, true, false);
+    } else {
+        SL_LAUNCH_SELECT(true, false, false);
+    }
+#undef SL_LAUNCH_SELECT
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -228,63 +303,17 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     if (c->pending) {
         if (ef && defer) {
             consume = true;
+            c->pending = false;
         } else {  // nothing will read them in flight (frozen step): write them out first
-            WorkerPtrs fp;
-            memset(&fp, 0, sizeof(fp));
-            for (int r = 0; r < c->cfg.R; ++r) fp.e[r] = c->pending_e[r];
-            sl_status s = launch_flush(c, fp, st);
+            sl_status s = flush_pending(c, st);
             if (s != SL_OK) return s;
-        }
-        c->pending = false;
-    }
-
-    // tile copies through tensor maps when the table allows it and every buffer got its maps
-    TmaArgs ta;
-    memset(&ta, 0, sizeof(ta));
-    ta.status = c->d_status;
-    bool use_tma = c->tma_on;
-    if (use_tma) {
-        ta.maps = c->d_maps;
-        ta.n_classes = c->n_classes;
-        for (int q = 0; q < c->n_classes; ++q) ta.class_rs[q] = c->class_rs[q];
-        for (int pass = 0; pass < 2 && use_tma; ++pass) {
-            // if the slot table fills up half-way, it is emptied and the assignment starts over: one
-            // call needs at most 2 R + 1 slots, which an empty table holds
-            c->slots_cleared = false;
-            ta.slot_s = tma_map_slot(c, theta_sync, st);
-            use_tma = ta.slot_s >= 0;
-            for (int r = 0; r < workers && use_tma; ++r) {
-                ta.slot_l[r] = tma_map_slot(c, ptrs.theta_local[r], st);
-                ta.slot_e[r] = ef ? tma_map_slot(c, ptrs.e[r], st) : 0;
-                use_tma = ta.slot_l[r] >= 0 && ta.slot_e[r] >= 0;
-            }
-            if (!c->slots_cleared) break;
-        }
-        if (use_tma) {
-            sl_status s = order_after_map_uploads(c, st);
-            if (s != SL_OK) return s;
-            ta.fresh = c->maps_fresh ? 1 : 0;
-            c->maps_fresh = false;
         }
     }
 
     prof_mark(c, -1, st);
-    {   // one persistent CTA per SM
-        const unsigned grid = (unsigned)(G < c->n_sms ? G : c->n_sms);
-        const int tm = use_tma ? 1 : 0;
-#define SL_LAUNCH_SELECT(EFV, PENDV)                                                                                  \
-    do {                                                                                                             \
-        if (k > kSelNarrowMaxK)                                                                                      \
-            ef_select_kernel<EFV, PENDV, true><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                          \
-                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
-        else                                                                                                         \
-            ef_select_kernel<EFV, PENDV, false><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                         \
-                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
-    } while (0)
-        if (!ef) SL_LAUNCH_SELECT(false, false);
-        else if (consume) SL_LAUNCH_SELECT(true, true);
-        else SL_LAUNCH_SELECT(true, false);
-#undef SL_LAUNCH_SELECT
+    {
+        sl_status s = launch_select(c, workers, theta_sync, ptrs, st, ef, consume, false);
+        if (s != SL_OK) return s;
     }
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
@@ -319,8 +348,9 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
 }
 
 // fuse: 0 = payloads in, 1 / 2 = also do the packing step of a compression in flight (see the kernel)
+// fuse 3 / 4: the Top-k baselines (raw staged values; 4 = Nesterov outer step with `momentum`, `mu`)
 sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* theta_sync, cudaStream_t st, int fuse = 0,
-                       const WorkerPtrs* fuse_ptrs = nullptr) {
+                       const WorkerPtrs* fuse_ptrs = nullptr, float* momentum = nullptr, float mu = 0.0f) {
     if (present == 0) return SL_OK;
     const int R = c->cfg.R;
     const double D = c->cfg.divide_by_present ? (double)present : (double)R;
@@ -336,7 +366,11 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
         fa.n_chunks = c->n_chunks;
         fa.n_tensors = c->n_tensors;
         fa.kp = c->kp;
-        wp = *fuse_ptrs;
+        fa.momentum = momentum;
+        fa.mu = mu;
+        fa.alpha = c->cfg.outer_lr;
+        fa.divisor = (float)D;
+        if (fuse_ptrs) wp = *fuse_ptrs;
     }
     // persistent CTAs: as many as are resident at once
     const long long resident = (long long)c->n_sms * kApplyCtasPerSm;
@@ -344,7 +378,9 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
 #define SL_APPLY(PPLV)                                                                                          \
     do {                                                                                                        \
         auto kern = fuse == 0 ? decode_avg_apply_kernel<PPLV, 0>                                                \
-                  : fuse == 1 ? decode_avg_apply_kernel<PPLV, 1> : decode_avg_apply_kernel<PPLV, 2>;            \
+                  : fuse == 1 ? decode_avg_apply_kernel<PPLV, 1>                                                \
+                  : fuse == 2 ? decode_avg_apply_kernel<PPLV, 2>                                                \
+                  : fuse == 3 ? decode_avg_apply_kernel<PPLV, 3> : decode_avg_apply_kernel<PPLV, 4>;            \
         kern<<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
     } while (0)
     if (ppl <= 1) SL_APPLY(1);
@@ -529,15 +565,21 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     SL_SELECT_ATTR(true, false, false); SL_SELECT_ATTR(true, true, false); SL_SELECT_ATTR(false, false, false);
     SL_SELECT_ATTR(true, false, true); SL_SELECT_ATTR(true, true, true); SL_SELECT_ATTR(false, false, true);
 #undef SL_SELECT_ATTR
+#define SL_SELECT_ATTR_D(EFV, WIDEV)                                                                                 \
+    if (e == cudaSuccess)                                                                                            \
+        e = cudaFuncSetAttribute(ef_select_kernel<EFV, false, WIDEV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 (int)sizeof(SelSmem))
+    SL_SELECT_ATTR_D(true, false); SL_SELECT_ATTR_D(false, false); SL_SELECT_ATTR_D(true, true); SL_SELECT_ATTR_D(false, true);
+#undef SL_SELECT_ATTR_D
     per_sm = 1;
     {   // the apply kernel's shared memory depends on k alone: sized once
         const int asz = (int)apply_smem_bytes(cfg->k);
 #define SL_APPLY_ATTR(PPLV, FUSEV)                                                                                     \
     if (e == cudaSuccess)                                                                                              \
         e = cudaFuncSetAttribute(decode_avg_apply_kernel<PPLV, FUSEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, asz)
-        SL_APPLY_ATTR(1, 0); SL_APPLY_ATTR(1, 1); SL_APPLY_ATTR(1, 2);
-        SL_APPLY_ATTR(2, 0); SL_APPLY_ATTR(2, 1); SL_APPLY_ATTR(2, 2);
-        SL_APPLY_ATTR(4, 0); SL_APPLY_ATTR(4, 1); SL_APPLY_ATTR(4, 2);
+        SL_APPLY_ATTR(1, 0); SL_APPLY_ATTR(1, 1); SL_APPLY_ATTR(1, 2); SL_APPLY_ATTR(1, 3); SL_APPLY_ATTR(1, 4);
+        SL_APPLY_ATTR(2, 0); SL_APPLY_ATTR(2, 1); SL_APPLY_ATTR(2, 2); SL_APPLY_ATTR(2, 3); SL_APPLY_ATTR(2, 4);
+        SL_APPLY_ATTR(4, 0); SL_APPLY_ATTR(4, 1); SL_APPLY_ATTR(4, 2); SL_APPLY_ATTR(4, 3); SL_APPLY_ATTR(4, 4);
 #undef SL_APPLY_ATTR
     }
     c->n_sms = n_sms;
@@ -812,6 +854,135 @@ sl_status sl_diloco_step(sl_ctx* c, float* theta_sync, const float* const* theta
         c->d_chunks, c->cfg.R, beta_outer, c->cfg.outer_lr, theta_sync, lp, momentum);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
+}
+
+namespace {
+
+// Writes +0 at the staged positions of every worker's buffer in `bufs` (what Top-k leaves behind there).
+sl_status launch_zero_selected(sl_ctx* c, float* const* bufs, cudaStream_t st) {
+    const int R = c->cfg.R;
+    WorkerPtrs zp;
+    memset(&zp, 0, sizeof(zp));
+    for (int r = 0; r < R; ++r) zp.e[r] = bufs[r];
+    ef_flush_kernel<true><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
+                                                                          carve(c, R), zp);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+// Common argument checks of the three baseline steps; fills the pointer tables.
+sl_status variant_args(sl_ctx* c, const float* theta_sync, const float* const* theta_local, float* const* e,
+                       float* const* m_r, float mu, WorkerPtrs& ptrs) {
+    if (!c || !theta_sync || !theta_local) return SL_ERR_INVALID_ARG;
+    if (!(mu >= 0.0f && mu <= 1.0f)) return SL_ERR_INVALID_ARG;
+    if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
+    memset(&ptrs, 0, sizeof(ptrs));
+    for (int r = 0; r < c->cfg.R; ++r) {
+        if (!theta_local[r] || (e && !e[r]) || (m_r && !m_r[r])) return SL_ERR_INVALID_ARG;
+        if (misaligned(theta_local[r]) || (e && misaligned(e[r])) || (m_r && misaligned(m_r[r]))) return SL_ERR_ALIGNMENT;
+        for (int q = 0; q < r; ++q)
+            if ((e && e[q] == e[r]) || (m_r && m_r[q] == m_r[r])) return SL_ERR_INVALID_ARG;
+        ptrs.theta_local[r] = theta_local[r];
+        ptrs.e[r] = e ? e[r] : nullptr;
+    }
+    return SL_OK;
+}
+
+}  // namespace
+
+sl_status sl_lom_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* m_r, float mu,
+                      int32_t sub_k, void* stream) {
+    WorkerPtrs ptrs;
+    if (!m_r) return SL_ERR_INVALID_ARG;
+    sl_status s = variant_args(c, theta_sync, theta_local, nullptr, m_r, mu, ptrs);
+    if (s != SL_OK) return s;
+    if (sub_k && (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R))) return SL_ERR_NOMEM;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int R = c->cfg.R;
+    MutableLocalPtrs lp;
+    MomentumPtrs mp;
+    memset(&lp, 0, sizeof(lp));
+    memset(&mp, 0, sizeof(mp));
+    for (int r = 0; r < R; ++r) {
+        lp.p[r] = const_cast<float*>(theta_local[r]);  // the stepping kernel only reads them
+        mp.p[r] = m_r[r];
+    }
+    lom_kernel<true><<<(unsigned)c->n_chunks, kThreads, 0, st>>>(c->d_chunks, R, mu, c->cfg.outer_lr, theta_sync, lp, mp);
+    SL_CUDA(cudaGetLastError());
+    if (sub_k) {  // m_r <- m_r - Top-k(m_r): select on the momenta themselves, zero what was selected
+        if ((s = flush_pending(c, st)) != SL_OK) return s;
+        WorkerPtrs sel;
+        memset(&sel, 0, sizeof(sel));
+        for (int r = 0; r < R; ++r) sel.theta_local[r] = m_r[r];
+        if ((s = launch_select(c, R, theta_sync, sel, st, false, false, true)) != SL_OK) return s;
+        return launch_zero_selected(c, m_r, st);
+    }
+    return SL_OK;
+}
+
+sl_status sl_diloco_topk_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+                              float* momentum, float mu, void* stream) {
+    WorkerPtrs ptrs;
+    if (!momentum) return SL_ERR_INVALID_ARG;
+    sl_status s = variant_args(c, theta_sync, theta_local, e, nullptr, mu, ptrs);
+    if (s != SL_OK) return s;
+    if (misaligned(momentum)) return SL_ERR_ALIGNMENT;
+    if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R)) return SL_ERR_NOMEM;
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((s = flush_pending(c, st)) != SL_OK) return s;
+    const int R = c->cfg.R;
+    c->last_workers = R;
+    if ((s = launch_select(c, R, theta_sync, ptrs, st, e != nullptr, false, false)) != SL_OK) return s;
+    if (e && (s = launch_zero_selected(c, e, st)) != SL_OK) return s;  // e_r = u_r - Top-k(u_r)
+    PayloadPtrs none;
+    memset(&none, 0, sizeof(none));
+    const int was = c->cfg.divide_by_present;
+    c->cfg.divide_by_present = 0;  // Alg. 3 averages over all R workers
+    s = launch_apply(c, none, R, theta_sync, st, 4, nullptr, momentum, mu);
+    c->cfg.divide_by_present = was;
+    return s;
+}
+
+sl_status sl_lom_topk_step(sl_ctx* c, float* theta_sync, float* const* theta_local, float* const* m_r, float* const* e,
+                           float mu, void* stream) {
+    WorkerPtrs ptrs;
+    if (!m_r) return SL_ERR_INVALID_ARG;
+    sl_status s = variant_args(c, theta_sync, theta_local, e, m_r, mu, ptrs);
+    if (s != SL_OK) return s;
+    if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R)) return SL_ERR_NOMEM;
+    const int R = c->cfg.R;
+    for (int r = 0; r < R; ++r)
+        for (int q = 0; q < r; ++q)
+            if (theta_local[q] == theta_local[r]) return SL_ERR_INVALID_ARG;  // they are written here
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((s = flush_pending(c, st)) != SL_OK) return s;
+    c->last_workers = R;
+    MutableLocalPtrs lp;
+    MomentumPtrs mp;
+    memset(&lp, 0, sizeof(lp));
+    memset(&mp, 0, sizeof(mp));
+    for (int r = 0; r < R; ++r) {
+        lp.p[r] = theta_local[r];
+        mp.p[r] = m_r[r];
+    }
+    // local momenta, and the local Nesterov directions in place of theta_r
+    lom_kernel<false><<<(unsigned)c->n_chunks, kThreads, 0, st>>>(c->d_chunks, R, mu, c->cfg.outer_lr, theta_sync, lp, mp);
+    SL_CUDA(cudaGetLastError());
+    if ((s = launch_select(c, R, theta_sync, ptrs, st, e != nullptr, false, true)) != SL_OK) return s;
+    if (e && (s = launch_zero_selected(c, e, st)) != SL_OK) return s;
+    PayloadPtrs none;
+    memset(&none, 0, sizeof(none));
+    const int was = c->cfg.divide_by_present;
+    c->cfg.divide_by_present = 0;
+    s = launch_apply(c, none, R, theta_sync, st, 3);
+    c->cfg.divide_by_present = was;
+    return s;
 }
 
 sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {

@@ -1,0 +1,130 @@
+"""GPU parity for the paper's Top-k / local-outer-momentum variants (Sec. 3.2; appendix "Exact algorithmic
+description of DiLoCo variants", Alg. 2-4) against the CPU oracle, through the C ABI.  What a worker keeps
+(m_r, e_r) is formed by the same single-rounded fp32 operations on both sides and must be bit-exact, and
+with it the Top-k selections; theta and the global momentum (fp32 recipe on the GPU, fp64 in the oracle)
+within 1e-6 x RMS of the tensor."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2508_15706_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+TENSORS = [I.TensorSpec("a", 128, 192, 0), I.TensorSpec("flat", 1, 5000, 0), I.TensorSpec("router", 8, 1024, 1),
+           I.TensorSpec("norm", 1, 768, 1), I.TensorSpec("tiny", 1, 40, 2), I.TensorSpec("b", 192, 64, 3)]
+TOL = 1e-6
+
+
+def _setup(R, k, seed):
+    from paper_2508_15706_b200.binding import SparseLoCo
+    O.set_threads(8)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    wl = I.Workload("variants", TENSORS, R=R, k=k, recipe="student_t4", seed=seed, outer_lr=0.7, beta=0.9)
+    shapes, offs = [(t.rows, t.cols) for t in TENSORS], I.offsets(TENSORS)
+    sl = SparseLoCo(shapes, offs, k=k, R=R, beta=wl.beta, outer_lr=wl.outer_lr)
+    cfg = O.Config(k=k, R=R, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=32)
+    tab = O.Table(shapes, offs)
+    theta = I.theta_sync(wl, dev)
+    return wl, sl, cfg, tab, theta, dev
+
+
+def _close(got: torch.Tensor, want: np.ndarray, what, ulps: float = 0.0):
+    """Max-abs error within 1e-6 x RMS of the tensor; with `ulps`, plus that many fp32 units in the last
+    place of the element (the global momentum is heavy-tailed -- a few selected entries are far above its
+    RMS -- and the fp32 recipe rounds it twice per step, the fp64 evaluation once)."""
+    offs = I.offsets(TENSORS)
+    g = got.cpu().numpy().astype(np.float64)
+    for t, off in zip(TENSORS, offs):
+        w = want[off:off + t.numel].astype(np.float64)
+        rms = float(np.sqrt(np.mean(w ** 2)))
+        err = np.abs(g[off:off + t.numel] - w)
+        bound = TOL * rms + ulps * 2.0 ** -23 * np.abs(w) + 1e-30
+        assert np.all(err <= bound), (what, t.name, float(err.max()), rms)
+
+
+def _bits_equal(got: torch.Tensor, want: np.ndarray, what):
+    assert np.array_equal(got.cpu().numpy().view(np.uint32), want.view(np.uint32)), what
+
+
+@pytest.mark.parametrize("sub_k", [False, True])
+def test_lom_step_alg2(sub_k):
+    wl, sl, cfg, tab, theta, dev = _setup(R=3, k=64, seed=61)
+    m = [I.initial_error(wl, r, dev, scale=0.3) for r in range(3)]
+    th_o, m_o = theta.cpu().numpy().copy(), [x.cpu().numpy().copy() for x in m]
+    for step in range(3):
+        local = [I.theta_local(wl, theta, r, step) for r in range(3)]
+        O.lom_step(cfg, tab, th_o, [(x.cpu().numpy()) for x in local], m_o, 0.9, sub_k=sub_k)
+        sl.lom_step(theta, local, m, 0.9, sub_k=sub_k)
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
+        for r in range(3):
+            _bits_equal(m[r], m_o[r], ("m", step, r))
+        _close(theta, th_o, ("theta", step))
+        theta.copy_(torch.from_numpy(th_o))  # both sides continue from the same parameters
+
+
+@pytest.mark.parametrize("use_ef,k", [(False, 64), (True, 64), (True, 41), (True, 200)])
+def test_diloco_topk_step_alg3(use_ef, k):
+    wl, sl, cfg, tab, theta, dev = _setup(R=4, k=k, seed=62)
+    e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(4)] if use_ef else None
+    mom = I.initial_error(wl, 9, dev, scale=0.2)
+    th_o, mom_o = theta.cpu().numpy().copy(), mom.cpu().numpy().copy()
+    e_o = [x.cpu().numpy().copy() for x in e] if use_ef else None
+    for step in range(3):
+        local = [I.theta_local(wl, theta, r, step) for r in range(4)]
+        O.diloco_topk_step(cfg, tab, th_o, [x.cpu().numpy() for x in local], e_o, mom_o, 0.8)
+        sl.diloco_topk_step(theta, local, e, mom, 0.8)
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
+        if use_ef:
+            for r in range(4):
+                _bits_equal(e[r], e_o[r], ("e", step, r))
+        _close(theta, th_o, ("theta", step))
+        _close(mom, mom_o, ("momentum", step), ulps=2.0)
+        theta.copy_(torch.from_numpy(th_o))
+        mom.copy_(torch.from_numpy(mom_o))
+
+
+@pytest.mark.parametrize("use_ef", [False, True])
+def test_lom_topk_step_alg4(use_ef):
+    wl, sl, cfg, tab, theta, dev = _setup(R=3, k=64, seed=63)
+    e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(3)] if use_ef else None
+    m = [I.initial_error(wl, 20 + r, dev, scale=0.3) for r in range(3)]
+    th_o = theta.cpu().numpy().copy()
+    m_o = [x.cpu().numpy().copy() for x in m]
+    e_o = [x.cpu().numpy().copy() for x in e] if use_ef else None
+    for step in range(3):
+        local = [I.theta_local(wl, theta, r, step) for r in range(3)]
+        O.lom_topk_step(cfg, tab, th_o, [x.cpu().numpy() for x in local], m_o, e_o, 0.6)
+        sl.lom_topk_step(theta, local, m, e, 0.6)   # consumes `local`
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
+        for r in range(3):
+            _bits_equal(m[r], m_o[r], ("m", step, r))
+            if use_ef:
+                _bits_equal(e[r], e_o[r], ("e", step, r))
+        _close(theta, th_o, ("theta", step))
+        theta.copy_(torch.from_numpy(th_o))
+
+
+def test_alg3_with_ef_and_no_momentum_equals_the_outer_step_without_quantiser_on_the_gpu():
+    """The reduction the paper's construction rests on, through the library: DiLoCo + Top-k + EF with
+    mu = 0 leaves the same error buffers as SparseLoCo's step (whose Top-k selection it shares; the
+    quantiser only changes what is sent), i.e. e differs exactly at the selected positions."""
+    wl, sl, cfg, tab, theta, dev = _setup(R=2, k=64, seed=64)
+    e_a = [I.initial_error(wl, r, dev, scale=0.5) for r in range(2)]
+    e_b = [x.clone() for x in e_a]
+    local = [I.theta_local(wl, theta, r, 0) for r in range(2)]
+    th_a, th_b = theta.clone(), theta.clone()
+    mom = torch.zeros_like(theta)
+    pay = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(2)]
+    sl.diloco_topk_step(th_a, local, e_a, mom, 0.0)
+    sl.outer_step(th_b, local, e_b, pay)
+    torch.cuda.synchronize()
+    chunks, slots = sl.num_chunks()
+    for r in range(2):
+        differ = (e_a[r].view(torch.int32) != e_b[r].view(torch.int32))
+        assert int(differ.sum()) <= slots                  # only selected entries can differ
+        assert bool((e_a[r][differ] == 0).all())           # and without a quantiser nothing stays behind there
