@@ -32,9 +32,10 @@ METRIC = "sparseloco_outer_step_params_per_s"
 UNIT = "params/s"
 DEFAULT_WORKLOAD = "c5_dense_d2048"
 
-# DRAM bytes per ef_topk launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
-# on a smaller case of the same kernel, as bytes per (parameter x worker); see profiles/.
-NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER = 12.551  # profiles/ncu_full_c5_layer0_top3_kernels.md
+# DRAM bytes per ef_select_kernel launch counted by ncu (dram__bytes_read.sum + dram__bytes_write.sum) on one
+# decoder layer of the same model, as bytes per (parameter x worker): 13.3245 GB / (67,112,960 x 16).
+# Set to None whenever the kernel changes until the counters are taken again.
+NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER = 12.409
 
 
 def record_stride(k: int) -> int:
@@ -449,6 +450,7 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
     torch.cuda.empty_cache()
 
     import dataclasses
+    out["variants_c5_l12_R8"] = variants_bench(torch, I, dev, build, peak)
     wl = dataclasses.replace(I.workload(DEFAULT_WORKLOAD), R=8)
     N = wl.numel
     sl, ws, theta, e, payloads = build(wl)
@@ -469,6 +471,47 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
         "ms_per_step": step_ms, "params_per_s": N / (step_ms * 1e-3),
         "step_gbs": algorithmic_bytes_per_param(8, wl.k) * N / (step_ms * 1e-3) / 1e9}
     del sl, ws, theta, e, payloads, storage, views
+    torch.cuda.empty_cache()
+    return out
+
+
+def variants_bench(torch, I, dev, build, peak: float) -> dict:
+    """The paper's Top-k / local-outer-momentum variants (its appendix on DiLoCo variants, Alg. 2-4) on the
+    12-layer stack with R = 8 (their per-worker momenta need R more model-sized buffers): ms per step and
+    the rate on each step's algorithmic bytes per parameter."""
+    import dataclasses
+    wl = dataclasses.replace(I.workload("c5_l12"), R=8)
+    N, R = wl.numel, 8
+    sl, ws, theta, e, payloads = build(wl)
+    sl.set_ef_deferred(False)
+    local = [I.theta_local(wl, theta, r, 0) for r in range(R)]
+    m_r = [I.initial_error(wl, 100 + r, dev, scale=0.3) for r in range(R)]
+    mom = I.initial_error(wl, 99, dev, scale=0.3)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps=3):
+        fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    pay = 2 * 6 * wl.k / 4096.0  # staged (index, value) pairs written and read, per worker and parameter
+    rows = {
+        "lom_step (Alg. 2)": (lambda: sl.lom_step(theta, local, m_r, 0.9), 12 * R + 8),
+        "lom_step sub_k (Alg. 2, Sub-k)": (lambda: sl.lom_step(theta, local, m_r, 0.9, sub_k=True), 16 * R + 8 + R * pay / 2),
+        "diloco_topk_step with EF (Alg. 3)": (lambda: sl.diloco_topk_step(theta, local, e, mom, 0.9), 12 * R + 4 + 16 + R * pay),
+        "lom_topk_step with EF (Alg. 4)": (lambda: sl.lom_topk_step(theta, local, m_r, e, 0.9), 28 * R + 12 + R * pay),
+    }
+    out = {"params": N, "R": R, "k": wl.k}
+    for name, (fn, bpp) in rows.items():
+        ms = timed(fn)
+        out[name] = {"ms_per_step": ms, "algorithmic_bytes_per_param": bpp, "gbs": bpp * N / (ms * 1e-3) / 1e9,
+                     "frac_of_measured_peak": bpp * N / (ms * 1e-3) / 1e9 / peak}
+    del sl, ws, theta, e, payloads, local, m_r, mom
     torch.cuda.empty_cache()
     return out
 
