@@ -33,9 +33,9 @@ UNIT = "params/s"
 DEFAULT_WORKLOAD = "c5_dense_d2048"
 
 # DRAM bytes per ef_select_kernel launch counted by ncu (dram__bytes_read.sum + dram__bytes_write.sum) on one
-# decoder layer of the same model, as bytes per (parameter x worker): 13.3245 GB / (67,112,960 x 16).
+# decoder layer of the same model, as bytes per (parameter x worker): 13.3264 GB / (67,112,960 x 16).
 # Set to None whenever the kernel changes until the counters are taken again.
-NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER = 12.409
+NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER = 12.410
 
 
 def record_stride(k: int) -> int:
