@@ -213,17 +213,19 @@ sl_status sl_encode_payload(sl_ctx* ctx, const uint8_t* payload, uint8_t* coded,
 sl_status sl_decode_payload(sl_ctx* ctx, const uint8_t* coded, size_t coded_bytes, uint8_t* payload,
                             void* cuda_stream);
 
-/* How the compression kernel moves the 64x64 blocks of theta_r and e (no counterpart in the paper).
- * 1: one tensor-map (TMA) block copy per block and direction, completion on shared-memory barriers --
- * the default whenever every full chunk starts on a 64-element boundary of the flat buffers (tensor
- * offsets that are multiples of 64) and the table has at most 8 distinct row lengths; else
- * UNSUPPORTED.  0: 16-byte asynchronous copies issued by every thread (works for any table).  Results
- * are identical.  The tensor maps of a buffer are built the first time its pointer is passed in.
+/* How the compression kernel moves the 64x64 blocks of theta, theta_r and e (no counterpart in the paper).
+ * 1: one tensor-map (TMA) block copy per block, issued by a producer thread, completion on
+ * shared-memory barriers -- the default whenever every full chunk starts on a 64-element boundary of
+ * the flat buffers (tensor offsets that are multiples of 64) and the table has at most 8 distinct row
+ * lengths; else UNSUPPORTED.  0: every chunk is read and written with plain 128-bit loads and stores by
+ * the warp that processes it (works for any table; short tail chunks always go this way).  Results are
+ * identical.  The tensor maps of a buffer are built the first time its pointer is passed in.
  *
- * The block-copy kernel waits for its copies with a bounded number of polls; if a wait ever runs
- * out the kernel records SL_ERR_TIMEOUT in a device status word and returns early, leaving e and the
- * staged selection of that call undefined.  sl_device_status() synchronises the stream, returns the
- * recorded status (SL_OK when nothing went wrong) and clears it. */
+ * The kernel waits for its copies with a bounded number of polls; if a wait ever runs out the kernel
+ * records SL_ERR_TIMEOUT in a device status word and returns early, leaving e and the staged selection
+ * of that call undefined.  sl_device_status() synchronises the stream, returns the recorded status
+ * (SL_OK when nothing went wrong; SL_ERR_BAD_PAYLOAD after sl_decode_payload met a damaged input) and
+ * clears it. */
 sl_status sl_set_tile_copies(sl_ctx* ctx, int32_t use_tensor_maps);
 sl_status sl_device_status(sl_ctx* ctx, void* cuda_stream);
 
