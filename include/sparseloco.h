@@ -48,7 +48,7 @@ typedef enum {
     SL_OK = 0,
     SL_ERR_INVALID_ARG = 1, /* NULL pointer, size or hyper-parameter out of range */
     SL_ERR_ALIGNMENT = 2,   /* a device pointer or tensor offset is not 16-byte aligned */
-    SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, bits != 2, ...) */
+    SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, bits other than 2 / 32, ...) */
     SL_ERR_BAD_PAYLOAD = 4, /* reported through the device status word of sl_validate_payload */
     SL_ERR_CUDA = 5,        /* a CUDA runtime call failed; see sl_last_cuda_error() */
     SL_ERR_NOMEM = 6,       /* workspace missing or too small; host allocation failed */
@@ -72,7 +72,8 @@ typedef struct {
     int32_t H;                 /* inner steps; carried for the caller, >= 1, unused by the math */
     float beta;                /* error-feedback decay, 0 <= beta <= 1 */
     float outer_lr;            /* alpha, finite */
-    int32_t quant_bits;        /* must be 2 */
+    int32_t quant_bits;        /* 2; or 32 = no quantiser: the selected values are averaged as they are
+                                  (sl_outer_step only: there is no payload format, payloads may be NULL) */
     int32_t ef_enabled;        /* 0 during the error-feedback freeze (App. "Freezing Error
                                   Feedback"): u = Delta and e is neither read nor written */
     int32_t divide_by_present; /* 0: average divides by R (Alg. 1); 1: by the payloads present */
@@ -261,6 +262,16 @@ sl_status sl_ef_flush(sl_ctx* ctx, float* const* e, int32_t keep_pending, void* 
 sl_status sl_outer_step_host(sl_ctx* ctx, float* theta_sync, const float* const* theta_local_host,
                              float* dev_stage, size_t stage_elems, float* const* e,
                              uint8_t* const* payloads, float* theta_sync_host, void* cuda_stream);
+
+/* Streaming SparseLoCo (App. "Streaming SparseLoCo": the model is cut into P fragments, each still
+ * synchronised every H inner steps, but in turn, so that a P-th of the payload travels every H / P
+ * steps).  A fragment is a context of its own whose tensor offsets point into the same flat buffers;
+ * this host-side helper is the schedule: after `inner_step` inner steps (counted from 1) fragment
+ *     p  is due  iff  inner_step mod H == ((p + 1) * H / P) mod H          (integer division),
+ * i.e. fragment 0 first, after H / P steps, fragment P - 1 at every multiple of H.  Writes the due
+ * fragment to *fragment, or -1 when none is.  Errors: INVALID_ARG (NULL, H < 1, P < 1, P > H,
+ * inner_step < 1). */
+sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fragment);
 
 /* Check one payload before trusting it: every index < chunk length and strictly ascending over
  * the used slots, unused slots and padding zero, table entries finite.  Writes SL_OK or

@@ -19,7 +19,7 @@ EXPORTS = (
     "sl_create", "sl_destroy", "sl_set_hyper", "sl_record_stride", "sl_payload_bytes", "sl_num_chunks",
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
-    "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step",
+    "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step", "sl_streaming_due",
 )
 PROFILE_SLOTS = 9
 
@@ -86,6 +86,7 @@ def _load():
     L.sl_ef_pending.argtypes = [P, C.POINTER(C.c_int32)]
     L.sl_ef_flush.argtypes = [P, P, C.c_int32, P]
     L.sl_read_stats.argtypes = [P, C.c_int32, P, P]
+    L.sl_streaming_due.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.POINTER(C.c_int32)]
     L.sl_strerror.argtypes = [C.c_int]
     L.sl_strerror.restype = C.c_char_p
     L.sl_last_cuda_error.restype = C.c_char_p
@@ -125,6 +126,13 @@ def _stream() -> int:
 
 def record_stride(k: int) -> int:
     return _L.sl_record_stride(k)
+
+
+def streaming_due(H: int, P: int, inner_step: int) -> int:
+    """Fragment of Streaming SparseLoCo that synchronises after `inner_step` inner steps, or -1."""
+    v = C.c_int32()
+    _check(_L.sl_streaming_due(H, P, inner_step, C.byref(v)))
+    return v.value
 
 
 def static_scratch_bytes() -> int:

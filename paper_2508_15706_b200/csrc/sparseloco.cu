@@ -212,6 +212,18 @@ sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
     return SL_OK;
 }
 
+// Writes +0 at the staged positions of every worker's buffer in `bufs` (what Top-k leaves behind there).
+sl_status launch_zero_selected(sl_ctx* c, float* const* bufs, cudaStream_t st) {
+    const int R = c->cfg.R;
+    WorkerPtrs zp;
+    memset(&zp, 0, sizeof(zp));
+    for (int r = 0; r < R; ++r) zp.e[r] = bufs[r];
+    ef_flush_kernel<true><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
+                                                                          carve(c, R), zp);
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
 // The waiting values of a deferred subtraction go into the buffers of the step that left them.
 sl_status flush_pending(sl_ctx* c, cudaStream_t st) {
     if (!c->pending) return SL_OK;
@@ -434,7 +446,8 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     *out = nullptr;
     if (cfg->k < 1 || cfg->R < 1 || cfg->H < 1) return SL_ERR_INVALID_ARG;
     if (!(cfg->beta >= 0.0f && cfg->beta <= 1.0f) || !isfinite(cfg->outer_lr)) return SL_ERR_INVALID_ARG;
-    if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile || cfg->quant_bits != 2) return SL_ERR_UNSUPPORTED;
+    if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile) return SL_ERR_UNSUPPORTED;
+    if (cfg->quant_bits != 2 && cfg->quant_bits != 32) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
 
     {   // element ranges: no overflow, no two tensors sharing an element (kernels of different chunks would race)
@@ -676,6 +689,7 @@ sl_status sl_set_workspace(sl_ctx* c, void* dev_ptr, size_t bytes) {
 sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
                       void* stream) {
     if (!c || !theta_sync || !theta_local || !payload) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(theta_local) || misaligned(e) || misaligned(payload))
         return SL_ERR_ALIGNMENT;
@@ -691,6 +705,7 @@ sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
 
 sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
     if (!c || !payloads || !theta_sync) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
     PayloadPtrs pl;
     memset(&pl, 0, sizeof(pl));
@@ -705,8 +720,51 @@ sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* t
     return launch_apply(c, pl, present, theta_sync, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+// The outer step without the quantiser (quant_bits = 32, the full-precision column of the paper's
+// quantisation ablation): Top-k sends the selected values exactly, so nothing stays behind at the
+// selected positions (e = u - u = +0 there) and the staged values are averaged as they are.
+sl_status outer_step_unquantised(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+                                 cudaStream_t st) {
+    const int R = c->cfg.R;
+    const bool ef = c->cfg.ef_enabled != 0;
+    if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, R)) return SL_ERR_NOMEM;
+    WorkerPtrs ptrs;
+    memset(&ptrs, 0, sizeof(ptrs));
+    for (int r = 0; r < R; ++r) {
+        if (!theta_local[r] || (ef && !e[r])) return SL_ERR_INVALID_ARG;
+        if (misaligned(theta_local[r]) || (ef && misaligned(e[r]))) return SL_ERR_ALIGNMENT;
+        for (int q = 0; q < r; ++q)
+            if (ef && e[q] == e[r]) return SL_ERR_INVALID_ARG;
+        ptrs.theta_local[r] = theta_local[r];
+        ptrs.e[r] = ef ? e[r] : nullptr;
+    }
+    sl_status s = flush_pending(c, st);
+    if (s != SL_OK) return s;
+    c->last_workers = R;
+    if ((s = launch_select(c, R, theta_sync, ptrs, st, ef, false, false)) != SL_OK) return s;
+    if (ef && (s = launch_zero_selected(c, e, st)) != SL_OK) return s;
+    PayloadPtrs none;
+    memset(&none, 0, sizeof(none));
+    const int was = c->cfg.divide_by_present;
+    c->cfg.divide_by_present = 0;
+    s = launch_apply(c, none, R, theta_sync, st, 3);
+    c->cfg.divide_by_present = was;
+    return s;
+}
+
+}  // namespace
+
 sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
                         uint8_t* const* payloads, void* stream) {
+    if (c && c->cfg.quant_bits == 32) {
+        if (!theta_sync || !theta_local || (c->cfg.ef_enabled && !e)) return SL_ERR_INVALID_ARG;
+        if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
+        DeviceGuard g(c->device);
+        if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+        return outer_step_unquantised(c, theta_sync, theta_local, e, static_cast<cudaStream_t>(stream));
+    }
     if (!c || !theta_sync || !theta_local || !payloads) return SL_ERR_INVALID_ARG;
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
@@ -857,18 +915,6 @@ sl_status sl_diloco_step(sl_ctx* c, float* theta_sync, const float* const* theta
 }
 
 namespace {
-
-// Writes +0 at the staged positions of every worker's buffer in `bufs` (what Top-k leaves behind there).
-sl_status launch_zero_selected(sl_ctx* c, float* const* bufs, cudaStream_t st) {
-    const int R = c->cfg.R;
-    WorkerPtrs zp;
-    memset(&zp, 0, sizeof(zp));
-    for (int r = 0; r < R; ++r) zp.e[r] = bufs[r];
-    ef_flush_kernel<true><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
-                                                                          carve(c, R), zp);
-    SL_CUDA(cudaGetLastError());
-    return SL_OK;
-}
 
 // Common argument checks of the three baseline steps; fills the pointer tables.
 sl_status variant_args(sl_ctx* c, const float* theta_sync, const float* const* theta_local, float* const* e,
@@ -1084,6 +1130,18 @@ sl_status sl_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* st
     sl_status s = launch_flush(c, ptrs, static_cast<cudaStream_t>(stream));
     if (s != SL_OK) return s;
     if (!keep_pending) c->pending = false;
+    return SL_OK;
+}
+
+sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fragment) {
+    if (!fragment || H < 1 || P < 1 || P > H || inner_step < 1) return SL_ERR_INVALID_ARG;
+    *fragment = -1;
+    const int64_t t = inner_step % H;
+    for (int32_t p = 0; p < P; ++p)
+        if (t == (((int64_t)(p + 1) * H) / P) % H) {
+            *fragment = p;
+            break;
+        }
     return SL_OK;
 }
 

@@ -128,3 +128,29 @@ def test_alg3_with_ef_and_no_momentum_equals_the_outer_step_without_quantiser_on
         differ = (e_a[r].view(torch.int32) != e_b[r].view(torch.int32))
         assert int(differ.sum()) <= slots                  # only selected entries can differ
         assert bool((e_a[r][differ] == 0).all())           # and without a quantiser nothing stays behind there
+
+
+@pytest.mark.parametrize("ef_enabled", [True, False])
+def test_outer_step_without_quantiser(ef_enabled):
+    """quant_bits = 32 (the full-precision column of the paper's quantisation ablation): sl_outer_step
+    against the oracle's compression with the same setting followed by its sparse aggregation."""
+    from paper_2508_15706_b200.binding import SparseLoCo
+    wl, _, cfg, tab, theta, dev = _setup(R=3, k=64, seed=65)
+    shapes, offs = [(t.rows, t.cols) for t in TENSORS], I.offsets(TENSORS)
+    sl = SparseLoCo(shapes, offs, k=64, R=3, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=32, ef_enabled=ef_enabled)
+    cfg = O.Config(k=64, R=3, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=32, ef_enabled=int(ef_enabled))
+    e = [I.initial_error(wl, r, dev, scale=0.5) for r in range(3)]
+    th_o, e_o = theta.cpu().numpy().copy(), [x.cpu().numpy().copy() for x in e]
+    for step in range(2):
+        local = [I.theta_local(wl, theta, r, step) for r in range(3)]
+        outs = [O.compress(cfg, tab, th_o, local[r].cpu().numpy(), e_o[r]) for r in range(3)]
+        O.aggregate_apply_sparse(cfg, tab, [o.sel_idx for o in outs], [o.sel_hat for o in outs], th_o)
+        sl.outer_step(theta, local, e if ef_enabled else None, [None] * 3)   # no payload format: none is written
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
+        for r in range(3):
+            _bits_equal(e[r], e_o[r], ("e", step, r))
+        _close(theta, th_o, ("theta", step))
+        theta.copy_(torch.from_numpy(th_o))
+    with pytest.raises(Exception):
+        sl.compress(theta, local[0], e[0], torch.zeros(64, dtype=torch.uint8, device=dev))
