@@ -11,9 +11,89 @@ namespace {
 // consecutive chunks of the tensor, the groups.
 // ------------------------------------------------------------------------------------------------
 
-// Visits the keff staged values of one unit in slot order: four 128-bit loads in flight at a time.
+// (worker, chunk) of work item i; chunks x workers < 2^31 (checked on the host)
+__device__ __forceinline__ void split_unit(long long i, long long n_chunks, int& r, int& g) {
+    const unsigned ui = (unsigned)i, nc = (unsigned)n_chunks;
+    r = (int)(ui / nc);
+    g = (int)(ui - (unsigned)r * nc);
+}
+
+// The per-unit passes below give one lane the ordered fp64 chain of one (worker, chunk) unit, but a
+// lane reading its own 256-byte run makes every load instruction of the warp touch 32 different
+// lines.  Instead a warp takes 32 consecutive units -- contiguous in the staging array -- loads them
+// together with fully coalesced 128-bit loads, 64 slots at a time, into a shared tile (row stride 65:
+// conflict-free both ways) and every lane then walks its own row in slot order.
+constexpr int kStatWarps = 4;      // per CTA
+constexpr int kStatSlots = 64;     // slots per round
+struct StatTile {
+    float v[32][kStatSlots + 1];
+};
+
+// f(x) is called for the staged values of unit i0 + lane in slot order (keff of them; none when the
+// unit does not exist).  Warp-collective.
 template <typename F>
-__device__ __forceinline__ void for_each_staged(const float* __restrict__ v, int keff, F f) {
+__device__ __forceinline__ void for_each_staged(const float* __restrict__ val, long long i0, long long n_units, int kp,
+                                                int keff, StatTile& tile, F f) {
+    const int lane = threadIdx.x & 31;
+    for (int sb = 0; sb < kp; sb += kStatSlots) {
+#pragma unroll 4
+        for (int j = 0; j < 16; ++j) {
+            const int row = 2 * j + (lane >> 4), c = 4 * (lane & 15);
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i0 + row < n_units && sb + c < kp)
+                x = __ldcs(reinterpret_cast<const float4*>(val + (i0 + row) * kp + sb + c));
+            tile.v[row][c + 0] = x.x;
+            tile.v[row][c + 1] = x.y;
+            tile.v[row][c + 2] = x.z;
+            tile.v[row][c + 3] = x.w;
+        }
+        __syncwarp();
+        const int n = min(kStatSlots, keff - sb);
+        for (int s0 = 0; s0 < n; ++s0) f(tile.v[lane][s0]);
+        __syncwarp();
+    }
+}
+
+// mode 0: sum of values; mode 1: sum of squared fp32-centred values.  One lane per (worker, chunk).
+template <int MODE>
+__global__ void __launch_bounds__(32 * kStatWarps)
+chunk_sum_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
+                 int k, int kp, Workspace ws) {
+    __shared__ StatTile tiles[kStatWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long total = n_chunks * n_workers;
+    const long long i0 = ((long long)blockIdx.x * kStatWarps + warp) * 32, i = i0 + lane;
+    if (i0 >= total) return;
+    int r = 0, g = 0, keff = 0;
+    float mu = 0.0f;
+    if (i < total) {
+        split_unit(i, n_chunks, r, g);
+        keff = min(k, chunks[g].len);
+        if (MODE == 1) mu = ws.tstat[(long long)r * n_tensors + chunks[g].tensor].mu;
+    }
+    double acc = 0.0;
+    for_each_staged(ws.val, i0, total, kp, keff, tiles[warp], [&](float x) {
+        if (MODE == 0) {
+            acc += (double)x;
+        } else {
+            const double d = (double)__fsub_rn(x, mu);
+            acc += d * d;  // d*d is exact in fp64, so fusing or not gives the same sum
+        }
+    });
+    if (i < total) ws.psum[i] = acc;
+}
+
+// Per-bin sums and counts of one chunk.  codes: (cen >= -t) + (cen >= 0) + (cen >= t).
+__device__ __forceinline__ int quant_code(float v, float mu, float t3) {
+    const float cen = __fsub_rn(v, mu);
+    return (cen >= -t3 ? 1 : 0) + (cen >= 0.0f ? 1 : 0) + (cen >= t3 ? 1 : 0);
+}
+
+// Visits the keff staged values of one unit in slot order, read by the thread itself: four 128-bit
+// loads in flight at a time.  (The per-bin pass does more arithmetic per value and runs best at full
+// occupancy, which the shared tiles of the cooperative form would halve.)
+template <typename F>
+__device__ __forceinline__ void for_each_staged_own(const float* __restrict__ v, int keff, F f) {
     int s0 = 0;
     for (; s0 + 16 <= keff; s0 += 16) {
         float4 x[4];
@@ -30,44 +110,6 @@ __device__ __forceinline__ void for_each_staged(const float* __restrict__ v, int
     for (; s0 < keff; ++s0) f(v[s0]);
 }
 
-// (worker, chunk) of work item i; chunks x workers < 2^31 (checked on the host)
-__device__ __forceinline__ void split_unit(long long i, long long n_chunks, int& r, int& g) {
-    const unsigned ui = (unsigned)i, nc = (unsigned)n_chunks;
-    r = (int)(ui / nc);
-    g = (int)(ui - (unsigned)r * nc);
-}
-
-// mode 0: sum of values; mode 1: sum of squared fp32-centred values.  One thread per (worker, chunk).
-template <int MODE>
-__global__ void __launch_bounds__(128)
-chunk_sum_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
-                 int k, int kp, Workspace ws) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n_chunks * n_workers) return;
-    int r, g;
-    split_unit(i, n_chunks, r, g);
-    const int keff = min(k, chunks[g].len);
-    const float* __restrict__ v = ws.val + i * kp;
-    float mu = 0.0f;
-    if (MODE == 1) mu = ws.tstat[(long long)r * n_tensors + chunks[g].tensor].mu;
-    double acc = 0.0;
-    for_each_staged(v, keff, [&](float x) {
-        if (MODE == 0) {
-            acc += (double)x;
-        } else {
-            const double d = (double)__fsub_rn(x, mu);
-            acc += d * d;  // d*d is exact in fp64, so fusing or not gives the same sum
-        }
-    });
-    ws.psum[i] = acc;
-}
-
-// Per-bin sums and counts of one chunk.  codes: (cen >= -t) + (cen >= 0) + (cen >= t).
-__device__ __forceinline__ int quant_code(float v, float mu, float t3) {
-    const float cen = __fsub_rn(v, mu);
-    return (cen >= -t3 ? 1 : 0) + (cen >= 0.0f ? 1 : 0) + (cen >= t3 ? 1 : 0);
-}
-
 __global__ void __launch_bounds__(128)
 chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
                   int k, int kp, Workspace ws) {
@@ -80,7 +122,7 @@ chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
     const TStat st = ws.tstat[(long long)r * n_tensors + chunks[g].tensor];
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
     unsigned n0 = 0, n1 = 0, n2 = 0, n3 = 0;
-    for_each_staged(v, keff, [&](float x) {
+    for_each_staged_own(v, keff, [&](float x) {
         const int c = quant_code(x, st.mu, st.t3);
         const double d = (double)x;
         // add only to the value's own bin (adding +0 elsewhere could flip a -0 sum); nearly all
