@@ -82,6 +82,13 @@ def lib():
         L.orc_topk_chunk.restype = C.c_int32
         L.orc_topk_chunk.argtypes = [P, C.c_int32, C.c_int32, P]
         L.orc_quantize_tensor.argtypes = [P, P, C.c_int64, P, P, P, P]
+        L.orc_quantize_tensor_q.argtypes = [P, P, C.c_int64, C.c_int32, P, P, P, P]
+        L.orc_record_stride_q.restype = C.c_int64
+        L.orc_record_stride_q.argtypes = [C.c_int32, C.c_int32]
+        L.orc_header_bytes.restype = C.c_int64
+        L.orc_header_bytes.argtypes = [C.c_int32]
+        L.orc_pack_record_q.argtypes = [P, P, C.c_int32, C.c_int32, C.c_int32, P]
+        L.orc_unpack_record_q.argtypes = [P, C.c_int32, C.c_int32, C.c_int32, P, P]
         L.orc_pack_record.argtypes = [P, P, C.c_int32, C.c_int32, P]
         L.orc_unpack_record.argtypes = [P, C.c_int32, C.c_int32, P, P]
         L.orc_compress.argtypes = [P, P, C.c_int32, P, P, P, P, P, P, P, P]
@@ -204,6 +211,41 @@ def quantize_tensor(v: np.ndarray, cnt: np.ndarray):
     return mu[0], sg[0], lut, code[:v.size]
 
 
+def quantize_tensor_q(v: np.ndarray, cnt: np.ndarray, bits: int):
+    """(mu, sigma, table[2^bits], codes) of the quantiser at `bits` bits per value."""
+    _chk(v, np.float32)
+    cnt = np.ascontiguousarray(cnt, dtype=np.int32)
+    mu = np.zeros(1, np.float32)
+    sg = np.zeros(1, np.float32)
+    lut = np.zeros(16, np.float32)
+    code = np.zeros(max(v.size, 1), np.uint8)
+    lib().orc_quantize_tensor_q(_ptr(v), _ptr(cnt), cnt.size, bits, _ptr(mu), _ptr(sg), _ptr(lut), _ptr(code))
+    return mu[0], sg[0], lut[:1 << bits], code[:v.size]
+
+
+def record_stride_q(k: int, bits: int) -> int:
+    return lib().orc_record_stride_q(k, bits)
+
+
+def header_bytes(bits: int) -> int:
+    return lib().orc_header_bytes(bits)
+
+
+def pack_record_q(idx: np.ndarray, code: np.ndarray, k: int, bits: int) -> np.ndarray:
+    idx = np.ascontiguousarray(idx, np.int32)
+    code = np.ascontiguousarray(code, np.uint8)
+    rec = np.zeros(record_stride_q(k, bits), np.uint8)
+    lib().orc_pack_record_q(_ptr(idx), _ptr(code), idx.size, k, bits, _ptr(rec))
+    return rec
+
+
+def unpack_record_q(rec: np.ndarray, m: int, k: int, bits: int):
+    idx = np.zeros(max(m, 1), np.int32)
+    code = np.zeros(max(m, 1), np.uint8)
+    lib().orc_unpack_record_q(_ptr(_chk(rec, np.uint8)), m, k, bits, _ptr(idx), _ptr(code))
+    return idx[:m], code[:m]
+
+
 def pack_record(idx: np.ndarray, code: np.ndarray, k: int) -> np.ndarray:
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     code = np.ascontiguousarray(code, dtype=np.uint8)
@@ -226,18 +268,18 @@ class Compressed:
     sel_idx: np.ndarray
     sel_val: np.ndarray
     sel_hat: np.ndarray
-    stats: np.ndarray  # per tensor: mu, sigma, lut[0..3]
+    stats: np.ndarray  # per tensor: mu, sigma, the table (2^bits entries, then zeros up to 16)
 
 
 def compress(cfg: Config, tab: Table, theta: np.ndarray, theta_r: np.ndarray, e: np.ndarray) -> Compressed:
     """One worker's compression + error feedback; `e` is updated in place."""
     c = cfg.c()
     slots = total_slots(cfg, tab)
-    payload = np.zeros(payload_bytes(cfg, tab), np.uint8) if cfg.quant_bits == 2 else None
+    payload = np.zeros(payload_bytes(cfg, tab), np.uint8) if cfg.quant_bits in (1, 2, 3, 4) else None
     sel_idx = np.empty(max(slots, 1), np.int32)
     sel_val = np.empty(max(slots, 1), np.float32)
     sel_hat = np.empty(max(slots, 1), np.float32)
-    stats = np.zeros((tab.n, 6), np.float32)
+    stats = np.zeros((tab.n, 18), np.float32)
     lib().orc_compress(C.byref(c), tab.ref(), tab.n, _ptr(_chk(theta, np.float32)),
                        _ptr(_chk(theta_r, np.float32)), _ptr(_chk(e, np.float32)), _ptr(payload),
                        _ptr(sel_idx), _ptr(sel_val), _ptr(sel_hat), _ptr(stats))

@@ -66,7 +66,7 @@ typedef struct {
     int32_t k;
     int32_t R, H;
     float beta, outer_lr;
-    int32_t quant_bits;        /* 2, or 32 = values sent unquantised */
+    int32_t quant_bits;        /* 2 (the paper's setting), 1 / 3 / 4 (its ablation), or 32 = values sent unquantised */
     int32_t ef_enabled;        /* 0 during the error-feedback freeze */
     int32_t divide_by_present; /* 0: divide by R; 1: by the number of payloads present */
 } orc_config;
@@ -136,9 +136,26 @@ int64_t orc_record_stride(int32_t k) {
     return (idx_bytes + code_bytes + 15) / 16 * 16;
 }
 
-/* Bytes of one worker's payload: one 16-byte table per tensor, then every chunk record. */
+/* The same for a quantiser of `bits` bits per value (1..4; the paper's ablation over quantisation
+ * widths): k 12-bit indices, then k codes of `bits` bits, rounded up to 16. */
+int64_t orc_record_stride_q(int32_t k, int32_t bits) {
+    int64_t idx_bytes = (12 * (int64_t)k + 7) / 8;
+    int64_t code_bytes = ((int64_t)bits * (int64_t)k + 7) / 8;
+    return (idx_bytes + code_bytes + 15) / 16 * 16;
+}
+
+/* Bytes of a tensor's table in the payload: 2^bits fp32 entries, at least 16 bytes. */
+int64_t orc_header_bytes(int32_t bits) {
+    int64_t b = 4 * ((int64_t)1 << bits);
+    return b < 16 ? 16 : b;
+}
+
+static int32_t payload_bits(const orc_config* c) { return c->quant_bits == 32 ? 2 : c->quant_bits; }
+
+/* Bytes of one worker's payload: one table per tensor (16 bytes at 2 bits), then every chunk record. */
 int64_t orc_payload_bytes(const orc_config* c, const orc_tensor* ts, int32_t nt) {
-    return 16 * (int64_t)nt + orc_record_stride(c->k) * orc_total_chunks(c, ts, nt);
+    const int32_t b = payload_bits(c);
+    return orc_header_bytes(b) * (int64_t)nt + orc_record_stride_q(c->k, b) * orc_total_chunks(c, ts, nt);
 }
 
 /* ---------------------------------------------------------------- pseudo-gradient + error feedback */
@@ -278,6 +295,93 @@ void orc_quantize_tensor(const float* v, const int32_t* cnt, int64_t n_chunks, f
     *sigma_out = sigma;
 }
 
+/* The quantiser of Sec. 4 at any width (the paper's ablation uses 1, 2, 3 and 4 bits): centred by
+ * the mean, [-6 sigma, 6 sigma] in 2^bits uniform bins, every bin stores the centroid of the raw
+ * values that fell into it.  Written like the 2-bit routine above, with the same fixed summation
+ * order: the inner edges are c_j sigma with c_j = -6 + 12 j / 2^bits (j = 1 .. 2^bits - 1; multiples
+ * of 0.75, exact in fp32), each the fp32 product of c_j and sigma, lower edge inclusive, so that
+ * code = number of edges the centred value reaches; values beyond +-6 sigma fall in the outer bins.
+ * At bits = 2 the edges are -3 sigma, 0, 3 sigma: the routine above. */
+void orc_quantize_tensor_q(const float* v, const int32_t* cnt, int64_t n_chunks, int32_t bits,
+                           float* mu_out, float* sigma_out, float* lut /* 2^bits */, uint8_t* code) {
+    const int nbins = 1 << bits;
+    int64_t n = 0;
+    for (int64_t c = 0; c < n_chunks; ++c) n += cnt[c];
+    for (int b = 0; b < nbins; ++b) lut[b] = 0.0f;
+    *mu_out = 0.0f;
+    *sigma_out = 0.0f;
+    if (n == 0) return;
+
+    double S = 0.0;
+    {
+        const float* q = v;
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double sg = 0.0;
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double sc = 0.0;
+                for (int32_t s = 0; s < cnt[c]; ++s) sc += (double)q[s];
+                sg += sc;
+                q += cnt[c];
+            }
+            S += sg;
+        }
+    }
+    const float mu = (float)(S / (double)n);
+
+    double V = 0.0;
+    {
+        const float* q = v;
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double vg = 0.0;
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double vc = 0.0;
+                for (int32_t s = 0; s < cnt[c]; ++s) {
+                    const float cen = q[s] - mu;
+                    vc += (double)cen * (double)cen;
+                }
+                vg += vc;
+                q += cnt[c];
+            }
+            V += vg;
+        }
+    }
+    const float sigma = (float)sqrt(V / (double)n);
+
+    float edge[15];
+    for (int j = 1; j < nbins; ++j) edge[j - 1] = (-6.0f + 12.0f * (float)j / (float)nbins) * sigma;
+
+    double Sb[16];
+    int64_t nb[16];
+    for (int b = 0; b < 16; ++b) { Sb[b] = 0.0; nb[b] = 0; }
+    {
+        const float* q = v;
+        uint8_t* cq = code;
+        for (int64_t c0 = 0; c0 < n_chunks; c0 += ORC_SUM_GROUP) {
+            double sgb[16];
+            for (int b = 0; b < 16; ++b) sgb[b] = 0.0;
+            for (int64_t c = c0; c < n_chunks && c < c0 + ORC_SUM_GROUP; ++c) {
+                double sb[16];
+                for (int b = 0; b < 16; ++b) sb[b] = 0.0;
+                for (int32_t s = 0; s < cnt[c]; ++s) {
+                    const float cen = q[s] - mu;
+                    int b = 0;
+                    for (int j = 0; j < nbins - 1; ++j) b += cen >= edge[j];
+                    cq[s] = (uint8_t)b;
+                    sb[b] += (double)q[s];
+                    nb[b] += 1;
+                }
+                for (int b = 0; b < nbins; ++b) sgb[b] += sb[b];
+                q += cnt[c];
+                cq += cnt[c];
+            }
+            for (int b = 0; b < nbins; ++b) Sb[b] += sgb[b];
+        }
+    }
+    for (int b = 0; b < nbins; ++b) lut[b] = nb[b] ? (float)(Sb[b] / (double)nb[b]) : 0.0f;
+    *mu_out = mu;
+    *sigma_out = sigma;
+}
+
 /* ---------------------------------------------------------------- packing (little-endian bit order) */
 
 static void put_bits(uint8_t* base, int64_t bit, int nbits, uint32_t val) {
@@ -313,6 +417,24 @@ void orc_unpack_record(const uint8_t* rec, int32_t m, int32_t k, int32_t* idx, u
     }
 }
 
+/* The same with codes of `bits` bits (1..4). */
+void orc_pack_record_q(const int32_t* idx, const uint8_t* code, int32_t m, int32_t k, int32_t bits, uint8_t* rec) {
+    memset(rec, 0, (size_t)orc_record_stride_q(k, bits));
+    int64_t code_base = ((12 * (int64_t)k + 7) / 8) * 8;
+    for (int32_t s = 0; s < m; ++s) {
+        put_bits(rec, 12 * (int64_t)s, 12, (uint32_t)idx[s]);
+        put_bits(rec, code_base + (int64_t)bits * s, bits, code[s]);
+    }
+}
+
+void orc_unpack_record_q(const uint8_t* rec, int32_t m, int32_t k, int32_t bits, int32_t* idx, uint8_t* code) {
+    int64_t code_base = ((12 * (int64_t)k + 7) / 8) * 8;
+    for (int32_t s = 0; s < m; ++s) {
+        idx[s] = (int32_t)get_bits(rec, 12 * (int64_t)s, 12);
+        code[s] = (uint8_t)get_bits(rec, code_base + (int64_t)bits * s, bits);
+    }
+}
+
 /* ---------------------------------------------------------------- one worker's compression */
 
 /*
@@ -322,16 +444,18 @@ void orc_unpack_record(const uint8_t* rec, int32_t m, int32_t k, int32_t* idx, u
  *   payload           : orc_payload_bytes() bytes, or NULL (also unused when quant_bits == 32).
  *   sel_idx, sel_val, sel_hat : optional (may be NULL) arrays of orc_total_slots() entries, in
  *                       (tensor, chunk, slot) order: in-chunk index, raw value u, decoded value.
- *   stats             : optional, 6 floats per tensor: mu, sigma, lut[0..3].
+ *   stats             : optional, 18 floats per tensor: mu, sigma, the table (2^bits entries, then zeros).
  */
 void orc_compress(const orc_config* cfg, const orc_tensor* ts, int32_t nt, const float* theta,
                   const float* theta_r, float* e, uint8_t* payload, int32_t* sel_idx,
                   float* sel_val, float* sel_hat, float* stats) {
     const int32_t k = cfg->k, C = cfg->chunk_elems;
-    const int64_t stride = orc_record_stride(k);
-    int64_t rec_off = 16 * (int64_t)nt; /* records follow the per-tensor tables */
+    const int32_t qb = cfg->quant_bits;            /* 1..4, or 32 = values travel unquantised */
+    const int quantised = qb >= 1 && qb <= 4;
+    const int64_t stride = orc_record_stride_q(k, payload_bits(cfg)), hdr = orc_header_bytes(payload_bits(cfg));
+    int64_t rec_off = hdr * (int64_t)nt; /* records follow the per-tensor tables */
     int64_t slot_off = 0;
-    if (payload && cfg->quant_bits == 2) memset(payload, 0, (size_t)orc_payload_bytes(cfg, ts, nt));
+    if (payload && quantised) memset(payload, 0, (size_t)orc_payload_bytes(cfg, ts, nt));
 
     for (int32_t j = 0; j < nt; ++j) {
         const orc_tensor* t = &ts[j];
@@ -370,25 +494,30 @@ void orc_compress(const orc_config* cfg, const orc_tensor* ts, int32_t nt, const
                 for (int32_t s = 0; s < cnt[ch]; ++s) v[w++] = val[ch * k + s];
         }
 
-        float mu = 0.0f, sigma = 0.0f, lut[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (cfg->quant_bits == 2) {
+        float mu = 0.0f, sigma = 0.0f, lut[16];
+        for (int b = 0; b < 16; ++b) lut[b] = 0.0f;
+        if (qb == 2) {
             orc_quantize_tensor(v, cnt, nc, &mu, &sigma, lut, code);
+            for (int64_t w = 0; w < m_total; ++w) vhat[w] = lut[code[w]];
+        } else if (quantised) {
+            orc_quantize_tensor_q(v, cnt, nc, qb, &mu, &sigma, lut, code);
             for (int64_t w = 0; w < m_total; ++w) vhat[w] = lut[code[w]];
         } else { /* 32: values travel unquantised */
             for (int64_t w = 0; w < m_total; ++w) vhat[w] = v[w];
         }
-        if (stats) {
-            stats[6 * j + 0] = mu;
-            stats[6 * j + 1] = sigma;
-            for (int b = 0; b < 4; ++b) stats[6 * j + 2 + b] = lut[b];
+        if (stats) { /* 18 floats per tensor: mu, sigma, table (2^bits entries, the rest 0) */
+            stats[18 * j + 0] = mu;
+            stats[18 * j + 1] = sigma;
+            for (int b = 0; b < 16; ++b) stats[18 * j + 2 + b] = lut[b];
         }
 
         /* payload: table, then records */
-        if (payload && cfg->quant_bits == 2) {
-            memcpy(payload + 16 * (int64_t)j, lut, 16);
+        if (payload && quantised) {
+            memcpy(payload + hdr * (int64_t)j, lut, (size_t)(4 << qb));
             int64_t w = 0;
             for (int64_t ch = 0; ch < nc; ++ch) {
-                orc_pack_record(idx + ch * k, code + w, cnt[ch], k, payload + rec_off + ch * stride);
+                if (qb == 2) orc_pack_record(idx + ch * k, code + w, cnt[ch], k, payload + rec_off + ch * stride);
+                else orc_pack_record_q(idx + ch * k, code + w, cnt[ch], k, qb, payload + rec_off + ch * stride);
                 w += cnt[ch];
             }
         }
@@ -474,18 +603,19 @@ void orc_aggregate_apply_sparse(const orc_config* cfg, const orc_tensor* ts, int
  * Sec. 4: values are dequantised through the table before aggregation. */
 void orc_decode_payload(const orc_config* cfg, const orc_tensor* ts, int32_t nt,
                         const uint8_t* payload, int32_t* sel_idx, float* sel_hat) {
-    const int32_t k = cfg->k;
-    const int64_t stride = orc_record_stride(k);
-    int64_t rec_off = 16 * (int64_t)nt, w = 0;
+    const int32_t k = cfg->k, qb = payload_bits(cfg);
+    const int64_t stride = orc_record_stride_q(k, qb), hdr = orc_header_bytes(qb);
+    int64_t rec_off = hdr * (int64_t)nt, w = 0;
     uint8_t* code = (uint8_t*)malloc((size_t)k);
     for (int32_t j = 0; j < nt; ++j) {
-        float lut[4];
-        memcpy(lut, payload + 16 * (int64_t)j, 16);
+        float lut[16];
+        memcpy(lut, payload + hdr * (int64_t)j, (size_t)(4 << qb));
         int64_t nc = orc_num_chunks(cfg, &ts[j]);
         for (int64_t ch = 0; ch < nc; ++ch) {
             int64_t L = orc_chunk_len(cfg, &ts[j], ch);
             int32_t m = (int32_t)(L < k ? L : k);
-            orc_unpack_record(payload + rec_off + ch * stride, m, k, sel_idx + w, code);
+            if (qb == 2) orc_unpack_record(payload + rec_off + ch * stride, m, k, sel_idx + w, code);
+            else orc_unpack_record_q(payload + rec_off + ch * stride, m, k, qb, sel_idx + w, code);
             for (int32_t s = 0; s < m; ++s) sel_hat[w + s] = lut[code[s]];
             w += m;
         }
