@@ -33,6 +33,11 @@
  *         bits  [12 s, 12 s + 12)                   in-chunk index of slot s
  *         bytes from ceil(12 k / 8): bits [2 s, 2 s + 2)   code of slot s
  *     slots >= min(k, chunk length) and all padding are zero.
+ * With quant_bits = b in {1, 3, 4} the same layout holds with b in place of 2: tables of 2^b fp32 entries
+ * (max(16, 4 * 2^b) bytes per tensor; entry j = centroid of the bin between the edges (-6 + 12 j / 2^b) sigma
+ * and (-6 + 12 (j + 1) / 2^b) sigma of the centred values, the outer bins open-ended), records of
+ * roundup16(ceil(12 k / 8) + ceil(b k / 8)) bytes with the code of slot s at bits [b s, b s + b) of the code
+ * block.  sl_payload_bytes() gives the size.
  */
 #ifndef SPARSELOCO_H
 #define SPARSELOCO_H
@@ -48,7 +53,8 @@ typedef enum {
     SL_OK = 0,
     SL_ERR_INVALID_ARG = 1, /* NULL pointer, size or hyper-parameter out of range */
     SL_ERR_ALIGNMENT = 2,   /* a device pointer or tensor offset is not 16-byte aligned */
-    SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, bits other than 2 / 32, ...) */
+    SL_ERR_UNSUPPORTED = 3, /* valid in the method, not built here (chunk != 4096, quant_bits not in 1..4 / 32,
+                               an entry point that serves the 2-bit payload only, ...) */
     SL_ERR_BAD_PAYLOAD = 4, /* reported through the device status word of sl_validate_payload */
     SL_ERR_CUDA = 5,        /* a CUDA runtime call failed; see sl_last_cuda_error() */
     SL_ERR_NOMEM = 6,       /* workspace missing or too small; host allocation failed */
@@ -72,8 +78,11 @@ typedef struct {
     int32_t H;                 /* inner steps; carried for the caller, >= 1, unused by the math */
     float beta;                /* error-feedback decay, 0 <= beta <= 1 */
     float outer_lr;            /* alpha, finite */
-    int32_t quant_bits;        /* 2; or 32 = no quantiser: the selected values are averaged as they are
-                                  (sl_outer_step only: there is no payload format, payloads may be NULL) */
+    int32_t quant_bits;        /* 2 (the paper's setting; the fast path); 1, 3 or 4 (its ablation: 2^bits
+                                  uniform bins over [-6 sigma, 6 sigma], plain kernels, no deferral, no wire
+                                  codec, no validation); or 32 = no quantiser: the selected values are averaged
+                                  as they are (sl_outer_step only: there is no payload format, payloads may be
+                                  NULL) */
     int32_t ef_enabled;        /* 0 during the error-feedback freeze (App. "Freezing Error
                                   Feedback"): u = Delta and e is neither read nor written */
     int32_t divide_by_present; /* 0: average divides by R (Alg. 1); 1: by the payloads present */

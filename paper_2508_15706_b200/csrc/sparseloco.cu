@@ -39,6 +39,7 @@
 #include "quantiser.cuh"
 #include "pack.cuh"
 #include "apply.cuh"
+#include "quant_wide.cuh"
 #include "misc.cuh"
 #include "index_codec.cuh"
 #include "dense.cuh"
@@ -55,6 +56,9 @@ struct sl_ctx {
     long long n_slots;
     long long flat_elems;
     int kp;
+    int qbits;          // bits per code in the payload (2 also when quant_bits = 32: no payload is written then)
+    int rec_stride;     // bytes of one chunk record
+    long long rec_base; // byte offset of the first record in a payload (after the tensor tables)
     std::vector<sl_tensor_desc> tensors;
     ChunkDesc* d_chunks;
     TensorInfo* d_tinfo;
@@ -123,11 +127,38 @@ sl_status cuda_fail(cudaError_t e, const char* what) {
 
 inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-size_t workspace_bytes_for(const sl_ctx* c, int workers) {
+// general-width quantiser (quant_bits 1, 3, 4): its per-unit bin partials and per-tensor tables follow
+// the arrays of the 2-bit path in the workspace
+inline bool wide_quant(const sl_ctx* c) { return c->cfg.quant_bits != 2 && c->cfg.quant_bits != 32; }
+size_t wide_bytes_for(const sl_ctx* c, int workers) {
+    if (!wide_quant(c)) return 0;
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->cfg.quant_bits;
+    return up256(WG * nb * sizeof(double)) + up256(WG * nb * sizeof(unsigned)) +
+           up256((size_t)workers * c->n_tensors * sizeof(TStatQ));
+}
+
+size_t narrow_bytes_for(const sl_ctx* c, int workers) {
     const size_t WG = (size_t)workers * (size_t)c->n_chunks;
     return up256(WG * c->kp * sizeof(float)) + up256(WG * c->kp * sizeof(uint16_t)) +
            up256(WG * sizeof(double)) + up256(WG * 4 * sizeof(double)) + up256(WG * 4 * sizeof(unsigned)) +
            up256((size_t)workers * c->n_tensors * sizeof(TStat));
+}
+
+size_t workspace_bytes_for(const sl_ctx* c, int workers) { return narrow_bytes_for(c, workers) + wide_bytes_for(c, workers); }
+
+struct WideSpace {
+    double* pbin;
+    unsigned* pcnt;
+    TStatQ* tq;
+};
+WideSpace carve_wide(const sl_ctx* c, int workers) {
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->cfg.quant_bits;
+    char* p = static_cast<char*>(c->ws_ptr) + narrow_bytes_for(c, workers);
+    WideSpace w;
+    w.pbin = reinterpret_cast<double*>(p);      p += up256(WG * nb * sizeof(double));
+    w.pcnt = reinterpret_cast<unsigned*>(p);    p += up256(WG * nb * sizeof(unsigned));
+    w.tq = reinterpret_cast<TStatQ*>(p);
+    return w;
 }
 
 Workspace carve(const sl_ctx* c, int workers) {
@@ -337,6 +368,28 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     prof_mark(c, 3, st);
     tensor_reduce_kernel<1><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 4, st);
+    if (wide_quant(c)) {  // 1, 3 or 4 bits: the general-width kernels, records and error correction in place
+        const WideSpace wq = carve_wide(c, workers);
+        const unsigned pbq = blocks_for(WG, 4);
+#define SL_WIDE(BITSV)                                                                                              \
+    do {                                                                                                            \
+        chunk_bins_q_kernel<BITSV><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.pbin, wq.pcnt);    \
+        tensor_table_q_kernel<BITSV><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, wq.pbin, wq.pcnt, wq.tq, ptrs); \
+        if (ef)                                                                                                     \
+            pack_q_kernel<BITSV, true><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
+        else                                                                                                        \
+            pack_q_kernel<BITSV, false><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
+    } while (0)
+        if (c->cfg.quant_bits == 1) SL_WIDE(1);
+        else if (c->cfg.quant_bits == 3) SL_WIDE(3);
+        else SL_WIDE(4);
+#undef SL_WIDE
+        prof_mark(c, 5, st);
+        prof_mark(c, 6, st);
+        prof_mark(c, 7, st);
+        SL_CUDA(cudaGetLastError());
+        return SL_OK;
+    }
     chunk_bins_kernel<<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
     prof_mark(c, 5, st);
     tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
@@ -367,6 +420,19 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const int R = c->cfg.R;
     const double D = c->cfg.divide_by_present ? (double)present : (double)R;
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
+    if (wide_quant(c) && fuse == 0) {  // payloads of 1, 3 or 4 bits per value
+        const unsigned grid = (unsigned)c->n_chunks;
+        if (c->cfg.quant_bits == 1)
+            apply_q_kernel<1><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
+        else if (c->cfg.quant_bits == 3)
+            apply_q_kernel<3><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
+        else
+            apply_q_kernel<4><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
+        prof_mark(c, 8, st);
+        if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
+        SL_CUDA(cudaGetLastError());
+        return SL_OK;
+    }
     const size_t smem = apply_smem_bytes(c->cfg.k);
     const int ppl = (c->cfg.k + 63) / 64;
     FuseArgs fa;
@@ -447,7 +513,7 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (cfg->k < 1 || cfg->R < 1 || cfg->H < 1) return SL_ERR_INVALID_ARG;
     if (!(cfg->beta >= 0.0f && cfg->beta <= 1.0f) || !isfinite(cfg->outer_lr)) return SL_ERR_INVALID_ARG;
     if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile) return SL_ERR_UNSUPPORTED;
-    if (cfg->quant_bits != 2 && cfg->quant_bits != 32) return SL_ERR_UNSUPPORTED;
+    if (cfg->quant_bits != 32 && (cfg->quant_bits < 1 || cfg->quant_bits > 4)) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
 
     {   // element ranges: no overflow, no two tensors sharing an element (kernels of different chunks would race)
@@ -489,10 +555,13 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     c->host_path_ready = false;
     c->tensors.assign(tensors, tensors + n_tensors);
 
-    const int stride = record_stride(cfg->k);
+    c->qbits = cfg->quant_bits == 32 ? 2 : cfg->quant_bits;
+    const int stride = record_stride_q(cfg->k, c->qbits);  // = record_stride(k) at 2 bits
+    c->rec_stride = stride;
+    c->rec_base = (long long)header_bytes_q(c->qbits) * n_tensors;
     std::vector<ChunkDesc> chunks;
     std::vector<TensorInfo> tinfo((size_t)n_tensors);
-    long long rec_off = 16ll * n_tensors, flat = 0, slots = 0;
+    long long rec_off = c->rec_base, flat = 0, slots = 0;
     for (int j = 0; j < n_tensors; ++j) {
         const sl_tensor_desc& t = tensors[j];
         if (t.rows < 1 || t.cols < 1 || t.offset < 0) { delete c; return SL_ERR_INVALID_ARG; }
@@ -654,7 +723,7 @@ sl_status sl_set_hyper(sl_ctx* c, float beta, float outer_lr, int32_t ef_enabled
 
 sl_status sl_payload_bytes(const sl_ctx* c, size_t* bytes) {
     if (!c || !bytes) return SL_ERR_INVALID_ARG;
-    *bytes = 16 * (size_t)c->n_tensors + (size_t)record_stride(c->cfg.k) * (size_t)c->n_chunks;
+    *bytes = (size_t)c->rec_base + (size_t)c->rec_stride * (size_t)c->n_chunks;
     return SL_OK;
 }
 
@@ -689,7 +758,7 @@ sl_status sl_set_workspace(sl_ctx* c, void* dev_ptr, size_t bytes) {
 sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
                       void* stream) {
     if (!c || !theta_sync || !theta_local || !payload) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
+    if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(theta_local) || misaligned(e) || misaligned(payload))
         return SL_ERR_ALIGNMENT;
@@ -705,7 +774,7 @@ sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
 
 sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
     if (!c || !payloads || !theta_sync) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;
+    if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
     PayloadPtrs pl;
     memset(&pl, 0, sizeof(pl));
@@ -788,6 +857,11 @@ sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (wide_quant(c)) {  // general widths: the plain sequence, every worker's compression, then the aggregation
+        sl_status s = launch_compress(c, R, theta_sync, ptrs, st, false);
+        if (s != SL_OK) return s;
+        return launch_apply(c, pl, R, theta_sync, st);
+    }
     const bool defer = c->deferred && c->cfg.ef_enabled;
     if (c->pending && defer) {  // the waiting values can only be substituted into the buffers they came from
         for (int r = 0; r < R; ++r)
@@ -803,6 +877,7 @@ sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* t
                              size_t stage_elems, float* const* e, uint8_t* const* payloads, float* theta_sync_host,
                              void* stream) {
     if (!c || !theta_sync || !theta_local_host || !dev_stage || !payloads) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(dev_stage)) return SL_ERR_ALIGNMENT;
     const int R = c->cfg.R;
@@ -1033,6 +1108,7 @@ sl_status sl_lom_topk_step(sl_ctx* c, float* theta_sync, float* const* theta_loc
 
 sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {
     if (!c || !bytes) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;  // the stream's bit offsets are 32-bit
     *bytes = c->ixc_capacity;
     return SL_OK;
@@ -1041,6 +1117,7 @@ sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {
 sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, uint64_t* dev_coded_bytes,
                             void* stream) {
     if (!c || !payload || !coded || !dev_coded_bytes) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (misaligned(payload) || misaligned(coded) || (reinterpret_cast<uintptr_t>(dev_coded_bytes) & 7u))
         return SL_ERR_ALIGNMENT;
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
@@ -1066,6 +1143,7 @@ sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, u
 
 sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, size_t coded_bytes, uint8_t* payload, void* stream) {
     if (!c || !coded || !payload) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (misaligned(coded) || misaligned(payload)) return SL_ERR_ALIGNMENT;
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
     // what the buffer is said to hold bounds every read; it must at least reach the index stream
@@ -1104,6 +1182,7 @@ sl_status sl_device_status(sl_ctx* c, void* stream) {
 
 sl_status sl_set_ef_deferred(sl_ctx* c, int32_t on) {
     if (!c) return SL_ERR_INVALID_ARG;
+    if (on && c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // only the 2-bit path defers
     c->deferred = on != 0;
     return SL_OK;
 }
@@ -1147,6 +1226,7 @@ sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fr
 
 sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {
     if (!c || !payload || !dev_status) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // checks the 2-bit payload only
     if (misaligned(payload)) return SL_ERR_ALIGNMENT;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
@@ -1161,6 +1241,7 @@ sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_st
 
 sl_status sl_read_stats(sl_ctx* c, int32_t worker, float* dev_out, void* stream) {
     if (!c || !dev_out || worker < 0 || worker >= c->last_workers) return SL_ERR_INVALID_ARG;
+    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // the 2-bit quantiser's table
     if (!c->ws_ptr) return SL_ERR_NOMEM;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");

@@ -52,7 +52,7 @@ class DeviceCase:
     write sits between guard bands, which check() and step() verify."""
 
     def __init__(self, wl: I.Workload, k: Optional[int] = None, distinct_local: Optional[int] = None,
-                 e_scale: float = 0.0, device=None, alias_shift: int = 0):
+                 e_scale: float = 0.0, device=None, alias_shift: int = 0, quant_bits: int = 2):
         from paper_2508_15706_b200.binding import SparseLoCo
         self.wl = wl
         self.k = wl.k if k is None else k
@@ -61,8 +61,9 @@ class DeviceCase:
         self.shapes = [(t.rows, t.cols) for t in wl.tensors]
         self.D = wl.R if distinct_local is None else distinct_local
         self.alias_shift = alias_shift if self.D < wl.R else 0
+        self.quant_bits = quant_bits
         self.sl = SparseLoCo(self.shapes, self.offs, k=self.k, R=wl.R, H=wl.H, beta=wl.beta,
-                             outer_lr=wl.outer_lr, alloc_workspace=False)
+                             outer_lr=wl.outer_lr, alloc_workspace=False, quant_bits=quant_bits)
         flat = I.flat_numel(wl.tensors)
         self.flat = flat
         self.guarded: List[Guarded] = []
@@ -94,11 +95,12 @@ class DeviceCase:
             self.payloads.append(buf)
         self.ws = guarded(self.sl.workspace_bytes(), torch.uint8)
         self.sl.set_workspace(self.ws)
-        self.cfg = O.Config(k=self.k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr)
+        self.cfg = O.Config(k=self.k, R=wl.R, H=wl.H, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=quant_bits)
         # payload geometry, from the oracle's definitions
         self.rec_off, self.n_chunks = [], []
-        stride = O.record_stride(self.k)
-        pos = 16 * len(self.shapes)
+        stride = O.record_stride_q(self.k, quant_bits)
+        self.hdr = O.header_bytes(quant_bits)
+        pos = self.hdr * len(self.shapes)
         for j, sh in enumerate(self.shapes):
             nc = O.num_chunks(self.cfg, O.Table([sh]), 0)
             self.rec_off.append(pos)
@@ -140,7 +142,7 @@ class DeviceCase:
 
     def tensor_payload(self, r: int, j: int) -> np.ndarray:
         p = self.payloads[r]
-        hdr = p[16 * j:16 * j + 16].cpu().numpy()
+        hdr = p[self.hdr * j:self.hdr * (j + 1)].cpu().numpy()
         recs = p[self.rec_off[j]:self.rec_off[j] + self.n_chunks[j] * self.stride].cpu().numpy()
         return np.concatenate([hdr, recs])
 
@@ -183,7 +185,7 @@ class DeviceCase:
         worst = 0.0
         report = {"tensors": 0, "payload_bytes": 0, "theta_max_err_over_rms": 0.0}
         cfg = O.Config(k=self.k, R=R, H=self.wl.H, beta=self.wl.beta, outer_lr=self.wl.outer_lr,
-                       ef_enabled=int(ef_enabled))
+                       ef_enabled=int(ef_enabled), quant_bits=self.quant_bits)
         for j, s in snap.items():
             t, off = self.wl.tensors[j], self.offs[j]
             tab = O.Table([(t.rows, t.cols)])

@@ -154,3 +154,56 @@ def test_outer_step_without_quantiser(ef_enabled):
         theta.copy_(torch.from_numpy(th_o))
     with pytest.raises(Exception):
         sl.compress(theta, local[0], e[0], torch.zeros(64, dtype=torch.uint8, device=dev))
+
+
+@pytest.mark.parametrize("bits,k", [(1, 64), (3, 64), (4, 64), (3, 41), (4, 123)])
+def test_quantiser_widths_of_the_ablation(bits, k):
+    """quant_bits 1, 3 and 4 (the paper's quantisation ablation; Sec. 4 defines the quantiser for any
+    width): the whole outer step against the oracle -- payload bytes (tables of 2^bits entries, codes of
+    `bits` bits) and error buffers bit for bit, theta within 1e-6 x RMS -- over two steps, on blocked,
+    flat, short and tiny tensors; and sl_compress + sl_aggregate_apply with an absent worker."""
+    from parity import DeviceCase, oracle_threads
+    oracle_threads()
+    tensors = TENSORS + [I.TensorSpec("wide", 320, 256, 4)]   # 20 chunks... and one of more than 64 chunks below
+    tensors = tensors + [I.TensorSpec("big", 576, 512, 5)]
+    wl = I.Workload("widths", tensors, R=3, k=k, recipe="student_t4", seed=300 + bits, outer_lr=0.7)
+    c = DeviceCase(wl, e_scale=0.5, quant_bits=bits)
+    assert c.sl.payload_bytes() == c.payload_bytes
+    for step in range(2):
+        c.fill_local(step)
+        snap = c.snapshot(range(len(tensors)))
+        c.step()
+        rep = c.check(snap)
+        assert rep["tensors"] == len(tensors)
+    # the two halves through their own entry points, worker 1 absent
+    c.fill_local(2)
+    snap = c.snapshot(range(len(tensors)))
+    for r in (0, 2):
+        c.sl.compress(c.theta, c.local_of(r), c.e[r], c.payloads[r])
+    e1 = c.e[1].clone()
+    c.sl.aggregate_apply([c.payloads[0], None, c.payloads[2]], c.theta)
+    torch.cuda.synchronize()
+    assert c.guards_intact()
+    c.e[1].copy_(e1)
+    cfg = O.Config(k=k, R=3, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=bits)
+    for j, t in enumerate(tensors):
+        tab = O.Table([(t.rows, t.cols)])
+        th = snap[j]["theta"].copy()
+        pays = []
+        for r in range(3):
+            if r == 1:
+                pays.append(None)
+                continue
+            out = O.compress(cfg, tab, snap[j]["theta"], snap[j]["local"][r], snap[j]["e"][r].copy())
+            assert np.array_equal(c.tensor_payload(r, j), out.payload), (t.name, r)
+            pays.append(out.payload)
+        O.aggregate_apply(cfg, tab, pays, th)
+        got = c.theta[c.offs[j]:c.offs[j] + t.numel].cpu().numpy()
+        rms = float(np.sqrt(np.mean(th.astype(np.float64) ** 2)))
+        assert float(np.max(np.abs(got.astype(np.float64) - th.astype(np.float64)))) <= 1e-6 * rms
+    from paper_2508_15706_b200 import binding as B
+    with pytest.raises(B.SlError) as ei:     # the wire codec, the validator and deferral serve the 2-bit payload only
+        c.sl.coded_payload_capacity()
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    with pytest.raises(B.SlError):
+        c.sl.set_ef_deferred(True)
