@@ -94,10 +94,12 @@ def test_ef_accumulate_freeze_and_beta_zero():
 
 # ----------------------------------------------------------------------------- Top-k
 
-@pytest.mark.parametrize("L,k", [(16, 1), (16, 5), (16, 16), (16, 20), (64, 7), (64, 63), (100, 33), (1, 1)])
+@pytest.mark.parametrize("L,k", [(16, 1), (16, 5), (16, 16), (16, 20), (64, 7), (64, 63), (100, 33), (1, 1),
+                                 (4096, 257), (4096, 512), (4096, 2048), (4096, 4095), (4096, 4096), (3000, 2048)])
 def test_topk_matches_bruteforce(L, k):
+    """(the densities of the paper's sweeps go up to 50 %, k = 2048 of 4096)"""
     rng = np.random.default_rng(L * 100 + k)
-    for trial in range(20):
+    for trial in range(20 if L <= 100 else 6):
         u = rng.standard_normal(L).astype(np.float32)
         if trial % 3 == 1:  # heavy ties, both signs
             u = (rng.integers(-2, 3, L)).astype(np.float32)
@@ -110,7 +112,7 @@ def test_topk_matches_bruteforce(L, k):
 
 def test_topk_invariants_full_chunk():
     rng = np.random.default_rng(7)
-    for k in (1, 41, 64, 123, 256):
+    for k in (1, 41, 64, 123, 256, 300, 1024, 2048):
         u = rng.standard_normal(4096).astype(np.float32)
         u[rng.integers(0, 4096, 300)] = np.float32(0.5)  # a tie group
         idx = O.topk_chunk(u, k)
@@ -278,7 +280,7 @@ def test_pack_handworked_bytes():
     assert list(rec[:6]) == [0x07, 0x80, 0x00, 0x00, 0x00, 0x0F]
 
 
-@pytest.mark.parametrize("k", [1, 41, 64, 82, 123, 256])
+@pytest.mark.parametrize("k", [1, 41, 64, 82, 123, 256, 257, 1000, 2048])
 def test_pack_roundtrip_and_stride(k):
     rng = np.random.default_rng(k)
     idx = np.sort(rng.choice(4096, k, replace=False)).astype(np.int32)
