@@ -73,7 +73,11 @@ typedef struct {
 typedef struct {
     int32_t chunk_elems;       /* C: must be 4096 */
     int32_t tile_dim;          /* must be 64 */
-    int32_t k;                 /* entries kept per chunk, 1..256 */
+    int32_t k;                 /* entries kept per chunk, 1..2048 (the paper's density sweeps reach half a
+                                  chunk).  The tuned kernels serve k <= 256; beyond that the selection is the exact
+                                  bitwise search and packing / decoding run in the plain kernels of the
+                                  quantiser ablation: no deferral, no wire codec, no validation, no quant_bits = 32,
+                                  no Top-k baselines */
     int32_t R;                 /* workers, 1..64 */
     int32_t H;                 /* inner steps; carried for the caller, >= 1, unused by the math */
     float beta;                /* error-feedback decay, 0 <= beta <= 1 */

@@ -9,7 +9,8 @@ constexpr int kTile = 64;
 constexpr int kThreads = 256;          // threads per CTA of the chunk kernels
 constexpr int kPerThread = kChunk / kThreads;  // 16 elements = 4 x float4
 constexpr int kMaxR = 64;
-constexpr int kMaxK = 256;
+constexpr int kMaxK = 2048;      // half a chunk: the densest setting of the paper's sweeps
+constexpr int kFastMaxK = 256;   // largest k of the fused 2-bit kernels, the waiting lists and the wire codec
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kProfSlots = 9;     // kernels of one outer step
 constexpr int kProfMaxSeq = 256;  // recorded sequences kept between two reads

@@ -121,8 +121,8 @@ struct SelSmem {
     float theta_s[kThetaRing][kChunk];
     float theta_l[kUnitSlots][kChunk];
     float e[kUnitSlots][kChunk];
-    __align__(16) float pend_val[kUnitSlots][kMaxK];
-    __align__(16) uint16_t pend_idx[kUnitSlots][kMaxK];
+    __align__(16) float pend_val[kUnitSlots][kFastMaxK];
+    __align__(16) uint16_t pend_idx[kUnitSlots][kFastMaxK];
     __align__(16) unsigned bitmap[kSelWarps][128];
     uint16_t cand[kSelWarps][kCandCap];
     unsigned long long full_s[kThetaRing], empty_s[kThetaRing];  // theta block landed / all R units done with it
@@ -413,6 +413,10 @@ __device__ __forceinline__ void select_unit(const float (&u)[128], const USource
     // groups of 16 values up to k = 128 (about 1.15 k candidates); beyond that a threshold taken from 256
     // group maxima lets too many elements through, and groups of 4 take over (WIDE: a kernel of its own,
     // so that the common case carries neither the code nor the registers of the other)
+    if (WIDE && keff > kFastMaxK) {  // beyond 256 of 4096 a threshold over group maxima no longer thins the field
+        select_slow<GLOBAL>(src, len, keff, bitmap, out_idx, out_val);
+        return;
+    }
     unsigned T, probe;
     group_threshold<WIDE ? 32 : 8>(u, keff, T, probe);
     if (T == 0u) {  // no usable threshold: exact search over everything

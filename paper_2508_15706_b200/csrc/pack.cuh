@@ -17,7 +17,7 @@ template <int MODE>
 __global__ void __launch_bounds__(128)
 pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
                 int k, int kp, Workspace ws, WorkerPtrs ptrs) {
-    __shared__ __align__(16) unsigned rec[4][(record_stride(kMaxK) / 4) + 4];
+    __shared__ __align__(16) unsigned rec[4][(record_stride(kFastMaxK) / 4) + 4];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long i = (long long)blockIdx.x * 4 + warp;
     if (i >= n_chunks * n_workers) return;

@@ -129,10 +129,14 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 // general-width quantiser (quant_bits 1, 3, 4): its per-unit bin partials and per-tensor tables follow
 // the arrays of the 2-bit path in the workspace
-inline bool wide_quant(const sl_ctx* c) { return c->cfg.quant_bits != 2 && c->cfg.quant_bits != 32; }
+// (also the 2-bit quantiser at k > 256, which the fused kernels are not laid out for)
+inline bool wide_quant(const sl_ctx* c) {
+    return c->cfg.quant_bits != 32 && (c->cfg.quant_bits != 2 || c->cfg.k > kFastMaxK);
+}
+inline bool fast_2bit(const sl_ctx* c) { return c->cfg.quant_bits == 2 && c->cfg.k <= kFastMaxK; }
 size_t wide_bytes_for(const sl_ctx* c, int workers) {
     if (!wide_quant(c)) return 0;
-    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->cfg.quant_bits;
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->qbits;
     return up256(WG * nb * sizeof(double)) + up256(WG * nb * sizeof(unsigned)) +
            up256((size_t)workers * c->n_tensors * sizeof(TStatQ));
 }
@@ -152,7 +156,7 @@ struct WideSpace {
     TStatQ* tq;
 };
 WideSpace carve_wide(const sl_ctx* c, int workers) {
-    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->cfg.quant_bits;
+    const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->qbits;
     char* p = static_cast<char*>(c->ws_ptr) + narrow_bytes_for(c, workers);
     WideSpace w;
     w.pbin = reinterpret_cast<double*>(p);      p += up256(WG * nb * sizeof(double));
@@ -380,8 +384,9 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
         else                                                                                                        \
             pack_q_kernel<BITSV, false><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
     } while (0)
-        if (c->cfg.quant_bits == 1) SL_WIDE(1);
-        else if (c->cfg.quant_bits == 3) SL_WIDE(3);
+        if (c->qbits == 1) SL_WIDE(1);
+        else if (c->qbits == 2) SL_WIDE(2);
+        else if (c->qbits == 3) SL_WIDE(3);
         else SL_WIDE(4);
 #undef SL_WIDE
         prof_mark(c, 5, st);
@@ -422,9 +427,11 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
     if (wide_quant(c) && fuse == 0) {  // payloads of 1, 3 or 4 bits per value
         const unsigned grid = (unsigned)c->n_chunks;
-        if (c->cfg.quant_bits == 1)
+        if (c->qbits == 1)
             apply_q_kernel<1><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
-        else if (c->cfg.quant_bits == 3)
+        else if (c->qbits == 2)
+            apply_q_kernel<2><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
+        else if (c->qbits == 3)
             apply_q_kernel<3><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
         else
             apply_q_kernel<4><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
@@ -515,6 +522,7 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (cfg->chunk_elems != kChunk || cfg->tile_dim != kTile) return SL_ERR_UNSUPPORTED;
     if (cfg->quant_bits != 32 && (cfg->quant_bits < 1 || cfg->quant_bits > 4)) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
+    if (cfg->k > kFastMaxK && cfg->quant_bits == 32) return SL_ERR_UNSUPPORTED;  // the unquantised kernels stop at 256
 
     {   // element ranges: no overflow, no two tensors sharing an element (kernels of different chunks would race)
         std::vector<std::pair<long long, long long>> span((size_t)n_tensors);
@@ -655,7 +663,7 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
 #undef SL_SELECT_ATTR_D
     per_sm = 1;
     {   // the apply kernel's shared memory depends on k alone: sized once
-        const int asz = (int)apply_smem_bytes(cfg->k);
+        const int asz = (int)apply_smem_bytes(cfg->k < kFastMaxK ? cfg->k : kFastMaxK);
 #define SL_APPLY_ATTR(PPLV, FUSEV)                                                                                     \
     if (e == cudaSuccess)                                                                                              \
         e = cudaFuncSetAttribute(decode_avg_apply_kernel<PPLV, FUSEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, asz)
@@ -1017,6 +1025,7 @@ sl_status sl_lom_step(sl_ctx* c, float* theta_sync, const float* const* theta_lo
     if (!m_r) return SL_ERR_INVALID_ARG;
     sl_status s = variant_args(c, theta_sync, theta_local, nullptr, m_r, mu, ptrs);
     if (s != SL_OK) return s;
+    if (sub_k && c->cfg.k > kFastMaxK) return SL_ERR_UNSUPPORTED;  // the unquantised kernels stop at 256
     if (sub_k && (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R))) return SL_ERR_NOMEM;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
@@ -1049,6 +1058,7 @@ sl_status sl_diloco_topk_step(sl_ctx* c, float* theta_sync, const float* const* 
     if (!momentum) return SL_ERR_INVALID_ARG;
     sl_status s = variant_args(c, theta_sync, theta_local, e, nullptr, mu, ptrs);
     if (s != SL_OK) return s;
+    if (c->cfg.k > kFastMaxK) return SL_ERR_UNSUPPORTED;  // the unquantised kernels stop at 256
     if (misaligned(momentum)) return SL_ERR_ALIGNMENT;
     if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R)) return SL_ERR_NOMEM;
     DeviceGuard g(c->device);
@@ -1074,6 +1084,7 @@ sl_status sl_lom_topk_step(sl_ctx* c, float* theta_sync, float* const* theta_loc
     if (!m_r) return SL_ERR_INVALID_ARG;
     sl_status s = variant_args(c, theta_sync, theta_local, e, m_r, mu, ptrs);
     if (s != SL_OK) return s;
+    if (c->cfg.k > kFastMaxK) return SL_ERR_UNSUPPORTED;  // the unquantised kernels stop at 256
     if (!c->ws_ptr || c->ws_bytes < workspace_bytes_for(c, c->cfg.R)) return SL_ERR_NOMEM;
     const int R = c->cfg.R;
     for (int r = 0; r < R; ++r)
@@ -1108,7 +1119,7 @@ sl_status sl_lom_topk_step(sl_ctx* c, float* theta_sync, float* const* theta_loc
 
 sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {
     if (!c || !bytes) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;  // the stream's bit offsets are 32-bit
     *bytes = c->ixc_capacity;
     return SL_OK;
@@ -1117,7 +1128,7 @@ sl_status sl_coded_payload_capacity(const sl_ctx* c, size_t* bytes) {
 sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, uint64_t* dev_coded_bytes,
                             void* stream) {
     if (!c || !payload || !coded || !dev_coded_bytes) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (misaligned(payload) || misaligned(coded) || (reinterpret_cast<uintptr_t>(dev_coded_bytes) & 7u))
         return SL_ERR_ALIGNMENT;
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
@@ -1143,7 +1154,7 @@ sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, u
 
 sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, size_t coded_bytes, uint8_t* payload, void* stream) {
     if (!c || !coded || !payload) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
     if (misaligned(coded) || misaligned(payload)) return SL_ERR_ALIGNMENT;
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
     // what the buffer is said to hold bounds every read; it must at least reach the index stream
@@ -1182,7 +1193,7 @@ sl_status sl_device_status(sl_ctx* c, void* stream) {
 
 sl_status sl_set_ef_deferred(sl_ctx* c, int32_t on) {
     if (!c) return SL_ERR_INVALID_ARG;
-    if (on && c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // only the 2-bit path defers
+    if (on && !fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // only the 2-bit path defers
     c->deferred = on != 0;
     return SL_OK;
 }
@@ -1226,7 +1237,7 @@ sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fr
 
 sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {
     if (!c || !payload || !dev_status) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // checks the 2-bit payload only
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // checks the 2-bit payload only
     if (misaligned(payload)) return SL_ERR_ALIGNMENT;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
@@ -1241,7 +1252,7 @@ sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_st
 
 sl_status sl_read_stats(sl_ctx* c, int32_t worker, float* dev_out, void* stream) {
     if (!c || !dev_out || worker < 0 || worker >= c->last_workers) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits != 2) return SL_ERR_UNSUPPORTED;  // the 2-bit quantiser's table
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // the 2-bit quantiser's table
     if (!c->ws_ptr) return SL_ERR_NOMEM;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
@@ -1323,7 +1334,7 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
                                     int64_t rows, int64_t cols, int32_t k, float beta, void* stream) {
     if (!theta_sync || !theta_local || !e || !payload) return SL_ERR_INVALID_ARG;
     if (rows < 1 || cols < 1 || k < 1 || !(beta >= 0.0f && beta <= 1.0f)) return SL_ERR_INVALID_ARG;
-    if (k > kMaxK) return SL_ERR_UNSUPPORTED;
+    if (k > kFastMaxK) return SL_ERR_UNSUPPORTED;
     if (misaligned(theta_sync) || misaligned(theta_local) || misaligned(e) || misaligned(payload)) return SL_ERR_ALIGNMENT;
     if (cols > 0x7FFFFFFFll || rows > (1ll << 40) / cols) return SL_ERR_TOO_LARGE;
     const long long n = rows * cols;

@@ -448,7 +448,7 @@ def test_argument_errors():
         B.SparseLoCo([(64, 64)], k=0, R=1)
     assert ei.value.status == B.SL_ERR_INVALID_ARG
     with pytest.raises(B.SlError) as ei:
-        B.SparseLoCo([(64, 64)], k=300, R=1)
+        B.SparseLoCo([(64, 64)], k=2049, R=1)
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
     with pytest.raises(B.SlError) as ei:
         B.SparseLoCo([(64, 64), (1, 10)], offsets=[0, 4098], k=8, R=1)

@@ -207,3 +207,32 @@ def test_quantiser_widths_of_the_ablation(bits, k):
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
     with pytest.raises(B.SlError):
         c.sl.set_ef_deferred(True)
+
+
+@pytest.mark.parametrize("bits,k", [(2, 257), (2, 512), (2, 2048), (4, 1000), (1, 2048)])
+def test_densities_up_to_half_a_chunk(bits, k):
+    """k beyond 256, up to 2048 of 4096 (the densest setting of the paper's density sweeps): the whole
+    outer step against the oracle, payload and error buffers bit for bit, theta within 1e-6 x RMS, two
+    steps; chunks shorter than k send all they have."""
+    from parity import DeviceCase, oracle_threads
+    oracle_threads()
+    tensors = TENSORS + [I.TensorSpec("big", 576, 512, 5)]
+    wl = I.Workload("dense_k", tensors, R=3, k=k, recipe="student_t4", seed=400 + k + bits, outer_lr=0.7)
+    c = DeviceCase(wl, e_scale=0.5, quant_bits=bits)
+    assert c.sl.payload_bytes() == c.payload_bytes
+    for step in range(2):
+        c.fill_local(step)
+        snap = c.snapshot(range(len(tensors)))
+        c.step()
+        rep = c.check(snap)
+        assert rep["tensors"] == len(tensors)
+    from paper_2508_15706_b200 import binding as B
+    with pytest.raises(B.SlError) as ei:     # deferral, the wire codec and the validator stop at k = 256
+        c.sl.set_ef_deferred(True)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    with pytest.raises(B.SlError) as ei:     # and so does the path without a quantiser
+        B.SparseLoCo(c.shapes, c.offs, k=k, R=3, quant_bits=32, alloc_workspace=False)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    with pytest.raises(B.SlError) as ei:
+        B.SparseLoCo(c.shapes, c.offs, k=2049, R=3, alloc_workspace=False)
+    assert ei.value.status == B.SL_ERR_UNSUPPORTED
