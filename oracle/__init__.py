@@ -37,7 +37,7 @@ class _Config(C.Structure):
     _fields_ = [("chunk_elems", C.c_int32), ("tile_dim", C.c_int32), ("k", C.c_int32),
                 ("R", C.c_int32), ("H", C.c_int32), ("beta", C.c_float), ("outer_lr", C.c_float),
                 ("quant_bits", C.c_int32), ("ef_enabled", C.c_int32),
-                ("divide_by_present", C.c_int32)]
+                ("divide_by_present", C.c_int32), ("storage_bf16", C.c_int32)]
 
 
 @dataclass
@@ -52,10 +52,12 @@ class Config:
     quant_bits: int = 2
     ef_enabled: int = 1
     divide_by_present: int = 0
+    storage_bf16: int = 0   # 1: theta, theta_r, e hold bfloat16 values (as fp32 arrays); stores are rounded
 
     def c(self) -> _Config:
         return _Config(self.chunk_elems, self.tile_dim, self.k, self.R, self.H, self.beta,
-                       self.outer_lr, self.quant_bits, self.ef_enabled, self.divide_by_present)
+                       self.outer_lr, self.quant_bits, self.ef_enabled, self.divide_by_present,
+                       self.storage_bf16)
 
 
 def lib():
@@ -78,6 +80,10 @@ def lib():
             getattr(L, nm).argtypes = [P, P, C.c_int32]
         L.orc_record_stride.restype = C.c_int64
         L.orc_record_stride.argtypes = [C.c_int32]
+        L.orc_bf16_round.restype = C.c_float
+        L.orc_bf16_round.argtypes = [C.c_float]
+        L.orc_bf16_round_d.restype = C.c_float
+        L.orc_bf16_round_d.argtypes = [C.c_double]
         L.orc_ef_accumulate.argtypes = [P, P, P, C.c_int64, C.c_float, C.c_int, P]
         L.orc_topk_chunk.restype = C.c_int32
         L.orc_topk_chunk.argtypes = [P, C.c_int32, C.c_int32, P]
@@ -284,6 +290,16 @@ def compress(cfg: Config, tab: Table, theta: np.ndarray, theta_r: np.ndarray, e:
                        _ptr(_chk(theta_r, np.float32)), _ptr(_chk(e, np.float32)), _ptr(payload),
                        _ptr(sel_idx), _ptr(sel_val), _ptr(sel_hat), _ptr(stats))
     return Compressed(payload, sel_idx[:slots], sel_val[:slots], sel_hat[:slots], stats)
+
+
+def bf16_round(x: float) -> float:
+    """The bfloat16 nearest to x (ties to even), x an fp32 value; returned as a Python float."""
+    return float(lib().orc_bf16_round(float(x)))
+
+
+def bf16_round_d(x: float) -> float:
+    """The bfloat16 nearest to the double x (ties to even), in one rounding."""
+    return float(lib().orc_bf16_round_d(float(x)))
 
 
 def decode_payload(cfg: Config, tab: Table, payload: np.ndarray):

@@ -38,6 +38,12 @@
  *     stores +0.
  *   - the average divides by R even when a worker's payload is absent, unless
  *     divide_by_present is set.
+ *   - bf16 storage (storage_bf16 = 1; the paper does not speak of storage types): theta,
+ *     theta_r and e hold bfloat16 values (here: fp32 arrays whose entries are bf16-representable).
+ *     All arithmetic is the fp32 / fp64 arithmetic above on the widened values, so the selection
+ *     and the quantiser see the unrounded u; only what is stored is rounded, once, to nearest-even
+ *     bfloat16: e = bf16(u) where nothing was selected, e = bf16(u - Delta_hat) where something
+ *     was, theta = bf16(theta - alpha Delta) for the elements some worker selected.
  *
  * Every function here is pinned by tests/test_oracle_*.py against brute force,
  * hand-worked cases, closed forms and invariants (none of them produced by this
@@ -69,7 +75,23 @@ typedef struct {
     int32_t quant_bits;        /* 2 (the paper's setting), 1 / 3 / 4 (its ablation), or 32 = values sent unquantised */
     int32_t ef_enabled;        /* 0 during the error-feedback freeze */
     int32_t divide_by_present; /* 0: divide by R; 1: by the number of payloads present */
+    int32_t storage_bf16;      /* 1: theta, theta_r and e are bfloat16 values; results are rounded on store */
 } orc_config;
+
+/* ---------------------------------------------------------------- bfloat16 rounding
+ * bfloat16 = sign, 8 exponent bits, 7 fraction bits (the upper half of an fp32).  Round to nearest,
+ * ties to even, in one step from the given value: |x| = f 2^ex with f in [0.5, 1) has its 8
+ * significant bits down to 2^(ex - 8); subnormals (below 2^-126) share the spacing 2^-133. */
+float orc_bf16_round_d(double x) {
+    if (x == 0.0 || !isfinite(x)) return (float)x;
+    int ex;
+    (void)frexp(x, &ex);
+    int lsb = ex - 8;
+    if (lsb < -133) lsb = -133;
+    double q = nearbyint(ldexp(x, -lsb)); /* exact scaling; nearbyint rounds half to even (default mode) */
+    return (float)ldexp(q, lsb);
+}
+float orc_bf16_round(float x) { return orc_bf16_round_d((double)x); }
 
 static int g_threads = 1;
 void orc_set_threads(int n) { g_threads = n < 1 ? 1 : n; }
@@ -532,6 +554,8 @@ void orc_compress(const orc_config* cfg, const orc_tensor* ts, int32_t nt, const
                     int64_t pos = orc_chunk_pos(cfg, t, ch, idx[ch * k + s]);
                     ej[pos] = u[pos] - vhat[w];
                 }
+            if (cfg->storage_bf16) /* the stored error is the bfloat16 nearest to it */
+                for (int64_t i = 0; i < n; ++i) ej[i] = orc_bf16_round(ej[i]);
         }
 
         {
@@ -592,7 +616,9 @@ void orc_aggregate_apply_sparse(const orc_config* cfg, const orc_tensor* ts, int
         }
         float* th = theta + t->offset;
         for (int64_t i = 0; i < n; ++i) {
-            if (hit[i]) th[i] = (float)((double)th[i] - (double)cfg->outer_lr * acc[i] / D);
+            if (!hit[i]) continue;
+            const double x = (double)th[i] - (double)cfg->outer_lr * acc[i] / D;
+            th[i] = cfg->storage_bf16 ? orc_bf16_round_d(x) : (float)x;
         }
         slot_off += m_tensor;
         free(acc); free(hit);
