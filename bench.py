@@ -451,6 +451,7 @@ def sharing_check(torch, I, dev, peak: float) -> dict:
 
     import dataclasses
     out["variants_c5_l12_R8"] = variants_bench(torch, I, dev, build, peak)
+    out["options_c5_l12_R8"] = options_bench(torch, I, dev, peak)
     wl = dataclasses.replace(I.workload(DEFAULT_WORKLOAD), R=8)
     N = wl.numel
     sl, ws, theta, e, payloads = build(wl)
@@ -513,6 +514,55 @@ def variants_bench(torch, I, dev, build, peak: float) -> dict:
                      "frac_of_measured_peak": bpp * N / (ms * 1e-3) / 1e9 / peak}
     del sl, ws, theta, e, payloads, local, m_r, mom
     torch.cuda.empty_cache()
+    return out
+
+
+def options_bench(torch, I, dev, peak: float) -> dict:
+    """The settings outside the paper's main configuration (quantiser widths of its ablation, no quantiser,
+    densities up to half a chunk, bfloat16 storage) on the 12-layer stack with R = 8: ms per outer step and
+    the rate on the state the step must stream ((12 R + 8) bytes per parameter in fp32, half in bfloat16:
+    theta_r and e read, e written per worker; theta read and written).  These run in plain kernels."""
+    import dataclasses
+    from paper_2508_15706_b200.binding import SparseLoCo
+    base = dataclasses.replace(I.workload("c5_l12"), R=8)
+    N, R = base.numel, 8
+    shapes, offs = [(t.rows, t.cols) for t in base.tensors], I.offsets(base.tensors)
+    theta32 = I.theta_sync(base, dev)
+    local32 = [I.theta_local(base, theta32, r, 0) for r in range(R)]
+    e32 = [I.initial_error(base, r, dev, scale=0.5) for r in range(R)]
+    stream = torch.cuda.current_stream()
+    cases = [("quant_bits=2 k=64 (the tuned path, materialised subtraction)", 2, 64, False),
+             ("quant_bits=1 k=64", 1, 64, False), ("quant_bits=3 k=64", 3, 64, False), ("quant_bits=4 k=64", 4, 64, False),
+             ("quant_bits=32 k=64 (no quantiser)", 32, 64, False),
+             ("quant_bits=2 k=512", 2, 512, False), ("quant_bits=2 k=2048", 2, 2048, False),
+             ("bf16 storage, quant_bits=2 k=64", 2, 64, True)]
+    out = {"params": N, "R": R}
+    for name, bits, k, half in cases:
+        sl = SparseLoCo(shapes, offs, k=k, R=R, beta=base.beta, outer_lr=base.outer_lr, quant_bits=bits,
+                        bf16_storage=half)
+        pay = [torch.zeros(sl.payload_bytes() if bits != 32 else 16, dtype=torch.uint8, device=dev) for _ in range(R)]
+        if half:
+            theta = theta32.to(torch.bfloat16)
+            local = [x.to(torch.bfloat16) for x in local32]
+            e = [x.to(torch.bfloat16) for x in e32]
+        else:
+            theta, local, e = theta32.clone(), local32, [x.clone() for x in e32]
+        for _ in range(2):
+            sl.outer_step(theta, local, e, pay)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(3):
+            sl.outer_step(theta, local, e, pay)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 3
+        bpp = (12 * R + 8) * (0.5 if half else 1.0)
+        out[name] = {"ms_per_step": ms, "state_bytes_per_param": bpp, "gbs": bpp * N / (ms * 1e-3) / 1e9,
+                     "frac_of_measured_peak": bpp * N / (ms * 1e-3) / 1e9 / peak}
+        del sl, pay, theta, e
+        if half:
+            del local
+        torch.cuda.empty_cache()
     return out
 
 

@@ -90,6 +90,8 @@ typedef struct {
     int32_t ef_enabled;        /* 0 during the error-feedback freeze (App. "Freezing Error
                                   Feedback"): u = Delta and e is neither read nor written */
     int32_t divide_by_present; /* 0: average divides by R (Alg. 1); 1: by the payloads present */
+    int32_t bf16_storage;      /* 0: theta, theta_r, e are fp32 arrays.  1: bfloat16 arrays, served by the
+                                  sl_*_bf16 entry points only (see there); not with quant_bits = 32 */
 } sl_config;
 
 typedef struct sl_ctx sl_ctx;
@@ -148,6 +150,25 @@ sl_status sl_aggregate_apply(sl_ctx* ctx, const uint8_t* const* payloads, float*
  * replay would not advance). */
 sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* theta_local,
                         float* const* e, uint8_t* const* payloads, void* cuda_stream);
+
+/* The same three calls for a context created with bf16_storage = 1: theta_sync, theta_local and e are
+ * arrays of bfloat16 bit patterns (the upper halves of fp32 values), same element offsets, same
+ * alignment rules (16-byte aligned pointers).  The paper states the method (Alg. 1, Eq. 2) without
+ * naming a storage type; this mode halves the state the outer step streams.  Definition: all
+ * arithmetic is that of the fp32 calls on the widened values -- Delta = theta - theta_r,
+ * u = fma(beta, e, Delta), selection and quantiser on the unrounded u, so the payload is the one the
+ * fp32 calls would write for these inputs -- and every store rounds once to the nearest bfloat16,
+ * ties to even: e = bf16(u), or bf16(u - table[code]) at the selected positions;
+ * theta = bf16(fma(-alpha / D, sum, theta)) where some worker selected the element, else unchanged.
+ * Plain kernels (no tile copies, no fusion, no deferral); any k up to 2048 and quant_bits 1..4.
+ * Errors as for the fp32 calls; UNSUPPORTED when the context is not a bf16_storage one (and the
+ * fp32 calls return UNSUPPORTED for a context that is). */
+sl_status sl_compress_bf16(sl_ctx* ctx, const uint16_t* theta_sync, const uint16_t* theta_local, uint16_t* e,
+                           uint8_t* payload, void* cuda_stream);
+sl_status sl_aggregate_apply_bf16(sl_ctx* ctx, const uint8_t* const* payloads, uint16_t* theta_sync,
+                                  void* cuda_stream);
+sl_status sl_outer_step_bf16(sl_ctx* ctx, uint16_t* theta_sync, const uint16_t* const* theta_local,
+                             uint16_t* const* e, uint8_t* const* payloads, void* cuda_stream);
 
 /* Dense baseline on the same buffers: DiLoCo's outer step with Nesterov outer momentum (Eq. 1),
  *     Dbar = (1/R) sum_r (theta - theta_r);  m = beta_outer m + Dbar;

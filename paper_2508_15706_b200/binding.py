@@ -20,6 +20,7 @@ EXPORTS = (
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
     "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step", "sl_streaming_due",
+    "sl_compress_bf16", "sl_aggregate_apply_bf16", "sl_outer_step_bf16",
 )
 PROFILE_SLOTS = 9
 
@@ -42,7 +43,7 @@ class _Config(C.Structure):
     _fields_ = [("chunk_elems", C.c_int32), ("tile_dim", C.c_int32), ("k", C.c_int32),
                 ("R", C.c_int32), ("H", C.c_int32), ("beta", C.c_float), ("outer_lr", C.c_float),
                 ("quant_bits", C.c_int32), ("ef_enabled", C.c_int32),
-                ("divide_by_present", C.c_int32)]
+                ("divide_by_present", C.c_int32), ("bf16_storage", C.c_int32)]
 
 
 def _load():
@@ -65,6 +66,9 @@ def _load():
     L.sl_compress.argtypes = [P, P, P, P, P, P]
     L.sl_aggregate_apply.argtypes = [P, P, P, P]
     L.sl_outer_step.argtypes = [P, P, P, P, P, P]
+    L.sl_compress_bf16.argtypes = [P, P, P, P, P, P]
+    L.sl_aggregate_apply_bf16.argtypes = [P, P, P, P]
+    L.sl_outer_step_bf16.argtypes = [P, P, P, P, P, P]
     L.sl_outer_step_host.argtypes = [P, P, P, P, C.c_size_t, P, P, P, P]
     L.sl_profile_enable.argtypes = [P, C.c_int32]
     L.sl_profile_read.argtypes = [P, P, P]
@@ -157,7 +161,8 @@ class SparseLoCo:
     def __init__(self, shapes: Sequence[Sequence[int]], offsets: Optional[Sequence[int]] = None, *,
                  k: int, R: int, H: int = 1, beta: float = 0.95, outer_lr: float = 1.0,
                  ef_enabled: bool = True, divide_by_present: bool = False, chunk_elems: int = 4096,
-                 tile_dim: int = 64, quant_bits: int = 2, alloc_workspace: bool = True):
+                 tile_dim: int = 64, quant_bits: int = 2, alloc_workspace: bool = True,
+                 bf16_storage: bool = False):
         n = len(shapes)
         descs = (_TensorDesc * n)()
         pos = 0
@@ -167,7 +172,9 @@ class SparseLoCo:
             descs[j] = _TensorDesc(rows, cols, off)
             pos = off + rows * cols
         cfg = _Config(chunk_elems, tile_dim, k, R, H, beta, outer_lr, quant_bits, int(ef_enabled),
-                      int(divide_by_present))
+                      int(divide_by_present), int(bf16_storage))
+        # element type of theta, theta_local and e; the library has one set of entry points per type
+        self.dtype = torch.bfloat16 if bf16_storage else torch.float32
         self._h = C.c_void_p()
         self.k, self.R = k, R
         self._beta, self._lr, self._ef, self._dbp = beta, outer_lr, int(ef_enabled), int(divide_by_present)
@@ -230,19 +237,22 @@ class SparseLoCo:
 
     # -- the path
     def compress(self, theta_sync, theta_local, e, payload) -> None:
-        _check(_L.sl_compress(self._h, _dev_ptr(theta_sync, torch.float32), _dev_ptr(theta_local, torch.float32),
-                              _dev_ptr(e, torch.float32), _dev_ptr(payload, torch.uint8), _stream()))
+        fn = _L.sl_compress_bf16 if self.dtype == torch.bfloat16 else _L.sl_compress
+        _check(fn(self._h, _dev_ptr(theta_sync, self.dtype), _dev_ptr(theta_local, self.dtype),
+                  _dev_ptr(e, self.dtype), _dev_ptr(payload, torch.uint8), _stream()))
 
     def aggregate_apply(self, payloads: List[Optional[torch.Tensor]], theta_sync) -> None:
         arr = _ptr_array([_dev_ptr(p, torch.uint8) for p in payloads])
-        _check(_L.sl_aggregate_apply(self._h, arr, _dev_ptr(theta_sync, torch.float32), _stream()))
+        fn = _L.sl_aggregate_apply_bf16 if self.dtype == torch.bfloat16 else _L.sl_aggregate_apply
+        _check(fn(self._h, arr, _dev_ptr(theta_sync, self.dtype), _stream()))
 
     def outer_step(self, theta_sync, theta_local: List[torch.Tensor], e: Optional[List[torch.Tensor]],
                    payloads: List[torch.Tensor]) -> None:
-        tl = _ptr_array([_dev_ptr(t, torch.float32) for t in theta_local])
-        ea = _ptr_array([_dev_ptr(t, torch.float32) for t in e]) if e is not None else None
+        tl = _ptr_array([_dev_ptr(t, self.dtype) for t in theta_local])
+        ea = _ptr_array([_dev_ptr(t, self.dtype) for t in e]) if e is not None else None
         pa = _ptr_array([_dev_ptr(t, torch.uint8) for t in payloads])
-        _check(_L.sl_outer_step(self._h, _dev_ptr(theta_sync, torch.float32), tl, ea, pa, _stream()))
+        fn = _L.sl_outer_step_bf16 if self.dtype == torch.bfloat16 else _L.sl_outer_step
+        _check(fn(self._h, _dev_ptr(theta_sync, self.dtype), tl, ea, pa, _stream()))
 
     def outer_step_host(self, theta_sync, theta_local_host: List[torch.Tensor], dev_stage,
                         e: Optional[List[torch.Tensor]], payloads: List[torch.Tensor],

@@ -3,6 +3,7 @@
 #pragma once
 #include "common.cuh"
 #include "quantiser.cuh"
+#include <cuda_bf16.h>
 
 // ================================================================================================
 // Sec. 4 describes the quantiser for any width: values centred by the tensor's mean, [-6 sigma, 6 sigma]
@@ -117,7 +118,8 @@ tensor_table_q_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, 
 }
 
 // Codes, record, and (FIX) e[index] = value - table[code].  One warp per (worker, chunk).
-template <int BITS, bool FIX>
+// HALF: the error buffers are bfloat16 arrays and the corrected value is rounded to nearest-even on the store.
+template <int BITS, bool FIX, bool HALF = false>
 __global__ void __launch_bounds__(128)
 pack_q_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors, int k, int kp,
               Workspace ws, const TStatQ* __restrict__ tq, long long rec_base, WorkerPtrs ptrs) {
@@ -146,8 +148,12 @@ pack_q_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_wo
         const int cbit = code_bit0 + BITS * s;
         atomicOr(&rec[warp][cbit >> 5], (unsigned)c << (cbit & 31));
         if ((cbit & 31) + BITS > 32) atomicOr(&rec[warp][(cbit >> 5) + 1], (unsigned)c >> (32 - (cbit & 31)));
-        if (FIX && p < (unsigned)cd.len)
-            ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = __fsub_rn(v, lut->lut[c]);
+        if (FIX && p < (unsigned)cd.len) {
+            const long long at = cd.base + chunk_elem_offset(cd.row_stride, (int)p);
+            const float fix = __fsub_rn(v, lut->lut[c]);
+            if (HALF) reinterpret_cast<__nv_bfloat16*>(ptrs.e[r])[at] = __float2bfloat16_rn(fix);
+            else ptrs.e[r][at] = fix;
+        }
     }
     __syncwarp();
     uint4* dst = reinterpret_cast<uint4*>(ptrs.payload[r] + rec_base + (long long)stride * g);
@@ -158,7 +164,8 @@ pack_q_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_wo
 // Decode + average + outer update from payloads of general width.  One CTA of 256 threads per chunk;
 // the workers are taken one after the other (a CTA barrier in between), so every position receives
 // its values in ascending worker order, as in decode_avg_apply_kernel.
-template <int BITS>
+// HALF: theta is a bfloat16 array, widened for the update and rounded to nearest-even on the store.
+template <int BITS, bool HALF = false>
 __global__ void __launch_bounds__(kThreads)
 apply_q_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float scale, PayloadPtrs pl, long long rec_base,
                float* __restrict__ theta_sync) {
@@ -187,6 +194,15 @@ apply_q_kernel(const ChunkDesc* __restrict__ chunks, int n_workers, int k, float
         }
     }
     __syncthreads();
+    if (HALF) {
+        __nv_bfloat16* __restrict__ th = reinterpret_cast<__nv_bfloat16*>(theta_sync) + cd.base;
+        for (int p = tid; p < cd.len; p += kThreads) {
+            const float a = acc[p];
+            const long long at = chunk_elem_offset(cd.row_stride, p);
+            if (!(scale < 0.0f && __float_as_uint(a) == 0u)) th[at] = __float2bfloat16_rn(__fmaf_rn(scale, a, __bfloat162float(th[at])));
+        }
+        return;
+    }
     float* __restrict__ th = theta_sync + cd.base;
     for (int p = tid; p < cd.len; p += kThreads) {
         const float a = acc[p];

@@ -40,6 +40,7 @@
 #include "pack.cuh"
 #include "apply.cuh"
 #include "quant_wide.cuh"
+#include "bf16_storage.cuh"
 #include "misc.cuh"
 #include "index_codec.cuh"
 #include "dense.cuh"
@@ -130,10 +131,12 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // general-width quantiser (quant_bits 1, 3, 4): its per-unit bin partials and per-tensor tables follow
 // the arrays of the 2-bit path in the workspace
 // (also the 2-bit quantiser at k > 256, which the fused kernels are not laid out for)
+// (and everything under bfloat16 storage)
+inline bool half_store(const sl_ctx* c) { return c->cfg.bf16_storage != 0; }
 inline bool wide_quant(const sl_ctx* c) {
-    return c->cfg.quant_bits != 32 && (c->cfg.quant_bits != 2 || c->cfg.k > kFastMaxK);
+    return c->cfg.quant_bits != 32 && (c->cfg.quant_bits != 2 || c->cfg.k > kFastMaxK || half_store(c));
 }
-inline bool fast_2bit(const sl_ctx* c) { return c->cfg.quant_bits == 2 && c->cfg.k <= kFastMaxK; }
+inline bool fast_2bit(const sl_ctx* c) { return c->cfg.quant_bits == 2 && c->cfg.k <= kFastMaxK && !half_store(c); }
 size_t wide_bytes_for(const sl_ctx* c, int workers) {
     if (!wide_quant(c)) return 0;
     const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->qbits;
@@ -278,6 +281,27 @@ sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const W
     const Workspace ws = carve(c, workers);
     const long long G = c->n_chunks;
     const int k = c->cfg.k, kp = c->kp;
+    if (half_store(c)) {  // bfloat16 arrays: the warp-per-unit kernel with plain loads
+        if (consume || delta) return SL_ERR_UNSUPPORTED;
+        const long long units = G * workers;
+        const long long want = (units + kHalfSelWarps - 1) / kHalfSelWarps;
+        const unsigned grid = (unsigned)(want < c->n_sms ? (want < 1 ? 1 : want) : c->n_sms);
+        const bf16_bits* ts = reinterpret_cast<const bf16_bits*>(theta_sync);
+#define SL_LAUNCH_HALF(EFV)                                                                                        \
+    do {                                                                                                           \
+        if (k > kSelNarrowMaxK)                                                                                    \
+            ef_select_bf16_kernel<EFV, true><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                  \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
+        else                                                                                                       \
+            ef_select_bf16_kernel<EFV, false><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                 \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
+    } while (0)
+        if (ef) SL_LAUNCH_HALF(true);
+        else SL_LAUNCH_HALF(false);
+#undef SL_LAUNCH_HALF
+        SL_CUDA(cudaGetLastError());
+        return SL_OK;
+    }
     // tile copies through tensor maps when the table allows it and every buffer got its maps
     TmaArgs ta;
     memset(&ta, 0, sizeof(ta));
@@ -379,7 +403,9 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     do {                                                                                                            \
         chunk_bins_q_kernel<BITSV><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.pbin, wq.pcnt);    \
         tensor_table_q_kernel<BITSV><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, wq.pbin, wq.pcnt, wq.tq, ptrs); \
-        if (ef)                                                                                                     \
+        if (ef && half_store(c))                                                                                    \
+            pack_q_kernel<BITSV, true, true><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
+        else if (ef)                                                                                                \
             pack_q_kernel<BITSV, true><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
         else                                                                                                        \
             pack_q_kernel<BITSV, false><<<pbq, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, wq.tq, c->rec_base, ptrs); \
@@ -427,14 +453,18 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const float scale = (float)(-(double)c->cfg.outer_lr / D);
     if (wide_quant(c) && fuse == 0) {  // payloads of 1, 3 or 4 bits per value
         const unsigned grid = (unsigned)c->n_chunks;
-        if (c->qbits == 1)
-            apply_q_kernel<1><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
-        else if (c->qbits == 2)
-            apply_q_kernel<2><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
-        else if (c->qbits == 3)
-            apply_q_kernel<3><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
-        else
-            apply_q_kernel<4><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync);
+#define SL_APPLY_Q(BITSV)                                                                                          \
+    do {                                                                                                           \
+        if (half_store(c))                                                                                         \
+            apply_q_kernel<BITSV, true><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync); \
+        else                                                                                                       \
+            apply_q_kernel<BITSV><<<grid, kThreads, 0, st>>>(c->d_chunks, R, c->cfg.k, scale, pl, c->rec_base, theta_sync); \
+    } while (0)
+        if (c->qbits == 1) SL_APPLY_Q(1);
+        else if (c->qbits == 2) SL_APPLY_Q(2);
+        else if (c->qbits == 3) SL_APPLY_Q(3);
+        else SL_APPLY_Q(4);
+#undef SL_APPLY_Q
         prof_mark(c, 8, st);
         if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
         SL_CUDA(cudaGetLastError());
@@ -523,6 +553,8 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (cfg->quant_bits != 32 && (cfg->quant_bits < 1 || cfg->quant_bits > 4)) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kMaxK || cfg->R > kMaxR) return SL_ERR_UNSUPPORTED;
     if (cfg->k > kFastMaxK && cfg->quant_bits == 32) return SL_ERR_UNSUPPORTED;  // the unquantised kernels stop at 256
+    if (cfg->bf16_storage != 0 && cfg->bf16_storage != 1) return SL_ERR_INVALID_ARG;
+    if (cfg->bf16_storage && cfg->quant_bits == 32) return SL_ERR_UNSUPPORTED;
 
     {   // element ranges: no overflow, no two tensors sharing an element (kernels of different chunks would race)
         std::vector<std::pair<long long, long long>> span((size_t)n_tensors);
@@ -661,6 +693,12 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
                                  (int)sizeof(SelSmem))
     SL_SELECT_ATTR_D(true, false); SL_SELECT_ATTR_D(false, false); SL_SELECT_ATTR_D(true, true); SL_SELECT_ATTR_D(false, true);
 #undef SL_SELECT_ATTR_D
+#define SL_HALF_ATTR(EFV, WIDEV)                                                                                     \
+    if (e == cudaSuccess)                                                                                            \
+        e = cudaFuncSetAttribute(ef_select_bf16_kernel<EFV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                 (int)sizeof(HalfSelSmem))
+    SL_HALF_ATTR(true, false); SL_HALF_ATTR(false, false); SL_HALF_ATTR(true, true); SL_HALF_ATTR(false, true);
+#undef SL_HALF_ATTR
     per_sm = 1;
     {   // the apply kernel's shared memory depends on k alone: sized once
         const int asz = (int)apply_smem_bytes(cfg->k < kFastMaxK ? cfg->k : kFastMaxK);
@@ -763,7 +801,49 @@ sl_status sl_set_workspace(sl_ctx* c, void* dev_ptr, size_t bytes) {
     return SL_OK;
 }
 
+namespace {
+sl_status do_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
+                      void* stream);
+sl_status do_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream);
+sl_status do_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+                        uint8_t* const* payloads, void* stream);
+}  // namespace
+
+// The fp32 entry points refuse a context made for bfloat16 storage and the other way round: the element
+// type of the arrays is fixed when the context is created.
 sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
+                      void* stream) {
+    if (c && half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_compress(c, theta_sync, theta_local, e, payload, stream);
+}
+sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
+    if (c && half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_aggregate_apply(c, payloads, theta_sync, stream);
+}
+sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+                        uint8_t* const* payloads, void* stream) {
+    if (c && half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_outer_step(c, theta_sync, theta_local, e, payloads, stream);
+}
+sl_status sl_compress_bf16(sl_ctx* c, const uint16_t* theta_sync, const uint16_t* theta_local, uint16_t* e,
+                           uint8_t* payload, void* stream) {
+    if (c && !half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_compress(c, reinterpret_cast<const float*>(theta_sync), reinterpret_cast<const float*>(theta_local),
+                       reinterpret_cast<float*>(e), payload, stream);
+}
+sl_status sl_aggregate_apply_bf16(sl_ctx* c, const uint8_t* const* payloads, uint16_t* theta_sync, void* stream) {
+    if (c && !half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_aggregate_apply(c, payloads, reinterpret_cast<float*>(theta_sync), stream);
+}
+sl_status sl_outer_step_bf16(sl_ctx* c, uint16_t* theta_sync, const uint16_t* const* theta_local, uint16_t* const* e,
+                             uint8_t* const* payloads, void* stream) {
+    if (c && !half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_outer_step(c, reinterpret_cast<float*>(theta_sync), reinterpret_cast<const float* const*>(theta_local),
+                         reinterpret_cast<float* const*>(e), payloads, stream);
+}
+
+namespace {
+sl_status do_compress(sl_ctx* c, const float* theta_sync, const float* theta_local, float* e, uint8_t* payload,
                       void* stream) {
     if (!c || !theta_sync || !theta_local || !payload) return SL_ERR_INVALID_ARG;
     if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
@@ -780,7 +860,7 @@ sl_status sl_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
     return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream), false);
 }
 
-sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
+sl_status do_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
     if (!c || !payloads || !theta_sync) return SL_ERR_INVALID_ARG;
     if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
@@ -797,7 +877,6 @@ sl_status sl_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* t
     return launch_apply(c, pl, present, theta_sync, static_cast<cudaStream_t>(stream));
 }
 
-namespace {
 
 // The outer step without the quantiser (quant_bits = 32, the full-precision column of the paper's
 // quantisation ablation): Top-k sends the selected values exactly, so nothing stays behind at the
@@ -831,9 +910,7 @@ sl_status outer_step_unquantised(sl_ctx* c, float* theta_sync, const float* cons
     return s;
 }
 
-}  // namespace
-
-sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
+sl_status do_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
                         uint8_t* const* payloads, void* stream) {
     if (c && c->cfg.quant_bits == 32) {
         if (!theta_sync || !theta_local || (c->cfg.ef_enabled && !e)) return SL_ERR_INVALID_ARG;
@@ -880,12 +957,13 @@ sl_status sl_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
     if (s != SL_OK) return s;
     return launch_apply(c, pl, R, theta_sync, st, fuse, &ptrs);
 }
+}  // namespace
 
 sl_status sl_outer_step_host(sl_ctx* c, float* theta_sync, const float* const* theta_local_host, float* dev_stage,
                              size_t stage_elems, float* const* e, uint8_t* const* payloads, float* theta_sync_host,
                              void* stream) {
     if (!c || !theta_sync || !theta_local_host || !dev_stage || !payloads) return SL_ERR_INVALID_ARG;
-    if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
+    if (c->cfg.quant_bits == 32 || half_store(c)) return SL_ERR_UNSUPPORTED;  // (no payload format / fp32 arrays only)
     if (c->cfg.ef_enabled && !e) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(dev_stage)) return SL_ERR_ALIGNMENT;
     const int R = c->cfg.R;
@@ -980,6 +1058,7 @@ const char* sl_profile_name(int32_t slot) {
 sl_status sl_diloco_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* momentum,
                          float beta_outer, void* stream) {
     if (!c || !theta_sync || !theta_local || !momentum) return SL_ERR_INVALID_ARG;
+    if (half_store(c)) return SL_ERR_UNSUPPORTED;  // the baselines work on fp32 arrays
     if (!(beta_outer >= 0.0f && beta_outer <= 1.0f)) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync) || misaligned(momentum)) return SL_ERR_ALIGNMENT;
     LocalPtrs lp;
@@ -1003,6 +1082,7 @@ namespace {
 sl_status variant_args(sl_ctx* c, const float* theta_sync, const float* const* theta_local, float* const* e,
                        float* const* m_r, float mu, WorkerPtrs& ptrs) {
     if (!c || !theta_sync || !theta_local) return SL_ERR_INVALID_ARG;
+    if (half_store(c)) return SL_ERR_UNSUPPORTED;  // the baselines work on fp32 arrays
     if (!(mu >= 0.0f && mu <= 1.0f)) return SL_ERR_INVALID_ARG;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
     memset(&ptrs, 0, sizeof(ptrs));
