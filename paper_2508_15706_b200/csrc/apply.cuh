@@ -7,10 +7,13 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------------
-// Decode + average + outer update (Eq. 2 lines 3-4).  Persistent CTAs of four warps, eight per SM;
+// Decode + average + outer update (Eq. 2 lines 3-4).  Persistent CTAs of four warps, up to six per SM;
 // a CTA takes whole chunks (b, b + grid, ...) and owns a 4096-float sum tile in shared memory.  For a
 // chunk it
-//   1. starts the loads of the chunk's theta (8 x 128 bits per thread, in registers until step 4),
+//   1. takes the chunk's theta (8 x 128 bits per thread, in registers until step 4) from the CTA's staging
+//      block, where asynchronous copies issued one chunk earlier have put it, and starts the copies of
+//      the next chunk's theta: a thread copies exactly the vectors it will own, so it waits for its own
+//      copies only and no barrier is involved; the copies of chunk g + grid fly while chunk g is decoded,
 //   2. decodes the workers in batches of 16, warp w the workers 4 w .. 4 w + 3 of the batch: a lane holds
 //      the slot pairs (2 m, 2 m + 1), m = lane + 32 j, of a worker and turns them into (index, table value),
 //   3. adds them into the tile in ascending worker order: the warps take turns (a CTA barrier between
@@ -45,13 +48,22 @@ struct FuseArgs {
 
 constexpr int kApplyWarps = 4;
 constexpr int kApplyThreads = 32 * kApplyWarps;
-constexpr int kApplyCtasPerSm = 8;
+constexpr int kApplyCtasPerSm = 6;   // what the shared memory of a CTA (tile, records, staging block) lets an SM hold
 constexpr int kApplyBatch = 16;                  // workers decoded between two rounds of ordered additions
 constexpr int kApplyPerWarp = kApplyBatch / kApplyWarps;
 constexpr int kApplyTile = kChunk + kApplyThreads;  // the sum tile + one dump slot per thread for entries that do not count
 
 __host__ __device__ constexpr size_t apply_smem_bytes(int k) {
-    return (size_t)kApplyTile * sizeof(float) + (size_t)kApplyBatch * (record_stride(k) + 32);
+    return (size_t)kApplyTile * sizeof(float) + (size_t)kApplyBatch * (record_stride(k) + 32) + (size_t)kChunk * sizeof(float);
+}
+
+// 16-byte asynchronous copy global -> shared (L2 only), and the wait for all of this thread's copies
+__device__ __forceinline__ void async_copy16(void* smem_dst, const void* gmem_src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void async_copy_wait_all() {
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
 }
 
 // PPL = slot pairs per lane: ceil(k / 64) rounded up to 1, 2 or 4
@@ -66,6 +78,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     uint8_t* recs = dyn + (size_t)kApplyTile * sizeof(float);
     // per worker of the batch: mean, 3 sigma, 0, present | the four table entries
     float4* tabs = reinterpret_cast<float4*>(recs + (size_t)kApplyBatch * stride);
+    float4* stage = tabs + 2 * kApplyBatch;  // theta of the chunk to come: vector i of thread t at [128 i + t]
     constexpr int WB = kApplyPerWarp;
     constexpr bool PACK = FUSE == 1 || FUSE == 2;  // quantise, write records and the error correction
     constexpr bool RAW = FUSE >= 3;                // staged values travel unquantised
@@ -76,19 +89,36 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     for (int i = tid; i < kApplyTile / 4; i += kApplyThreads) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
 
+    // thread t owns in-chunk indices 512 i + 4 t + j: block row 8 i + t / 16, column 4 (t % 16)
+    auto prefetch_theta = [&](const ChunkDesc& d) {
+        const int prs = d.row_stride ? d.row_stride : kTile;
+        const float* src = theta_sync + d.base + (long long)(tid >> 4) * prs + 4 * (tid & 15);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) async_copy16(&stage[128 * i + tid], src + (long long)i * 8 * prs);
+    };
+    ChunkDesc cd_next;
+    if ((long long)blockIdx.x < n_chunks) {
+        cd_next = chunks[blockIdx.x];
+        if (cd_next.len == kChunk) prefetch_theta(cd_next);
+    }
+
     for (long long g = blockIdx.x; g < n_chunks; g += gridDim.x) {
-        const ChunkDesc cd = chunks[g];
+        const ChunkDesc cd = cd_next;
         const int keff = min(k, cd.len);
         const bool full = cd.len == kChunk;
         const int rs = cd.row_stride ? cd.row_stride : kTile;
         float* __restrict__ th = theta_sync + cd.base;
-        // thread t owns in-chunk indices 512 i + 4 t + j: block row 8 i + t / 16, column 4 (t % 16)
         float* __restrict__ th_vec = th + (long long)(tid >> 4) * rs + 4 * (tid & 15);
         const long long vec_step = 8ll * rs;
         float4 a[8];
+        async_copy_wait_all();  // (this thread's copies; nothing is outstanding after a short chunk)
         if (full) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(th_vec + i * vec_step);
+            for (int i = 0; i < 8; ++i) a[i] = stage[128 * i + tid];
+        }
+        if (g + gridDim.x < n_chunks) {  // the block is free again (this thread's part of it): the next chunk's theta
+            cd_next = chunks[g + gridDim.x];
+            if (cd_next.len == kChunk) prefetch_theta(cd_next);
         }
         // which of this lane's slots exist in this chunk (the same for every worker)
         bool in0[PPL], in1[PPL];

@@ -36,7 +36,7 @@ __device__ __forceinline__ void bf16_store4(bf16_bits* p, const float4& x) {
     *reinterpret_cast<uint2*>(p) = w;
 }
 
-constexpr int kHalfSelWarps = 8;
+constexpr int kHalfSelWarps = 12;  // what shared memory (16 KB of u per warp) and the register file allow
 constexpr int kHalfSelThreads = 32 * kHalfSelWarps;
 struct HalfSelSmem {
     __align__(16) float u[kHalfSelWarps][kChunk];
@@ -46,7 +46,7 @@ struct HalfSelSmem {
 
 // One warp per (chunk, worker) unit, units taken chunk-major so that the workers of a chunk follow one
 // another (theta's block is re-read from L2).  The WorkerPtrs / theta pointers address bfloat16 arrays.
-template <bool EF, bool WIDE>
+template <bool EF, int WIDE>
 __global__ void __launch_bounds__(kHalfSelThreads, 1)
 ef_select_bf16_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                       const bf16_bits* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
@@ -66,6 +66,42 @@ ef_select_bf16_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, 
         bf16_bits* __restrict__ er = EF ? reinterpret_cast<bf16_bits*>(ptrs.e[r]) + cd.base : nullptr;
         *reinterpret_cast<uint4*>(&bitmap[4 * lane]) = make_uint4(0u, 0u, 0u, 0u);
         float u[128];
+        if (cd.len == kChunk) {
+            // a full chunk: the loads of 8 vectors per array are issued before any of them is used (the stores
+            // into e would otherwise order every later load of e behind them)
+#pragma unroll
+            for (int i0 = 0; i0 < 32; i0 += 8) {
+                uint2 wa[8], wl[8], we[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const long long off = chunk_elem_offset(cd.row_stride, 128 * (i0 + j) + 4 * lane);
+                    wa[j] = __ldg(reinterpret_cast<const uint2*>(tsp + off));
+                    wl[j] = __ldcs(reinterpret_cast<const uint2*>(tlp + off));
+                    if (EF) we[j] = __ldcs(reinterpret_cast<const uint2*>(er + off));
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int i = i0 + j, p0 = 128 * i + 4 * lane;
+                    float4 x;
+                    x.x = __fsub_rn(bf16_widen(wa[j].x & 0xFFFFu), bf16_widen(wl[j].x & 0xFFFFu));
+                    x.y = __fsub_rn(bf16_widen(wa[j].x >> 16), bf16_widen(wl[j].x >> 16));
+                    x.z = __fsub_rn(bf16_widen(wa[j].y & 0xFFFFu), bf16_widen(wl[j].y & 0xFFFFu));
+                    x.w = __fsub_rn(bf16_widen(wa[j].y >> 16), bf16_widen(wl[j].y >> 16));
+                    if (EF) {
+                        x.x = __fmaf_rn(beta, bf16_widen(we[j].x & 0xFFFFu), x.x);
+                        x.y = __fmaf_rn(beta, bf16_widen(we[j].x >> 16), x.y);
+                        x.z = __fmaf_rn(beta, bf16_widen(we[j].y & 0xFFFFu), x.z);
+                        x.w = __fmaf_rn(beta, bf16_widen(we[j].y >> 16), x.w);
+                        bf16_store4(er + chunk_elem_offset(cd.row_stride, p0), x);
+                    }
+                    *reinterpret_cast<float4*>(&scratch[p0]) = x;
+                    u[4 * i + 0] = x.x;
+                    u[4 * i + 1] = x.y;
+                    u[4 * i + 2] = x.z;
+                    u[4 * i + 3] = x.w;
+                }
+            }
+        } else
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             const int p0 = 128 * i + 4 * lane;

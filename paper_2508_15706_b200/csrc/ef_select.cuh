@@ -165,7 +165,9 @@ __device__ __forceinline__ unsigned lane_pos(int lane, int q) { return 128u * (q
 // Writes (index, value) of the entries marked in the warp's 4096-bit map to their slots, in ascending
 // index order, reading the values back through `src`.  Word w of the map covers indices 32 w ..; lane l
 // owns words 4 l .. 4 l + 3.
-template <bool GLOBAL>
+// BATCH > 1: the values of BATCH entries are fetched before any of them is stored (with many entries per lane
+// the fetches, L2 reads when `src` is global, would otherwise wait for one another).
+template <bool GLOBAL, int BATCH = 1>
 __device__ __forceinline__ void emit_from_map(const unsigned* bitmap, const USource& src, int keff,
                                               uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
     const int lane = threadIdx.x & 31;
@@ -183,14 +185,27 @@ __device__ __forceinline__ void emit_from_map(const unsigned* bitmap, const USou
     for (int q = 0; q < 4; ++q) {
         unsigned mm = words[q];
         while (mm) {
-            const unsigned b = __ffs(mm) - 1;
-            mm &= mm - 1;
-            const unsigned p = 128u * lane + 32u * q + b;
-            if (slot < (unsigned)keff) {
-                out_idx[slot] = (uint16_t)p;
-                out_val[slot] = __uint_as_float(usrc_load<GLOBAL>(src, p));
+            unsigned p[BATCH], v[BATCH];
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                p[t] = 0xFFFFu;
+                if (mm) {
+                    p[t] = 128u * lane + 32u * q + (__ffs(mm) - 1);
+                    mm &= mm - 1;
+                }
             }
-            ++slot;
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) v[t] = p[t] != 0xFFFFu ? usrc_load<GLOBAL>(src, p[t]) : 0u;
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                if (p[t] != 0xFFFFu) {
+                    if (slot < (unsigned)keff) {
+                        out_idx[slot] = (uint16_t)p[t];
+                        out_val[slot] = __uint_as_float(v[t]);
+                    }
+                    ++slot;
+                }
+            }
         }
     }
 }
@@ -257,6 +272,134 @@ __device__ __noinline__ void select_slow(USource src, int len, int keff, unsigne
     }
     __syncwarp();
     emit_from_map<GLOBAL>(bitmap, src, keff, out_idx, out_val);
+}
+
+// Selection for large keff (beyond 256 of 4096: the dense settings of the paper's sweeps), on the warp's
+// registers.  A bitwise search narrows a key interval [lo, hi) around the cut until it holds at most
+// kCandCap elements (about ten rounds over the 128 registers instead of the 31 + 12 of the exact
+// fallback); the elements inside the interval are listed and a search over that short list finds the
+// cut (key, and index among equal keys); everything at or above hi was marked in the map straight from the
+// registers, the winners of the list are added, and the entries are written from the map.  Falls back to
+// select_slow when the interval cannot be narrowed (a run of more than kCandCap equal keys at the cut).
+// Warp-collective.
+template <bool GLOBAL>
+__device__ __forceinline__ void select_dense(const float (&u)[128], USource src, int len, int keff, unsigned* bitmap,
+                                          uint16_t* cand, uint16_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    const int lane = threadIdx.x & 31;
+    unsigned mx = 0;
+#pragma unroll
+    for (int q = 0; q < 128; ++q) mx = max(mx, __float_as_uint(u[q]) & 0x7FFFFFFFu);
+    const unsigned M = __reduce_max_sync(kFull, mx);
+    unsigned lo = 0, hi = M + 1u, c_lo = (unsigned)kChunk, c_hi = 0;  // count(>= lo) = c_lo >= keff > c_hi = count(>= hi)
+    // first guesses: one and two binades below the largest key
+    unsigned x = M > (1u << 23) ? M - (1u << 23) : (M >> 1);
+    while (c_lo - c_hi > (unsigned)kCandCap && hi - lo > 1) {
+        if (!(x > lo && x < hi)) x = lo + ((hi - lo) >> 1);
+        unsigned c = 0;
+#pragma unroll
+        for (int q = 0; q < 128; ++q) c += (__float_as_uint(u[q]) & 0x7FFFFFFFu) >= x ? 1u : 0u;
+        c = __reduce_add_sync(kFull, c);
+        if (c >= (unsigned)keff) {
+            lo = x;
+            c_lo = c;
+            x = hi;  // (out of range: the next guess is the midpoint)
+        } else {
+            hi = x;
+            c_hi = c;
+            x = x > (1u << 23) ? x - (1u << 23) : 0u;  // still too few: try a binade lower
+        }
+    }
+    if (c_lo - c_hi > (unsigned)kCandCap) {  // more than a list's worth of equal keys at the cut
+        select_slow<GLOBAL>(src, len, keff, bitmap, out_idx, out_val);
+        return;
+    }
+    // elements at or above hi are selected: marked in the map straight from the registers (four consecutive
+    // indices of a lane share a map word with seven other lanes); the ones inside the interval are listed.
+    // (The registers are not needed after this: what follows works on the list and on the map.)
+    unsigned hm[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        unsigned nib = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const unsigned key = __float_as_uint(u[4 * i + j]) & 0x7FFFFFFFu;
+            nib |= key >= hi ? (1u << j) : 0u;
+            hm[i >> 3] |= (key >= lo && key < hi) ? (1u << ((4 * i + j) & 31)) : 0u;
+        }
+        if (nib) atomicOr(&bitmap[4 * i + (lane >> 3)], nib << (4 * (lane & 7)));
+    }
+    // the list of the elements inside the interval
+    const unsigned mine = __popc(hm[0]) + __popc(hm[1]) + __popc(hm[2]) + __popc(hm[3]);
+    unsigned inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned o = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += o;
+    }
+    const unsigned n_b = __shfl_sync(kFull, inc, 31);  // = c_lo - c_hi
+    {
+        unsigned at = inc - mine;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            unsigned mm = hm[w];
+            while (mm) {
+                const unsigned b = __ffs(mm) - 1;
+                mm &= mm - 1;
+                cand[at++] = (uint16_t)lane_pos(lane, 32 * w + (int)b);
+            }
+        }
+    }
+    __syncwarp();
+    // the `need` largest of the list, ties to the lower index
+    constexpr int CPL = kCandCap / 32;
+    const unsigned need = (unsigned)keff - c_hi;  // 1 .. n_b
+    unsigned cp[CPL], ck[CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        const unsigned t = lane + 32u * j;
+        cp[j] = t < n_b ? cand[t] : 0u;
+        ck[j] = t < n_b ? (usrc_load<GLOBAL>(src, cp[j]) & 0x7FFFFFFFu) : 0u;
+    }
+    // (an empty place has key 0; when lo = 0 it would count, so empty places are excluded by position)
+    unsigned l2 = lo, h2 = hi, cl2 = n_b, ch2 = 0;  // count(>= l2) = cl2 >= need > ch2 = count(>= h2), within the list
+    while (cl2 != need && h2 - l2 > 1) {
+        const unsigned xm = l2 + ((h2 - l2) >> 1);
+        unsigned c = 0;
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) c += (lane + 32u * j < n_b && ck[j] >= xm) ? 1u : 0u;
+        c = __reduce_add_sync(kFull, c);
+        if (c >= need) {
+            l2 = xm;
+            cl2 = c;
+        } else {
+            h2 = xm;
+            ch2 = c;
+        }
+    }
+    unsigned P = 4095u;
+    const bool clean = cl2 == need;
+    if (!clean) {
+        const unsigned want = need - ch2;
+        int plo = -1, phi = 4095;
+        while (phi - plo > 1) {
+            const int mid = plo + ((phi - plo) >> 1);
+            unsigned c = 0;
+#pragma unroll
+            for (int j = 0; j < CPL; ++j) c += (lane + 32u * j < n_b && ck[j] == l2 && (int)cp[j] <= mid) ? 1u : 0u;
+            c = __reduce_add_sync(kFull, c);
+            if (c >= want) phi = mid;
+            else plo = mid;
+        }
+        P = (unsigned)phi;
+    }
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        const bool in = lane + 32u * j < n_b;
+        const bool sel = in && (clean ? ck[j] >= l2 : (ck[j] > l2 || (ck[j] == l2 && cp[j] <= P)));
+        if (sel) atomicOr(&bitmap[cp[j] >> 5], 1u << (cp[j] & 31));
+    }
+    __syncwarp();
+    emit_from_map<GLOBAL, 8>(bitmap, src, keff, out_idx, out_val);
 }
 
 // Steps D-F for a candidate list of n_c <= 32 CPL entries.  Warp-collective.
@@ -405,7 +548,9 @@ __device__ __forceinline__ void group_threshold(const float (&u)[128], int keff,
 }
 
 // Steps A-F on the warp's registers.  `u` = this lane's 128 values (0 at indices >= len).
-template <bool GLOBAL, bool WIDE>
+// WIDE: 0 = k <= 128, 1 = k <= 256, 2 = beyond (kernels of their own, so that the common case carries neither the
+// code nor the registers of the others)
+template <bool GLOBAL, int WIDE>
 __device__ __forceinline__ void select_unit(const float (&u)[128], const USource& src, int len, int keff,
                                             unsigned* bitmap, uint16_t* cand, uint16_t* __restrict__ out_idx,
                                             float* __restrict__ out_val) {
@@ -413,8 +558,8 @@ __device__ __forceinline__ void select_unit(const float (&u)[128], const USource
     // groups of 16 values up to k = 128 (about 1.15 k candidates); beyond that a threshold taken from 256
     // group maxima lets too many elements through, and groups of 4 take over (WIDE: a kernel of its own,
     // so that the common case carries neither the code nor the registers of the other)
-    if (WIDE && keff > kFastMaxK) {  // beyond 256 of 4096 a threshold over group maxima no longer thins the field
-        select_slow<GLOBAL>(src, len, keff, bitmap, out_idx, out_val);
+    if (WIDE == 2 && keff > kFastMaxK) {  // beyond 256 of 4096 a threshold over group maxima no longer thins the field
+        select_dense<GLOBAL>(u, src, len, keff, bitmap, cand, out_idx, out_val);
         return;
     }
     unsigned T, probe;
@@ -460,7 +605,7 @@ __device__ __forceinline__ void select_unit(const float (&u)[128], const USource
 
 // DELTA: the "theta_r" buffers hold the vector to compress itself (a local Nesterov direction, a
 // momentum: the Top-k baselines of Alg. 2 and 4) instead of parameters to subtract from theta.
-template <bool EF, bool PENDING, bool WIDE, bool DELTA = false>
+template <bool EF, bool PENDING, int WIDE, bool DELTA = false>
 __global__ void __launch_bounds__(kSelThreads, 1)
 ef_select_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                  const float* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws, TmaArgs tma, int use_tma) {

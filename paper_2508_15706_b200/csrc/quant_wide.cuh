@@ -57,8 +57,7 @@ chunk_bins_q_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, in
         sb[b] = 0.0;
         nb[b] = 0;
     }
-    for (int s = 0; s < keff; ++s) {
-        const float x = v[s];
+    for_each_staged_own(v, keff, [&](float x) {
         const int c = quant_code_q<BITS>(x, st.mu, st.sigma);
 #pragma unroll
         for (int b = 0; b < NB; ++b)  // only the value's own bin (adding +0 elsewhere could flip a -0 sum)
@@ -66,7 +65,7 @@ chunk_bins_q_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, in
                 sb[b] += (double)x;
                 ++nb[b];
             }
-    }
+    });
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         pbin[i * NB + b] = sb[b];
@@ -91,24 +90,41 @@ tensor_table_q_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, 
     const long long first = (long long)r * n_chunks + ti.first_chunk;
     const long long n_groups = (ti.n_chunks + kSumGroup - 1) / kSumGroup;
     float* hdr = reinterpret_cast<float*>(ptrs.payload[r] + (long long)header_bytes_q(BITS) * t);
-    for (int b = 0; b < NB; ++b) {
-        double acc = 0.0;
-        unsigned long long cn = 0;
-        for (long long g0 = 0; g0 < n_groups; g0 += 32) {
-            double gs = 0.0;
-            const long long c0 = (g0 + lane) * kSumGroup;
-            const int cnt = (int)max(0ll, min((long long)kSumGroup, ti.n_chunks - c0));
-            for (int c = 0; c < cnt; ++c) {
-                gs += pbin[(first + c0 + c) * NB + b];
-                cn += pcnt[(first + c0 + c) * NB + b];
-            }
-            const int ng = (int)min(32ll, n_groups - g0);
-            for (int l = 0; l < ng; ++l) acc += __shfl_sync(kFull, gs, l);
-        }
+    double acc[NB];              // all bins in one walk over the chunk partials (each bin keeps its own order)
+    unsigned long long cn[NB];
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) cn += __shfl_xor_sync(kFull, cn, d);
+    for (int b = 0; b < NB; ++b) {
+        acc[b] = 0.0;
+        cn[b] = 0;
+    }
+    for (long long g0 = 0; g0 < n_groups; g0 += 32) {
+        double gs[NB];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) gs[b] = 0.0;
+        const long long c0 = (g0 + lane) * kSumGroup;
+        const int cnt = (int)max(0ll, min((long long)kSumGroup, ti.n_chunks - c0));
+        for (int c = 0; c < cnt; ++c) {
+            const double* pb = pbin + (first + c0 + c) * NB;
+            const unsigned* pc = pcnt + (first + c0 + c) * NB;
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                gs[b] += pb[b];
+                cn[b] += pc[b];
+            }
+        }
+        const int ng = (int)min(32ll, n_groups - g0);
+        for (int l = 0; l < ng; ++l) {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) acc[b] += __shfl_sync(kFull, gs[b], l);
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        unsigned long long n = cn[b];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) n += __shfl_xor_sync(kFull, n, d);
         if (lane == 0) {
-            const float v = cn ? (float)(acc / (double)cn) : 0.0f;
+            const float v = n ? (float)(acc[b] / (double)n) : 0.0f;
             tq[(long long)r * n_tensors + t].lut[b] = v;
             hdr[b] = v;
         }

@@ -289,11 +289,14 @@ sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const W
         const bf16_bits* ts = reinterpret_cast<const bf16_bits*>(theta_sync);
 #define SL_LAUNCH_HALF(EFV)                                                                                        \
     do {                                                                                                           \
-        if (k > kSelNarrowMaxK)                                                                                    \
-            ef_select_bf16_kernel<EFV, true><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                  \
+        if (k > kFastMaxK)                                                                                         \
+            ef_select_bf16_kernel<EFV, 2><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                     \
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
+        else if (k > kSelNarrowMaxK)                                                                               \
+            ef_select_bf16_kernel<EFV, 1><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                     \
                 c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
         else                                                                                                       \
-            ef_select_bf16_kernel<EFV, false><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                 \
+            ef_select_bf16_kernel<EFV, 0><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                     \
                 c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
     } while (0)
         if (ef) SL_LAUNCH_HALF(true);
@@ -337,13 +340,21 @@ sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const W
 #define SL_LAUNCH_SELECT(EFV, PENDV, DELTAV)                                                                         \
     do {                                                                                                             \
         if (k > kSelNarrowMaxK)                                                                                      \
-            ef_select_kernel<EFV, PENDV, true, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                  \
+            ef_select_kernel<EFV, PENDV, 1, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                     \
                 c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
         else                                                                                                         \
-            ef_select_kernel<EFV, PENDV, false, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                 \
+            ef_select_kernel<EFV, PENDV, 0, DELTAV><<<grid, kSelThreads, sizeof(SelSmem), st>>>(                     \
                 c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);                          \
     } while (0)
-    if (delta) {
+    if (k > kFastMaxK) {  // the dense settings: no waiting lists, no baselines (refused before this point)
+        if (consume || delta) return SL_ERR_UNSUPPORTED;
+        if (ef)
+            ef_select_kernel<true, false, 2><<<grid, kSelThreads, sizeof(SelSmem), st>>>(
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
+        else
+            ef_select_kernel<false, false, 2><<<grid, kSelThreads, sizeof(SelSmem), st>>>(
+                c->d_chunks, G, workers, k, kp, c->cfg.beta, theta_sync, ptrs, ws, ta, tm);
+    } else if (delta) {
         if (ef) SL_LAUNCH_SELECT(true, false, true);
         else SL_LAUNCH_SELECT(false, false, true);
     } else if (!ef) {
@@ -488,7 +499,9 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
         if (fuse_ptrs) wp = *fuse_ptrs;
     }
     // persistent CTAs: as many as are resident at once
-    const long long resident = (long long)c->n_sms * kApplyCtasPerSm;
+    // (a CTA's shared memory grows with k: 227 KB per SM, 1 KB reserved per CTA)
+    const long long fit = (227ll * 1024) / ((long long)smem + 1024);
+    const long long resident = (long long)c->n_sms * (fit < kApplyCtasPerSm ? (fit < 1 ? 1 : fit) : kApplyCtasPerSm);
     const unsigned grid = (unsigned)(c->n_chunks < resident ? c->n_chunks : resident);
 #define SL_APPLY(PPLV)                                                                                          \
     do {                                                                                                        \
@@ -684,20 +697,22 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     if (e == cudaSuccess)                                                                                            \
         e = cudaFuncSetAttribute(ef_select_kernel<EFV, PENDV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
                                  (int)sizeof(SelSmem))
-    SL_SELECT_ATTR(true, false, false); SL_SELECT_ATTR(true, true, false); SL_SELECT_ATTR(false, false, false);
-    SL_SELECT_ATTR(true, false, true); SL_SELECT_ATTR(true, true, true); SL_SELECT_ATTR(false, false, true);
+    SL_SELECT_ATTR(true, false, 0); SL_SELECT_ATTR(true, true, 0); SL_SELECT_ATTR(false, false, 0);
+    SL_SELECT_ATTR(true, false, 1); SL_SELECT_ATTR(true, true, 1); SL_SELECT_ATTR(false, false, 1);
+    SL_SELECT_ATTR(true, false, 2); SL_SELECT_ATTR(false, false, 2);
 #undef SL_SELECT_ATTR
 #define SL_SELECT_ATTR_D(EFV, WIDEV)                                                                                 \
     if (e == cudaSuccess)                                                                                            \
         e = cudaFuncSetAttribute(ef_select_kernel<EFV, false, WIDEV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  (int)sizeof(SelSmem))
-    SL_SELECT_ATTR_D(true, false); SL_SELECT_ATTR_D(false, false); SL_SELECT_ATTR_D(true, true); SL_SELECT_ATTR_D(false, true);
+    SL_SELECT_ATTR_D(true, 0); SL_SELECT_ATTR_D(false, 0); SL_SELECT_ATTR_D(true, 1); SL_SELECT_ATTR_D(false, 1);
 #undef SL_SELECT_ATTR_D
 #define SL_HALF_ATTR(EFV, WIDEV)                                                                                     \
     if (e == cudaSuccess)                                                                                            \
         e = cudaFuncSetAttribute(ef_select_bf16_kernel<EFV, WIDEV>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
                                  (int)sizeof(HalfSelSmem))
-    SL_HALF_ATTR(true, false); SL_HALF_ATTR(false, false); SL_HALF_ATTR(true, true); SL_HALF_ATTR(false, true);
+    SL_HALF_ATTR(true, 0); SL_HALF_ATTR(false, 0); SL_HALF_ATTR(true, 1); SL_HALF_ATTR(false, 1);
+    SL_HALF_ATTR(true, 2); SL_HALF_ATTR(false, 2);
 #undef SL_HALF_ATTR
     per_sm = 1;
     {   // the apply kernel's shared memory depends on k alone: sized once
@@ -1477,10 +1492,10 @@ sl_status sl_compress_tensor_static(const float* theta_sync, const float* theta_
     memset(&no_tma, 0, sizeof(no_tma));
     no_tma.status = su.status;
     if (k > kSelNarrowMaxK)
-        ef_select_kernel<true, false, true><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
+        ef_select_kernel<true, false, 1><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
                                                                                         ptrs, ws, no_tma, 0);
     else
-        ef_select_kernel<true, false, false><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
+        ef_select_kernel<true, false, 0><<<ef_grid, kSelThreads, sizeof(SelSmem), st>>>(d_chunks, G, 1, k, kp, beta, theta_sync,
                                                                                          ptrs, ws, no_tma, 0);
     const unsigned cb = blocks_for(G, 128);
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(d_chunks, G, 1, 1, k, kp, ws);

@@ -99,7 +99,7 @@ def test_ef_accumulate_freeze_and_beta_zero():
 def test_topk_matches_bruteforce(L, k):
     """(the densities of the paper's sweeps go up to 50 %, k = 2048 of 4096)"""
     rng = np.random.default_rng(L * 100 + k)
-    for trial in range(20 if L <= 100 else 6):
+    for trial in range(20 if L <= 100 else 3):
         u = rng.standard_normal(L).astype(np.float32)
         if trial % 3 == 1:  # heavy ties, both signs
             u = (rng.integers(-2, 3, L)).astype(np.float32)
