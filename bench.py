@@ -363,6 +363,24 @@ def run_ours(args) -> dict:
             "payload_bytes": sl.payload_bytes(), "coded_bytes": nbytes, "round_trip_identical": bool(torch.equal(back, payloads[0])),
             "index_bits_per_value": 8.0 * (nbytes - 16 * len(wl.tensors) - code_block * chunks) / slots,
             "encode_ms": c0.elapsed_time(c1) / 10, "decode_ms": c1.elapsed_time(c2) / 10}
+        # the update straight from R coded payloads (decoding fused into the update kernel) beside the
+        # update from R 12-bit payloads; every worker's slot is given the same coded payload here
+        many = [coded] * wl.R
+        sl.ef_flush()
+        sl.aggregate_apply_coded(many, theta, [nbytes] * wl.R)
+        sl.aggregate_apply(payloads, theta)
+        c3, c4, c5 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        c3.record(stream)
+        for _ in range(3):
+            sl.aggregate_apply_coded(many, theta, [nbytes] * wl.R)
+        c4.record(stream)
+        for _ in range(3):
+            sl.aggregate_apply(payloads, theta)
+        c5.record(stream)
+        torch.cuda.synchronize()
+        result["index_codec"]["aggregate_apply_coded_ms"] = c3.elapsed_time(c4) / 3
+        result["index_codec"]["aggregate_apply_ms"] = c4.elapsed_time(c5) / 3
+        result["index_codec"]["decode_all_workers_then_apply_ms"] = wl.R * result["index_codec"]["decode_ms"] + c4.elapsed_time(c5) / 3
     if rank == 0 and world == 1 and not args.no_e2e:
         del local, locals_r
         torch.cuda.empty_cache()

@@ -241,12 +241,25 @@ sl_status sl_lom_topk_step(sl_ctx* ctx, float* theta_sync, float* const* theta_l
  *                               wrong but well-formed-sized record, never an out-of-range access.
  *                               Such an input (also a directory that does not ascend) records
  *                               SL_ERR_BAD_PAYLOAD in the device status word (sl_device_status); run
- *                               sl_validate_payload on the result as well. */
+ *                               sl_validate_payload on the result as well.
+ *   sl_aggregate_apply_coded  : Eq. 2 lines 3-4 (decode, average, outer update) straight from R coded
+ *                               payloads, the decoding fused into the update kernel: what
+ *                               sl_decode_payload for every worker followed by sl_aggregate_apply does,
+ *                               bit for bit, without the 12-bit payloads in between.  `coded` = HOST
+ *                               array of R DEVICE pointers (NULL = absent worker), `coded_bytes` = HOST
+ *                               array of the R sizes as for sl_decode_payload (NULL or 0 = full
+ *                               capacity).  Reads stay inside the stated sizes; a damaged input gives
+ *                               a wrong update of in-range elements and SL_ERR_BAD_PAYLOAD in the
+ *                               device status word, so validate untrusted payloads first
+ *                               (sl_decode_payload + sl_validate_payload).  UNSUPPORTED when the
+ *                               per-CTA staging would not fit shared memory (R x k beyond about 64 x 256). */
 sl_status sl_coded_payload_capacity(const sl_ctx* ctx, size_t* bytes);
 sl_status sl_encode_payload(sl_ctx* ctx, const uint8_t* payload, uint8_t* coded, uint64_t* dev_coded_bytes,
                             void* cuda_stream);
 sl_status sl_decode_payload(sl_ctx* ctx, const uint8_t* coded, size_t coded_bytes, uint8_t* payload,
                             void* cuda_stream);
+sl_status sl_aggregate_apply_coded(sl_ctx* ctx, const uint8_t* const* coded, const size_t* coded_bytes,
+                                   float* theta_sync, void* cuda_stream);
 
 /* How the compression kernel moves the 64x64 blocks of theta, theta_r and e (no counterpart in the paper).
  * 1: one tensor-map (TMA) block copy per block, issued by a producer thread, completion on

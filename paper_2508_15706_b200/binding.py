@@ -20,7 +20,7 @@ EXPORTS = (
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
     "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step", "sl_streaming_due",
-    "sl_compress_bf16", "sl_aggregate_apply_bf16", "sl_outer_step_bf16",
+    "sl_compress_bf16", "sl_aggregate_apply_bf16", "sl_outer_step_bf16", "sl_aggregate_apply_coded",
 )
 PROFILE_SLOTS = 9
 
@@ -67,6 +67,7 @@ def _load():
     L.sl_aggregate_apply.argtypes = [P, P, P, P]
     L.sl_outer_step.argtypes = [P, P, P, P, P, P]
     L.sl_compress_bf16.argtypes = [P, P, P, P, P, P]
+    L.sl_aggregate_apply_coded.argtypes = [P, P, P, P, P]
     L.sl_aggregate_apply_bf16.argtypes = [P, P, P, P]
     L.sl_outer_step_bf16.argtypes = [P, P, P, P, P, P]
     L.sl_outer_step_host.argtypes = [P, P, P, P, C.c_size_t, P, P, P, P]
@@ -314,6 +315,16 @@ class SparseLoCo:
         (0: the tensor's size); a damaged input shows in device_status() as SL_ERR_BAD_PAYLOAD."""
         _check(_L.sl_decode_payload(self._h, _dev_ptr(coded, torch.uint8), coded_bytes or coded.numel(),
                                     _dev_ptr(payload, torch.uint8), _stream()))
+
+    def aggregate_apply_coded(self, coded: List[Optional[torch.Tensor]], theta_sync,
+                              coded_bytes: Optional[Sequence[int]] = None) -> None:
+        """Decode, average and apply straight from entropy-coded payloads (None = absent worker).
+        `coded_bytes[r]` = readable bytes of coded[r] (default: the tensor's size)."""
+        arr = _ptr_array([_dev_ptr(p, torch.uint8) for p in coded])
+        sizes = (C.c_size_t * len(coded))()
+        for r, p in enumerate(coded):
+            sizes[r] = 0 if p is None else int(coded_bytes[r] if coded_bytes is not None and coded_bytes[r] else p.numel())
+        _check(_L.sl_aggregate_apply_coded(self._h, arr, sizes, _dev_ptr(theta_sync, torch.float32), _stream()))
 
     def set_tile_copies(self, use_tensor_maps: bool) -> None:
         _check(_L.sl_set_tile_copies(self._h, int(use_tensor_maps)))

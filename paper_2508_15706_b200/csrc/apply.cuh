@@ -3,6 +3,7 @@
 #pragma once
 #include "common.cuh"
 #include "quantiser.cuh"
+#include "index_codec.cuh"
 
 namespace {
 
@@ -33,6 +34,15 @@ namespace {
 // value - table[code] for FUSE 1; the same value back into the staging array for FUSE 2, the deferred
 // form), i.e. it does what pack_fix_kernel<1> / <2> does, saving that kernel's pass.
 //
+// FUSE 5: the payloads are in the entropy-coded wire form (index_codec.cuh) and are decoded here instead of
+// being expanded to records first.  A chunk's position in a worker's index stream is known only after
+// the chunks before it in its group of 16 (one directory entry per group), so a CTA takes whole groups
+// and walks their chunks in order; thread r keeps worker r's read position and decodes the chunk's gaps
+// through a 64-bit register window over the stream into a shared index list, and the rest of the kernel
+// reads the list and the code blocks.  Reads of a
+// stream are confined to the size its buffer is said to have; a stream that runs out reads as zeros
+// and is recorded as SL_ERR_BAD_PAYLOAD.
+//
 // A slot pair is 24 bits of the index block (bytes 3 m .. 3 m + 2) and one nibble of the code block, so
 // a lane assembles its part of a record with byte stores into the CTA's record buffer and the finished
 // records leave as 16-byte vectors.
@@ -44,6 +54,10 @@ struct FuseArgs {
     // FUSE 4 only: the global outer momentum and its coefficient, alpha and the divisor
     float* momentum;
     float mu, alpha, divisor;
+    // FUSE 5 only: layout of a coded payload, bits of index stream each worker's buffer holds
+    unsigned long long dir_off, stream_off;
+    unsigned long long stream_bits[kMaxR];
+    int* status;
 };
 
 constexpr int kApplyWarps = 4;
@@ -81,10 +95,24 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     float4* stage = tabs + 2 * kApplyBatch;  // theta of the chunk to come: vector i of thread t at [128 i + t]
     constexpr int WB = kApplyPerWarp;
     constexpr bool PACK = FUSE == 1 || FUSE == 2;  // quantise, write records and the error correction
-    constexpr bool RAW = FUSE >= 3;                // staged values travel unquantised
+    constexpr bool RAW = FUSE == 3 || FUSE == 4;   // staged values travel unquantised
+    constexpr bool STAGED = FUSE >= 1 && FUSE <= 4;  // the entries come from the staging arrays
+    constexpr bool CODED = FUSE == 5;              // the entries come from entropy-coded payloads
     const unsigned dump = (unsigned)(kChunk + tid);  // where an entry that does not count adds its 0
     // per-worker strides of the staging arrays, in index pairs / value pairs (kp is a multiple of 8)
-    const long long wstride = FUSE ? fa.n_chunks * (long long)fa.kp / 2 : 0;
+    const long long wstride = STAGED ? fa.n_chunks * (long long)fa.kp / 2 : 0;
+    // CODED: per worker kp decoded indices
+    uint16_t* sidx = reinterpret_cast<uint16_t*>(stage + kChunk / 4);
+    unsigned long long my_pos = 0;   // thread r: worker r's read position in its index stream
+    bool my_bad = false;
+    const int cb = (2 * k + 7) / 8;  // bytes of a chunk's code block in a coded payload
+    // the CTA's walk: chunk after chunk inside a group of kIxcGroup when CODED, else every gridDim-th chunk
+    auto next_of = [&](long long g) -> long long {
+        if (!CODED) return g + gridDim.x;
+        if ((g + 1) % kIxcGroup != 0 && g + 1 < n_chunks) return g + 1;
+        return (g / kIxcGroup + gridDim.x) * kIxcGroup;
+    };
+    const long long g_first = CODED ? (long long)blockIdx.x * kIxcGroup : (long long)blockIdx.x;
 
     for (int i = tid; i < kApplyTile / 4; i += kApplyThreads) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
@@ -97,12 +125,12 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
         for (int i = 0; i < 8; ++i) async_copy16(&stage[128 * i + tid], src + (long long)i * 8 * prs);
     };
     ChunkDesc cd_next;
-    if ((long long)blockIdx.x < n_chunks) {
-        cd_next = chunks[blockIdx.x];
+    if (g_first < n_chunks) {
+        cd_next = chunks[g_first];
         if (cd_next.len == kChunk) prefetch_theta(cd_next);
     }
 
-    for (long long g = blockIdx.x; g < n_chunks; g += gridDim.x) {
+    for (long long g = g_first; g < n_chunks; g = next_of(g)) {
         const ChunkDesc cd = cd_next;
         const int keff = min(k, cd.len);
         const bool full = cd.len == kChunk;
@@ -116,9 +144,85 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
 #pragma unroll
             for (int i = 0; i < 8; ++i) a[i] = stage[128 * i + tid];
         }
-        if (g + gridDim.x < n_chunks) {  // the block is free again (this thread's part of it): the next chunk's theta
-            cd_next = chunks[g + gridDim.x];
+        if (next_of(g) < n_chunks) {  // the block is free again (this thread's part of it): the next chunk's theta
+            cd_next = chunks[next_of(g)];
             if (cd_next.len == kChunk) prefetch_theta(cd_next);
+        }
+        if (CODED) {
+            if (tid < n_workers && pl.p[tid]) {
+                const unsigned long long sbits = fa.stream_bits[tid];
+                if (g == g_first || g % kIxcGroup == 0) {  // a new group: its directory entry
+                    my_pos = reinterpret_cast<const unsigned*>(pl.p[tid] + fa.dir_off)[g / kIxcGroup];
+                    if (my_pos > sbits) {
+                        my_bad = true;
+                        my_pos = sbits;
+                    }
+                }
+                const unsigned* __restrict__ stream = reinterpret_cast<const unsigned*>(pl.p[tid] + fa.stream_off);
+                const unsigned long long wtot = sbits >> 5;
+                // a 64-bit window over the stream, refilled a word at a time (consecutive words: mostly L1 hits;
+                // words past the stated size read as zeros)
+                unsigned long long win = 0, wnext = my_pos >> 5;
+                int have = 0;
+                auto refill = [&]() {  // at least 32 valid bits
+                    while (have < 32) {
+                        const unsigned x = wnext < wtot ? __ldg(stream + wnext) : 0u;
+                        win |= (unsigned long long)x << have;
+                        have += 32;
+                        ++wnext;
+                    }
+                };
+                refill();
+                {
+                    const int skip = (int)(my_pos & 31ull);
+                    win >>= skip;
+                    have -= skip;
+                }
+                const IxcCode code = ixc_code(cd.len, keff);
+                unsigned consumed = 0;
+                int prev = -1;
+                uint16_t* out = sidx + (size_t)tid * fa.kp;
+                for (int s = 0; s < keff; ++s) {
+                    refill();
+                    unsigned q = 0, inv = ~(unsigned)win;
+                    while (inv == 0u && q < 4096u) {  // 32 one-bits; a damaged stream cannot run away
+                        q += 32;
+                        win >>= 32;
+                        have -= 32;
+                        consumed += 32;
+                        refill();
+                        inv = ~(unsigned)win;
+                    }
+                    const int ones = inv ? __ffs(inv) - 1 : 0;  // one-bits up to the zero-bit
+                    q += ones;
+                    win >>= ones + 1;
+                    have -= ones + 1;
+                    consumed += ones + 1;
+                    unsigned r = 0;
+                    if (code.M > 1u) {  // truncated binary, most significant bit first
+                        refill();
+                        const int nb = (int)code.b - 1;
+                        if (nb) r = __brev((unsigned)win) >> (32 - nb);
+                        win >>= nb;
+                        have -= nb;
+                        consumed += nb;
+                        if (r >= code.cut) {
+                            r = ((r << 1) | ((unsigned)win & 1u)) - code.cut;
+                            win >>= 1;
+                            have -= 1;
+                            consumed += 1;
+                        }
+                    }
+                    prev = prev + 1 + (int)(q * code.M + r);
+                    out[s] = (uint16_t)((unsigned)prev & 0xFFFu);
+                }
+                my_pos += consumed;
+                if (my_pos > sbits) {
+                    my_bad = true;
+                    my_pos = sbits;
+                }
+            }
+            __syncthreads();  // the index lists of this chunk are complete
         }
         // which of this lane's slots exist in this chunk (the same for every worker)
         bool in0[PPL], in1[PPL];
@@ -128,9 +232,9 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
             in0[j] = 2 * m < keff;
             in1[j] = 2 * m + 1 < keff;
         }
-        const unsigned* idx_pairs = FUSE ? reinterpret_cast<const unsigned*>(fa.ws.idx + g * fa.kp) : nullptr;
-        float2* val_pairs = FUSE ? reinterpret_cast<float2*>(fa.ws.val + g * fa.kp) : nullptr;
-        const TStat* tstat = FUSE ? fa.ws.tstat + cd.tensor : nullptr;
+        const unsigned* idx_pairs = STAGED ? reinterpret_cast<const unsigned*>(fa.ws.idx + g * fa.kp) : nullptr;
+        float2* val_pairs = STAGED ? reinterpret_cast<float2*>(fa.ws.val + g * fa.kp) : nullptr;
+        const TStat* tstat = STAGED ? fa.ws.tstat + cd.tensor : nullptr;
 
         for (int r0 = 0; r0 < n_workers; r0 += kApplyBatch) {
             const int nb = min(kApplyBatch, n_workers - r0);
@@ -143,7 +247,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     const int r = r0 + tid;
                     if (RAW) {
                         h.w = 1.f;
-                    } else if (FUSE) {
+                    } else if (STAGED) {
                         const float4* st = reinterpret_cast<const float4*>(tstat + (long long)r * fa.n_tensors);
                         const float4 s0 = st[0], s1 = st[1];  // mu, sigma, 3 sigma, table[0] | table[1..3], pad
                         h = make_float4(s0.x, s0.z, 0.f, 1.f);
@@ -169,9 +273,16 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     pos[q][j] = 0u;
                     val[q][j] = make_float2(0.f, 0.f);
                     if (w0 + q < nb && in0[j]) {
-                        if (FUSE) {
+                        if (STAGED) {
                             pos[q][j] = idx_pairs[r * wstride + m];
                             val[q][j] = val_pairs[r * wstride + m];
+                        } else if (CODED) {
+                            if (pl.p[r]) {  // the decoded index pair and the pair's nibble of the chunk's code block
+                                const unsigned x = reinterpret_cast<const unsigned*>(sidx + (size_t)r * fa.kp)[m];
+                                const unsigned nib = (__ldg(pl.p[r] + 16ll * fa.n_tensors + (long long)cb * g + (m >> 1)) >> ((m & 1) * 4)) & 0xFu;
+                                pos[q][j] = x;
+                                val[q][j] = make_float2(__uint_as_float(nib & 3u), __uint_as_float(nib >> 2));
+                            }
                         } else if (pl.p[r]) {
                             // 24 bits at byte 3 m of the record, from the aligned words around it (the second
                             // word may belong to the code block or the padding: inside the record either way)
@@ -321,6 +432,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
         }
         // (the next chunk's first additions come after several CTA barriers: the cleared tile is seen by all)
     }
+    if (CODED && my_bad) atomicExch(fa.status, (int)SL_ERR_BAD_PAYLOAD);
 }
 
 }  // namespace

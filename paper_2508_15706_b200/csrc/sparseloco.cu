@@ -80,6 +80,7 @@ struct sl_ctx {
     int* d_status;                      // device status word (SL_OK or what a kernel recorded)
     // entropy-coded payload: byte offsets of the directory and the index stream, worst-case size
     size_t ixc_dir_off, ixc_stream_off, ixc_capacity;
+    bool coded_attr_set;
     bool deferred;              // deferred error-feedback subtraction (sl_set_ef_deferred)
     bool pending;               // corrected values of the last step still wait in the workspace
     float* pending_e[kMaxR];    // the error buffers they belong to
@@ -517,6 +518,47 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
 #undef SL_APPLY
     prof_mark(c, 8, st);
     if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
+    SL_CUDA(cudaGetLastError());
+    return SL_OK;
+}
+
+// Eq. 2 lines 3-4 straight from entropy-coded payloads (decode_avg_apply_kernel<., 5>).
+sl_status launch_apply_coded(sl_ctx* c, const PayloadPtrs& pl, const size_t* coded_bytes, int present, float* theta_sync,
+                             cudaStream_t st) {
+    if (present == 0) return SL_OK;
+    const int R = c->cfg.R;
+    const double D = c->cfg.divide_by_present ? (double)present : (double)R;
+    const float scale = (float)(-(double)c->cfg.outer_lr / D);
+    FuseArgs fa;
+    memset(&fa, 0, sizeof(fa));
+    fa.n_chunks = c->n_chunks;
+    fa.n_tensors = c->n_tensors;
+    fa.kp = c->kp;
+    fa.dir_off = c->ixc_dir_off;
+    fa.stream_off = c->ixc_stream_off;
+    fa.status = c->d_status;
+    for (int r = 0; r < R; ++r) fa.stream_bits[r] = pl.p[r] ? (unsigned long long)((coded_bytes[r] - c->ixc_stream_off) / 4 * 4) * 8ull : 0ull;
+    WorkerPtrs wp;
+    memset(&wp, 0, sizeof(wp));
+    const size_t smem = (apply_smem_bytes(c->cfg.k) + (size_t)R * c->kp * sizeof(uint16_t) + 15) / 16 * 16;
+    if (smem > 227u * 1024u) return SL_ERR_UNSUPPORTED;
+    const long long groups = (c->n_chunks + kIxcGroup - 1) / kIxcGroup;
+    const long long fit = (227ll * 1024) / ((long long)smem + 1024);
+    const long long resident = (long long)c->n_sms * (fit < kApplyCtasPerSm ? (fit < 1 ? 1 : fit) : kApplyCtasPerSm);
+    const unsigned grid = (unsigned)(groups < resident ? groups : resident);
+    const int ppl = (c->cfg.k + 63) / 64;
+    if (!c->coded_attr_set) {  // (once per context: the attribute call is slow)
+        if (ppl <= 1) SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else if (ppl <= 2) SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<2, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<4, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        c->coded_attr_set = true;
+    }
+    if (ppl <= 1)
+        decode_avg_apply_kernel<1, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
+    else if (ppl <= 2)
+        decode_avg_apply_kernel<2, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
+    else
+        decode_avg_apply_kernel<4, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -1265,6 +1307,30 @@ sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, size_t coded_bytes,
         payload, c->d_status);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
+}
+
+sl_status sl_aggregate_apply_coded(sl_ctx* c, const uint8_t* const* coded, const size_t* coded_bytes, float* theta_sync,
+                                   void* stream) {
+    if (!c || !coded || !theta_sync) return SL_ERR_INVALID_ARG;
+    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
+    if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
+    if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
+    PayloadPtrs pl;
+    memset(&pl, 0, sizeof(pl));
+    size_t sizes[kMaxR];
+    int present = 0;
+    for (int r = 0; r < c->cfg.R; ++r) {
+        if (misaligned(coded[r])) return SL_ERR_ALIGNMENT;
+        pl.p[r] = coded[r];
+        present += coded[r] != nullptr;
+        size_t n = coded_bytes ? coded_bytes[r] : 0;
+        if (n == 0 || n > c->ixc_capacity) n = c->ixc_capacity;
+        if (coded[r] && n < c->ixc_stream_off) return SL_ERR_INVALID_ARG;
+        sizes[r] = n;
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
+    return launch_apply_coded(c, pl, sizes, present, theta_sync, static_cast<cudaStream_t>(stream));
 }
 
 sl_status sl_set_tile_copies(sl_ctx* c, int32_t use_tensor_maps) {

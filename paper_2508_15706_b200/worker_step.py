@@ -60,8 +60,13 @@ class WorkerStep:
     """One rank of the worker-per-rank outer step.  `ops` is a context created with R = world size."""
 
     def __init__(self, ops, payload_bytes: int, world: int, rank: int, device, group=None, coded: bool = False,
-                 coded_capacity: int = 0):
+                 coded_capacity: int = 0, expand_coded: bool = False):
+        """`coded`: entropy-coded indices on the wire.  The gathered coded payloads then go straight into
+        `aggregate_apply_coded` (decoding fused into the update); with `expand_coded` each is first
+        expanded to the 12-bit form with `decode_payload` (what a receiver does that wants to run the
+        payload validator on untrusted input) and `aggregate_apply` consumes those."""
         self.ops, self.world, self.rank, self.coded = ops, world, rank, coded
+        self.expand_coded = expand_coded
         self.own = torch.zeros(payload_bytes, dtype=torch.uint8, device=device)
         if coded:
             # entropy-coded indices on the wire: about 0.68 of the plain payload at k = 64
@@ -87,6 +92,10 @@ class WorkerStep:
                 self.ops.encode_payload(self.own, self.own_coded, self.coded_size)
                 used = int(self.coded_size.item())
             rows, flags, sizes = self.exchange.gather(self.own_coded, participate, used)
+            if not self.expand_coded:
+                self.ops.aggregate_apply_coded([rows[r] if flags[r] else None for r in range(self.world)], theta_sync,
+                                               sizes)
+                return flags
             payloads = []
             for r in range(self.world):
                 if not flags[r]:

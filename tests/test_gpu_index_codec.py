@@ -139,3 +139,75 @@ def test_damaged_coded_payloads_stay_inside_the_buffer():
 
     back, st, val = run(lambda h: None, stream_off + 16)  # truncated: most of the stream is missing
     assert st == 4
+
+
+@pytest.mark.parametrize("k,R", [(1, 2), (8, 3), (41, 3), (64, 16), (123, 5), (256, 3), (64, 40)])
+def test_aggregate_apply_straight_from_coded_payloads(k, R):
+    """sl_aggregate_apply_coded (the decoding fused into the update kernel; Eq. 2 lines 3-4) must leave the
+    bits that sl_decode_payload for every worker + sl_aggregate_apply leave, with an absent worker and with
+    the exact coded sizes as read limits; and agree with the oracle's update within 1e-6 x RMS."""
+    wl = I.Workload("codec_apply", SHAPES, R=R, k=k, recipe="student_t4", seed=800 + k + R, outer_lr=0.7)
+    c = _case(wl, e_scale=0.5)
+    c.fill_local(0)
+    c.step()
+    cap = c.sl.coded_payload_capacity()
+    size = torch.zeros(1, dtype=torch.int64, device=c.dev)
+    coded, sizes = [], []
+    for r in range(R):
+        buf = torch.full((cap,), 0x5A, dtype=torch.uint8, device=c.dev)
+        c.sl.encode_payload(c.payloads[r], buf, size)
+        sizes.append(int(size.item()))
+        coded.append(buf)
+    absent = 1 if R > 1 else None
+    plain = [None if r == absent else c.payloads[r] for r in range(R)]
+    theta_a = c.theta.clone()
+    c.sl.aggregate_apply(plain, theta_a)
+    theta_b = torch.cat([c.theta.clone(), torch.full((1024,), 7.5, device=c.dev)])  # a band that must survive
+    c.sl.aggregate_apply_coded([None if r == absent else coded[r] for r in range(R)], theta_b, sizes)
+    torch.cuda.synchronize()
+    assert c.sl.device_status() == 0
+    n = c.theta.numel()
+    assert torch.equal(theta_b[:n].view(torch.int32), theta_a.view(torch.int32))
+    assert bool((theta_b[n:] == 7.5).all())
+    # the oracle on the same payloads
+    tab = O.Table(c.shapes, c.offs)
+    cfg = O.Config(k=k, R=R, outer_lr=wl.outer_lr)
+    th = c.theta.cpu().numpy().copy()
+    O.aggregate_apply(cfg, tab, [None if p is None else p.cpu().numpy() for p in plain], th)
+    rms = float(np.sqrt(np.mean(th.astype(np.float64) ** 2)))
+    assert float(np.max(np.abs(theta_b[:n].cpu().numpy().astype(np.float64) - th))) <= 1e-6 * rms
+
+
+def test_coded_apply_with_a_cut_stream_stays_in_bounds_and_reports():
+    """A coded payload whose stated size cuts the index stream short: the update of that call is wrong by
+    definition, but every access stays inside the stated sizes and inside theta, and the device status
+    says SL_ERR_BAD_PAYLOAD."""
+    from paper_2508_15706_b200 import binding as B
+    k, R = 64, 2
+    wl = I.Workload("codec_cut", SHAPES, R=R, k=k, recipe="student_t4", seed=31, outer_lr=0.7)
+    c = _case(wl, e_scale=0.5)
+    c.fill_local(0)
+    c.step()
+    cap = c.sl.coded_payload_capacity()
+    size = torch.zeros(1, dtype=torch.int64, device=c.dev)
+    coded, sizes = [], []
+    for r in range(R):
+        buf = torch.zeros(cap, dtype=torch.uint8, device=c.dev)
+        c.sl.encode_payload(c.payloads[r], buf, size)
+        sizes.append(int(size.item()))
+        coded.append(buf)
+    # the buffer really ends where the call is told it ends: a copy of exactly that many bytes
+    cut = (sizes[0] + c.sl.coded_payload_capacity() * 0) // 2 // 16 * 16
+    fixed = 16 * len(c.shapes)  # (tables; the stream starts well after this)
+    assert cut > fixed
+    short = coded[0][:cut].clone()
+    theta = torch.cat([c.theta.clone(), torch.full((1024,), 7.5, device=c.dev)])
+    try:
+        c.sl.aggregate_apply_coded([short, coded[1]], theta, [cut, sizes[1]])
+        torch.cuda.synchronize()
+        st = c.sl.device_status()
+        assert st == B.SL_ERR_BAD_PAYLOAD
+    except B.SlError as e:   # a size that does not even reach the stream is refused on the host
+        assert e.status == B.SL_ERR_INVALID_ARG
+    assert bool((theta[c.theta.numel():] == 7.5).all())
+    assert bool(torch.isfinite(theta).all())

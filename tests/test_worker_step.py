@@ -53,6 +53,9 @@ class OracleOps:  # the binding's method names over the CPU oracle (the kernels'
         size[0] = c.size
     def decode_payload(self, coded, payload, coded_bytes=0):
         payload.copy_(torch.from_numpy(O.ixc_decode_payload(cfg, tab, coded[:coded_bytes].numpy().copy())))
+    def aggregate_apply_coded(self, coded, theta, sizes):
+        plain = [None if c is None else O.ixc_decode_payload(cfg, tab, c[:n].numpy().copy()) for c, n in zip(coded, sizes)]
+        O.aggregate_apply(cfg, tab, plain, theta.numpy())
 
 
 theta = I.theta_sync(wl, "cpu")
@@ -60,7 +63,8 @@ local = I.theta_local(wl, theta, rank, 0)
 e = I.initial_error(wl, rank, "cpu", scale=0.5)
 nbytes = O.payload_bytes(cfg, tab)
 coded = mode.startswith("coded")
-ws = WorkerStep(OracleOps(), nbytes, world, rank, "cpu", coded=coded, coded_capacity=2 * nbytes)
+expand = mode == "coded_expand"
+ws = WorkerStep(OracleOps(), nbytes, world, rank, "cpu", coded=coded, coded_capacity=2 * nbytes, expand_coded=expand)
 sits_out = mode.startswith("absent") and rank == world - 1
 flags = ws.step(theta, local, e, participate=not sits_out)
 
@@ -77,8 +81,14 @@ for r in range(world):
         assert np.array_equal(ws.own.numpy(), out.payload)
 O.aggregate_apply(cfg, tab, pays, theta_ref)
 same = bool(np.array_equal(theta.numpy().view(np.uint32), theta_ref.view(np.uint32)))
-rows_ok = all(p is None or np.array_equal((ws.plain[r] if coded else ws.exchange.gathered[r]).numpy(), p)
-              for r, p in enumerate(pays))
+def row(r):
+    if not coded:
+        return ws.exchange.gathered[r].numpy()
+    if expand:
+        return ws.plain[r].numpy()
+    n = int(ws.exchange.meta[r, 1])   # the gathered coded row, expanded here
+    return O.ixc_decode_payload(cfg, tab, ws.exchange.gathered[r][:n].numpy().copy())
+rows_ok = all(p is None or np.array_equal(row(r), p) for r, p in enumerate(pays))
 wire = int(ws.exchange.meta[:, 1].max())
 dist.barrier()
 print(json.dumps({"rank": rank, "same": same, "rows_ok": rows_ok, "flags": flags, "wire": wire, "plain": nbytes}))
@@ -86,7 +96,7 @@ dist.destroy_process_group()
 """
 
 
-@pytest.mark.parametrize("mode,world", [("plain", 2), ("plain", 3), ("coded", 2), ("absent_R", 3), ("absent_present", 3)])
+@pytest.mark.parametrize("mode,world", [("plain", 2), ("plain", 3), ("coded", 2), ("coded_expand", 2), ("absent_R", 3), ("absent_present", 3)])
 def test_worker_per_rank_step_equals_one_process_step(tmp_path, mode, world):
     port = _free_port()
     script = tmp_path / "w.py"
@@ -104,7 +114,7 @@ def test_worker_per_rank_step_equals_one_process_step(tmp_path, mode, world):
         assert got["rank"] == rank and got["same"] and got["rows_ok"], got
         want_flags = [not (mode.startswith("absent") and r == world - 1) for r in range(world)]
         assert got["flags"] == want_flags
-        if mode == "coded":
+        if mode.startswith("coded"):
             assert got["wire"] < got["plain"]      # fewer bytes travel than the 12-bit form has
         else:
             assert got["wire"] == got["plain"]
