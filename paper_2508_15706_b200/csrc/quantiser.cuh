@@ -138,9 +138,9 @@ chunk_bins_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
     *reinterpret_cast<uint4*>(ws.pcnt + i * 4) = make_uint4(n0, n1, n2, n3);
 }
 
-// One warp per (worker, tensor): the chunk partials are added group by group (64 consecutive chunks
-// per group, left to right inside the group: one lane per group, 32 groups at a time), then the
-// group sums are added left to right.
+// One CTA of four warps per (worker, tensor): the chunk partials are added group by group (64 consecutive
+// chunks per group, left to right inside the group: one thread per group, 128 groups at a time, group sums
+// parked in shared memory), then the group sums are added left to right by the first warp.
 // STAGE 0: psum -> mu.  STAGE 1: psum -> sigma, 3 sigma.  STAGE 2: pbin/pcnt -> table (+ payload header).
 constexpr int kSumGroup = 64;
 
@@ -149,9 +149,11 @@ __global__ void __launch_bounds__(128)
 tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, int n_workers, int n_tensors,
                      Workspace ws, WorkerPtrs ptrs) {
     constexpr int NV = STAGE < 2 ? 1 : 4;  // running sums
-    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long w = (long long)blockIdx.x * 4 + wib;
-    if (w >= (long long)n_workers * n_tensors) return;
+    __shared__ double gsum[128][NV];
+    __shared__ unsigned long long cnt_s[4][4];
+    const int tid = threadIdx.x, wib = tid >> 5, lane = tid & 31;
+    const long long w = blockIdx.x;
+    if (w >= (long long)n_workers * n_tensors) return;  // (whole CTA)
     const int r = (int)(w / n_tensors), t = (int)(w - (long long)r * n_tensors);
     const TensorInfo ti = tinfo[t];
     const long long first = (long long)r * n_chunks + ti.first_chunk;
@@ -163,39 +165,39 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = 0.0;
     unsigned long long cn[4] = {0, 0, 0, 0};
-    for (long long g0 = 0; g0 < n_groups; g0 += 32) {
-        // this lane's group
+    for (long long g0 = 0; g0 < n_groups; g0 += 128) {
+        // this thread's group
         double gs[NV];
 #pragma unroll
         for (int v = 0; v < NV; ++v) gs[v] = 0.0;
-        const long long c0 = (g0 + lane) * kSumGroup;
+        const long long c0 = (g0 + tid) * kSumGroup;
         const int cnt = (int)max(0ll, min((long long)kSumGroup, ti.n_chunks - c0));
         if (STAGE < 2) {
             const double* __restrict__ src = ws.psum + first + c0;
             int c = 0;
-            for (; c + 8 <= cnt; c += 8) {
-                double x[8];
+            for (; c + 16 <= cnt; c += 16) {  // sixteen loads in flight, additions in chunk order
+                double x[16];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) x[q] = src[c + q];
+                for (int q = 0; q < 16; ++q) x[q] = src[c + q];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) gs[0] += x[q];
+                for (int q = 0; q < 16; ++q) gs[0] += x[q];
             }
             for (; c < cnt; ++c) gs[0] += src[c];
         } else {
             const double2* __restrict__ src = reinterpret_cast<const double2*>(ws.pbin + (first + c0) * 4);
             const uint4* __restrict__ csrc = reinterpret_cast<const uint4*>(ws.pcnt + (first + c0) * 4);
             int c = 0;
-            for (; c + 4 <= cnt; c += 4) {  // loads of four chunks in flight, additions in chunk order
-                double2 lo[4], hi[4];
-                uint4 pc[4];
+            for (; c + 8 <= cnt; c += 8) {  // loads of eight chunks in flight, additions in chunk order
+                double2 lo[8], hi[8];
+                uint4 pc[8];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < 8; ++q) {
                     lo[q] = src[2 * (c + q)];
                     hi[q] = src[2 * (c + q) + 1];
                     pc[q] = csrc[c + q];
                 }
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < 8; ++q) {
                     gs[0] += lo[q].x; gs[1 % NV] += lo[q].y; gs[2 % NV] += hi[q].x; gs[3 % NV] += hi[q].y;
                     cn[0] += pc[q].x; cn[1] += pc[q].y; cn[2] += pc[q].z; cn[3] += pc[q].w;
                 }
@@ -207,13 +209,31 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
                 cn[0] += pc.x; cn[1] += pc.y; cn[2] += pc.z; cn[3] += pc.w;
             }
         }
-        // the group sums of these 32 groups, in group order (every lane runs the same chain)
-        const int ng = (int)min(32ll, n_groups - g0);
-        for (int l = 0; l < ng; ++l) {
 #pragma unroll
-            for (int v = 0; v < NV; ++v) acc[v] += __shfl_sync(kFull, gs[v], l);
+        for (int v = 0; v < NV; ++v) gsum[tid][v] = gs[v];
+        __syncthreads();
+        // the group sums of these 128 groups, in group order (every lane of the first warp runs the same chain)
+        if (wib == 0) {
+            const int ng = (int)min(128ll, n_groups - g0);
+            for (int l = 0; l < ng; ++l) {
+#pragma unroll
+                for (int v = 0; v < NV; ++v) acc[v] += gsum[l][v];
+            }
         }
+        __syncthreads();
     }
+    if (STAGE == 2) {  // the counts: integers, any order
+#pragma unroll
+        for (int bb = 0; bb < 4; ++bb) {
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) cn[bb] += __shfl_xor_sync(kFull, cn[bb], d);
+            if (lane == 0) cnt_s[wib][bb] = cn[bb];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int bb = 0; bb < 4; ++bb) cn[bb] = cnt_s[0][bb] + cnt_s[1][bb] + cnt_s[2][bb] + cnt_s[3][bb];
+    }
+    if (wib != 0) return;
 
     if (STAGE < 2) {
         if (lane == 0) {
@@ -226,11 +246,6 @@ tensor_reduce_kernel(const TensorInfo* __restrict__ tinfo, long long n_chunks, i
             }
         }
     } else {
-#pragma unroll
-        for (int bb = 0; bb < 4; ++bb) {
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) cn[bb] += __shfl_xor_sync(kFull, cn[bb], d);
-        }
         if (lane == 0) {
             float lut[4];
 #pragma unroll

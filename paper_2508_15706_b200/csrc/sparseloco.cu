@@ -400,13 +400,14 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     }
     prof_mark(c, 0, st);
     const unsigned cb = blocks_for(WG, 128), tb = blocks_for((long long)workers * T, 4);
+    const unsigned tr = (unsigned)((long long)workers * T);  // tensor_reduce_kernel: one CTA per (worker, tensor)
     chunk_sum_kernel<0><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
     prof_mark(c, 1, st);
-    tensor_reduce_kernel<0><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    tensor_reduce_kernel<0><<<tr, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 2, st);
     chunk_sum_kernel<1><<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
     prof_mark(c, 3, st);
-    tensor_reduce_kernel<1><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    tensor_reduce_kernel<1><<<tr, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 4, st);
     if (wide_quant(c)) {  // 1, 3 or 4 bits: the general-width kernels, records and error correction in place
         const WideSpace wq = carve_wide(c, workers);
@@ -435,7 +436,7 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     }
     chunk_bins_kernel<<<cb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws);
     prof_mark(c, 5, st);
-    tensor_reduce_kernel<2><<<tb, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
+    tensor_reduce_kernel<2><<<tr, 128, 0, st>>>(c->d_tinfo, G, workers, T, ws, ptrs);
     prof_mark(c, 6, st);
     const unsigned pb = blocks_for(WG, 4);
     if (skip_pack)
