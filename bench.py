@@ -236,13 +236,7 @@ def run_ours(args) -> dict:
     ef_ms, ef_n = prof["ef_select"]
     ef_avg_ms = ef_ms / max(ef_n, 1)
     ef_bytes = ef_select_bytes_per_param(wl.R) * N
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except Exception:
-        pass
-    peak = float(peaks.get("hbm_gbs", 6650.0))
-    peak_src = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
+    peak, peak_src = measured_peak_gbs()
     achieved = ef_bytes / (ef_avg_ms * 1e-3) / 1e9
     traffic = None
     if NCU_EF_SELECT_DRAM_BYTES_PER_PARAM_WORKER is not None:
@@ -535,15 +529,26 @@ def variants_bench(torch, I, dev, build, peak: float) -> dict:
     return out
 
 
-def options_bench(torch, I, dev, peak: float) -> dict:
+def measured_peak_gbs():
+    """(HBM copy bandwidth in GB/s, where the figure comes from)."""
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    return float(peaks.get("hbm_gbs", 6650.0)), \
+        ("measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s")
+
+
+def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int = 8) -> dict:
     """The settings outside the paper's main configuration (quantiser widths of its ablation, no quantiser,
     densities up to half a chunk, bfloat16 storage) on the 12-layer stack with R = 8: ms per outer step and
     the rate on the state the step must stream ((12 R + 8) bytes per parameter in fp32, half in bfloat16:
     theta_r and e read, e written per worker; theta read and written).  These run in plain kernels."""
     import dataclasses
     from paper_2508_15706_b200.binding import SparseLoCo
-    base = dataclasses.replace(I.workload("c5_l12"), R=8)
-    N, R = base.numel, 8
+    base = dataclasses.replace(I.workload(workload), R=R)
+    N = base.numel
     shapes, offs = [(t.rows, t.cols) for t in base.tensors], I.offsets(base.tensors)
     theta32 = I.theta_sync(base, dev)
     local32 = [I.theta_local(base, theta32, r, 0) for r in range(R)]
@@ -554,7 +559,7 @@ def options_bench(torch, I, dev, peak: float) -> dict:
              ("quant_bits=32 k=64 (no quantiser)", 32, 64, False),
              ("quant_bits=2 k=512", 2, 512, False), ("quant_bits=2 k=2048", 2, 2048, False),
              ("bf16 storage, quant_bits=2 k=64", 2, 64, True)]
-    out = {"params": N, "R": R}
+    out = {"workload": workload, "params": N, "R": R}
     for name, bits, k, half in cases:
         sl = SparseLoCo(shapes, offs, k=k, R=R, beta=base.beta, outer_lr=base.outer_lr, quant_bits=bits,
                         bf16_storage=half)
@@ -805,6 +810,9 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense DiLoCo comparator line")
     ap.add_argument("--codec", action="store_true", help="also time the entropy-coded index format on one payload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--options-only", action="store_true",
+                    help="time only the settings outside the main configuration (options_bench) on --workload")
+    ap.add_argument("--options-workers", type=int, default=8)
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")
     args = ap.parse_args()
@@ -813,6 +821,13 @@ def main():
         sys.exit(spawn_ranks(args.gpus))
     if args.impl == "reference":
         out = run_reference(args)
+    elif args.options_only:  # the settings outside the main configuration alone (small workloads: profiler captures)
+        import torch
+        from paper_2508_15706_b200 import inputs as I
+        torch.cuda.set_device(0)
+        out = options_bench(torch, I, torch.device("cuda", 0), measured_peak_gbs()[0],
+                            workload=args.workload if args.workload != DEFAULT_WORKLOAD else "c5_l12",
+                            R=args.options_workers)
     elif args.mode == "worker-per-gpu":
         out = run_worker_per_gpu(args)
     else:
