@@ -80,7 +80,6 @@ struct sl_ctx {
     int* d_status;                      // device status word (SL_OK or what a kernel recorded)
     // entropy-coded payload: byte offsets of the directory and the index stream, worst-case size
     size_t ixc_dir_off, ixc_stream_off, ixc_capacity;
-    bool coded_attr_set;
     bool deferred;              // deferred error-feedback subtraction (sl_set_ef_deferred)
     bool pending;               // corrected values of the last step still wait in the workspace
     float* pending_e[kMaxR];    // the error buffers they belong to
@@ -548,12 +547,6 @@ sl_status launch_apply_coded(sl_ctx* c, const PayloadPtrs& pl, const size_t* cod
     const long long resident = (long long)c->n_sms * (fit < kApplyCtasPerSm ? (fit < 1 ? 1 : fit) : kApplyCtasPerSm);
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
     const int ppl = (c->cfg.k + 63) / 64;
-    if (!c->coded_attr_set) {  // (once per context: the attribute call is slow)
-        if (ppl <= 1) SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        else if (ppl <= 2) SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<2, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        else SL_CUDA(cudaFuncSetAttribute(decode_avg_apply_kernel<4, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        c->coded_attr_set = true;
-    }
     if (ppl <= 1)
         decode_avg_apply_kernel<1, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
     else if (ppl <= 2)
@@ -758,14 +751,16 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
     SL_HALF_ATTR(true, 2); SL_HALF_ATTR(false, 2);
 #undef SL_HALF_ATTR
     per_sm = 1;
-    {   // the apply kernel's shared memory depends on k alone: sized once
-        const int asz = (int)apply_smem_bytes(cfg->k < kFastMaxK ? cfg->k : kFastMaxK);
+    {   // the apply kernel's shared memory grows with k (and, for coded payloads, with R): the limit is a property of
+        // the function, shared by every context of the process, so it is set to the most any context can ask for
+        const int asz = 227 * 1024;
 #define SL_APPLY_ATTR(PPLV, FUSEV)                                                                                     \
     if (e == cudaSuccess)                                                                                              \
         e = cudaFuncSetAttribute(decode_avg_apply_kernel<PPLV, FUSEV>, cudaFuncAttributeMaxDynamicSharedMemorySize, asz)
         SL_APPLY_ATTR(1, 0); SL_APPLY_ATTR(1, 1); SL_APPLY_ATTR(1, 2); SL_APPLY_ATTR(1, 3); SL_APPLY_ATTR(1, 4);
         SL_APPLY_ATTR(2, 0); SL_APPLY_ATTR(2, 1); SL_APPLY_ATTR(2, 2); SL_APPLY_ATTR(2, 3); SL_APPLY_ATTR(2, 4);
         SL_APPLY_ATTR(4, 0); SL_APPLY_ATTR(4, 1); SL_APPLY_ATTR(4, 2); SL_APPLY_ATTR(4, 3); SL_APPLY_ATTR(4, 4);
+        SL_APPLY_ATTR(1, 5); SL_APPLY_ATTR(2, 5); SL_APPLY_ATTR(4, 5);
 #undef SL_APPLY_ATTR
     }
     c->n_sms = n_sms;

@@ -496,3 +496,29 @@ def test_read_stats_matches_the_oracle_statistics():
             mu, sigma, lut = out.stats[0, 0], out.stats[0, 1], out.stats[0, 2:6]
             want = np.array([mu, sigma, np.float32(3.0) * sigma, *lut, 0.0], np.float32)
             assert np.array_equal(got[j].view(np.uint32), want.view(np.uint32)), (r, t.name, got[j], want)
+
+
+def test_two_live_contexts_with_different_k():
+    """Kernel attributes (the dynamic shared-memory limit) belong to the function, not to a context: a
+    context created later with a smaller k must not take away what an earlier one with a larger k needs."""
+    from paper_2508_15706_b200 import binding as B
+    dev = torch.device("cuda", torch.cuda.current_device())
+    shapes = [(128, 128), (1, 5000)]
+    big = B.SparseLoCo(shapes, k=256, R=2)
+    small = B.SparseLoCo(shapes, k=8, R=2)       # created after `big`
+    n = big.flat_elems()
+    g = torch.Generator(device=dev).manual_seed(5)
+    theta = torch.randn(n, device=dev, generator=g) * 0.02
+    for sl in (big, small, big):
+        local = [theta - 1e-3 * torch.randn(n, device=dev, generator=g) for _ in range(2)]
+        e = [torch.zeros(n, device=dev) for _ in range(2)]
+        pay = [torch.zeros(sl.payload_bytes(), dtype=torch.uint8, device=dev) for _ in range(2)]
+        sl.outer_step(theta, local, e, pay)
+        sl.aggregate_apply(pay, theta)
+        cap = sl.coded_payload_capacity()
+        coded = torch.zeros(cap, dtype=torch.uint8, device=dev)
+        size = torch.zeros(1, dtype=torch.int64, device=dev)
+        sl.encode_payload(pay[0], coded, size)
+        sl.aggregate_apply_coded([coded, None], theta, [int(size.item()), 0])
+        torch.cuda.synchronize()
+        assert sl.device_status() == 0
