@@ -76,7 +76,7 @@ typedef struct {
     int32_t k;                 /* entries kept per chunk, 1..2048 (the paper's density sweeps reach half a
                                   chunk).  The tuned kernels serve k <= 256; beyond that the selection is the exact
                                   bitwise search and packing / decoding run in the plain kernels of the
-                                  quantiser ablation: no deferral, no wire codec, no validation, no quant_bits = 32,
+                                  quantiser ablation: no deferral, no wire codec, no quant_bits = 32,
                                   no Top-k baselines */
     int32_t R;                 /* workers, 1..64 */
     int32_t H;                 /* inner steps; carried for the caller, >= 1, unused by the math */
@@ -84,7 +84,7 @@ typedef struct {
     float outer_lr;            /* alpha, finite */
     int32_t quant_bits;        /* 2 (the paper's setting; the fast path); 1, 3 or 4 (its ablation: 2^bits
                                   uniform bins over [-6 sigma, 6 sigma], plain kernels, no deferral, no wire
-                                  codec, no validation); or 32 = no quantiser: the selected values are averaged
+                                  codec); or 32 = no quantiser: the selected values are averaged
                                   as they are (sl_outer_step only: there is no payload format, payloads may be
                                   NULL) */
     int32_t ef_enabled;        /* 0 during the error-feedback freeze (App. "Freezing Error
@@ -322,7 +322,9 @@ sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fr
 
 /* Check one payload before trusting it: every index < chunk length and strictly ascending over
  * the used slots, unused slots and padding zero, table entries finite.  Writes SL_OK or
- * SL_ERR_BAD_PAYLOAD to *dev_status (device int32); never traps. */
+ * SL_ERR_BAD_PAYLOAD to *dev_status (device int32); never traps.  Serves every quantiser width and
+ * every k (the record layout is the same: 12-bit indices, then the codes); UNSUPPORTED only with
+ * quant_bits = 32, which has no payload. */
 sl_status sl_validate_payload(sl_ctx* ctx, const uint8_t* payload, int32_t* dev_status,
                               void* cuda_stream);
 

@@ -358,7 +358,8 @@ __device__ __forceinline__ void select_dense(const float (&u)[128], USource src,
     for (int j = 0; j < CPL; ++j) {
         const unsigned t = lane + 32u * j;
         cp[j] = t < n_b ? cand[t] : 0u;
-        ck[j] = t < n_b ? (usrc_load<GLOBAL>(src, cp[j]) & 0x7FFFFFFFu) : 0u;
+        // (indices at or beyond the chunk's length hold key 0 and are never fetched: nothing exists there)
+        ck[j] = (t < n_b && (int)cp[j] < len) ? (usrc_load<GLOBAL>(src, cp[j]) & 0x7FFFFFFFu) : 0u;
     }
     // (an empty place has key 0; when lo = 0 it would count, so empty places are excluded by position)
     unsigned l2 = lo, h2 = hi, cl2 = n_b, ch2 = 0;  // count(>= l2) = cl2 >= need > ch2 = count(>= h2), within the list

@@ -1394,14 +1394,15 @@ sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fr
 
 sl_status sl_validate_payload(sl_ctx* c, const uint8_t* payload, int32_t* dev_status, void* stream) {
     if (!c || !payload || !dev_status) return SL_ERR_INVALID_ARG;
-    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // checks the 2-bit payload only
+    if (c->cfg.quant_bits == 32) return SL_ERR_UNSUPPORTED;  // unquantised values have no payload format
     if (misaligned(payload)) return SL_ERR_ALIGNMENT;
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     set_status_kernel<<<1, 1, 0, st>>>(dev_status, (int)SL_OK);
     const long long items = c->n_chunks > c->n_tensors ? c->n_chunks : c->n_tensors;
-    validate_kernel<<<blocks_for(items, 128), 128, 0, st>>>(c->d_chunks, c->n_chunks, c->n_tensors, c->cfg.k, payload,
+    validate_kernel<<<blocks_for(items, 128), 128, 0, st>>>(c->d_chunks, c->n_chunks, c->n_tensors, c->cfg.k, c->qbits,
+                                                            header_bytes_q(c->qbits), c->rec_base, c->rec_stride, payload,
                                                             dev_status);
     SL_CUDA(cudaGetLastError());
     return SL_OK;

@@ -404,9 +404,11 @@ def test_runs_are_bit_reproducible():
         assert torch.equal(x, y)
 
 
-def test_validate_payload_flags_corruption():
-    wl = I.Workload("val", SMALL, R=1, k=41, recipe="normal", seed=71)
-    c = _case(wl)
+@pytest.mark.parametrize("bits,k", [(2, 41), (1, 41), (3, 64), (4, 41), (2, 300), (4, 1000)])
+def test_validate_payload_flags_corruption(bits, k):
+    """(every quantiser width and k beyond 256 share the record layout: 12-bit indices, then the codes)"""
+    wl = I.Workload("val", SMALL, R=1, k=k, recipe="normal", seed=71)
+    c = _case(wl, quant_bits=bits)
     c.fill_local(0)
     c.step()
     status = torch.full((1,), -1, dtype=torch.int32, device=c.dev)
@@ -419,9 +421,10 @@ def test_validate_payload_flags_corruption():
     p = c.payloads[0].clone()
     p[first] = 0xFF; p[first + 1] = 0xFF  # index 0xFFF first, then a smaller one: not ascending
     corruptions.append(p)
-    p = c.payloads[0].clone()
-    p[first + stride - 1] = 1  # padding must be zero
-    corruptions.append(p)
+    if (12 * k + 7) // 8 + (bits * k + 7) // 8 < stride:   # (some k fill the stride exactly: no padding to spoil)
+        p = c.payloads[0].clone()
+        p[first + stride - 1] = 1  # padding must be zero
+        corruptions.append(p)
     p = c.payloads[0].clone()
     p[0:4] = torch.tensor(np.frombuffer(np.float32(np.inf).tobytes(), np.uint8).copy())  # table not finite
     corruptions.append(p)
@@ -429,6 +432,10 @@ def test_validate_payload_flags_corruption():
     tiny_rec = c.rec_off[4]  # the 40-element tensor: slots >= 40 must be zero
     p[tiny_rec + (12 * 40) // 8 + 1] = 0x10
     corruptions.append(p)
+    if bits == 1:  # a 1-bit table is 8 bytes of a 16-byte header: the rest must be zero
+        p = c.payloads[0].clone()
+        p[12] = 1
+        corruptions.append(p)
     for bad in corruptions:
         c.sl.validate_payload(bad, status)
         torch.cuda.synchronize()

@@ -202,7 +202,7 @@ def test_quantiser_widths_of_the_ablation(bits, k):
         rms = float(np.sqrt(np.mean(th.astype(np.float64) ** 2)))
         assert float(np.max(np.abs(got.astype(np.float64) - th.astype(np.float64)))) <= 1e-6 * rms
     from paper_2508_15706_b200 import binding as B
-    with pytest.raises(B.SlError) as ei:     # the wire codec, the validator and deferral serve the 2-bit payload only
+    with pytest.raises(B.SlError) as ei:     # the wire codec and deferral serve the 2-bit payload only
         c.sl.coded_payload_capacity()
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
     with pytest.raises(B.SlError):
@@ -227,7 +227,7 @@ def test_densities_up_to_half_a_chunk(bits, k):
         rep = c.check(snap)
         assert rep["tensors"] == len(tensors)
     from paper_2508_15706_b200 import binding as B
-    with pytest.raises(B.SlError) as ei:     # deferral, the wire codec and the validator stop at k = 256
+    with pytest.raises(B.SlError) as ei:     # deferral and the wire codec stop at k = 256
         c.sl.set_ef_deferred(True)
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
     with pytest.raises(B.SlError) as ei:     # and so does the path without a quantiser
