@@ -97,3 +97,27 @@ def test_config5_dense_d2048_as_benchmarked():
         for j in ids[:2]:
             assert np.array_equal(got[r][j].view(np.uint32), want[r][j].view(np.uint32))
     assert c.guards_intact()
+
+
+def test_repeated_runs_leave_identical_bits():
+    """The same three steps from the same state on two independent sets of buffers: theta, every error
+    buffer, every payload and the values waiting in the workspace must agree bit for bit, whatever the
+    scheduling of warps and CTAs was (the ordered additions of Eq. 2 line 3, the deterministic candidate
+    lists and tie rule of the selection).  Run on the 162 M-parameter config, where every kernel spans
+    many waves."""
+    wl = I.workload("c2_dense_d768")
+    a = _case(wl, e_scale=0.5)
+    b = _case(wl, e_scale=0.5)
+    for step in range(3):
+        a.fill_local(step)
+        b.fill_local(step)
+        a.step()
+        b.step()
+        torch.cuda.synchronize()
+        assert torch.equal(a.theta.view(torch.int32), b.theta.view(torch.int32)), step
+        for r in range(wl.R):
+            assert torch.equal(a.payloads[r], b.payloads[r]), (step, r)
+            assert torch.equal(a.e[r].view(torch.int32), b.e[r].view(torch.int32)), (step, r)
+    ea, eb = a.true_error(), b.true_error()
+    for r in range(wl.R):
+        assert torch.equal(ea[r].view(torch.int32), eb[r].view(torch.int32)), r
