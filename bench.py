@@ -540,7 +540,7 @@ def measured_peak_gbs():
         ("measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s")
 
 
-def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int = 8) -> dict:
+def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int = 8, only: str = "") -> dict:
     """The settings outside the paper's main configuration (quantiser widths of its ablation, no quantiser,
     densities up to half a chunk, bfloat16 storage) on the 12-layer stack with R = 8: ms per outer step and
     the rate on the state the step must stream ((12 R + 8) bytes per parameter in fp32, half in bfloat16:
@@ -550,9 +550,6 @@ def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int =
     base = dataclasses.replace(I.workload(workload), R=R)
     N = base.numel
     shapes, offs = [(t.rows, t.cols) for t in base.tensors], I.offsets(base.tensors)
-    theta32 = I.theta_sync(base, dev)
-    local32 = [I.theta_local(base, theta32, r, 0) for r in range(R)]
-    e32 = [I.initial_error(base, r, dev, scale=0.5) for r in range(R)]
     stream = torch.cuda.current_stream()
     cases = [("quant_bits=2 k=64 (the tuned path, materialised subtraction)", 2, 64, False),
              ("quant_bits=1 k=64", 1, 64, False), ("quant_bits=3 k=64", 3, 64, False), ("quant_bits=4 k=64", 4, 64, False),
@@ -560,11 +557,24 @@ def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int =
              ("quant_bits=2 k=512", 2, 512, False), ("quant_bits=2 k=2048", 2, 2048, False),
              ("bf16 storage, quant_bits=2 k=64", 2, 64, True)]
     out = {"workload": workload, "params": N, "R": R}
+    cases = [c for c in cases if only in c[0]]
+    if all(c[3] for c in cases):
+        # bfloat16 cases alone (a workload whose fp32 state would not fit): build the state buffer by buffer
+        theta32 = I.theta_sync(base, dev)
+        local32 = e32 = None
+    else:
+        theta32 = I.theta_sync(base, dev)
+        local32 = [I.theta_local(base, theta32, r, 0) for r in range(R)]
+        e32 = [I.initial_error(base, r, dev, scale=0.5) for r in range(R)]
     for name, bits, k, half in cases:
         sl = SparseLoCo(shapes, offs, k=k, R=R, beta=base.beta, outer_lr=base.outer_lr, quant_bits=bits,
                         bf16_storage=half)
         pay = [torch.zeros(sl.payload_bytes() if bits != 32 else 16, dtype=torch.uint8, device=dev) for _ in range(R)]
-        if half:
+        if half and local32 is None:
+            theta = theta32.to(torch.bfloat16)
+            local = [I.theta_local(base, theta32, r, 0).to(torch.bfloat16) for r in range(R)]
+            e = [I.initial_error(base, r, dev, scale=0.5).to(torch.bfloat16) for r in range(R)]
+        elif half:
             theta = theta32.to(torch.bfloat16)
             local = [x.to(torch.bfloat16) for x in local32]
             e = [x.to(torch.bfloat16) for x in e32]
@@ -811,8 +821,10 @@ def main():
     ap.add_argument("--codec", action="store_true", help="also time the entropy-coded index format on one payload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--options-only", action="store_true",
-                    help="time only the settings outside the main configuration (options_bench) on --workload")
+                    help="time only the settings outside the main configuration (options_bench) on --options-workload")
+    ap.add_argument("--options-workload", default="c5_l12")
     ap.add_argument("--options-workers", type=int, default=8)
+    ap.add_argument("--options-filter", default="", help="run only the options cases whose name contains this")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--reference-budget", type=float, default=150.0, help="seconds for the whole reference run")
     args = ap.parse_args()
@@ -826,8 +838,8 @@ def main():
         from paper_2508_15706_b200 import inputs as I
         torch.cuda.set_device(0)
         out = options_bench(torch, I, torch.device("cuda", 0), measured_peak_gbs()[0],
-                            workload=args.workload if args.workload != DEFAULT_WORKLOAD else "c5_l12",
-                            R=args.options_workers)
+                            workload=args.options_workload,
+                            R=args.options_workers, only=args.options_filter)
     elif args.mode == "worker-per-gpu":
         out = run_worker_per_gpu(args)
     else:
