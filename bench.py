@@ -555,7 +555,9 @@ def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int =
              ("quant_bits=1 k=64", 1, 64, False), ("quant_bits=3 k=64", 3, 64, False), ("quant_bits=4 k=64", 4, 64, False),
              ("quant_bits=32 k=64 (no quantiser)", 32, 64, False),
              ("quant_bits=2 k=512", 2, 512, False), ("quant_bits=2 k=2048", 2, 2048, False),
-             ("bf16 storage, quant_bits=2 k=64", 2, 64, True)]
+             ("bf16 storage, quant_bits=2 k=64", 2, 64, True),
+             ("bf16 storage, quant_bits=2 k=64, deferred subtraction (one flush in the timed region)", 2, 64, True),
+             ("quant_bits=2 k=64, deferred subtraction (the headline's mode; one flush in the timed region)", 2, 64, False)]
     out = {"workload": workload, "params": N, "R": R}
     cases = [c for c in cases if only in c[0]]
     if all(c[3] for c in cases):
@@ -580,15 +582,21 @@ def options_bench(torch, I, dev, peak: float, workload: str = "c5_l12", R: int =
             e = [x.to(torch.bfloat16) for x in e32]
         else:
             theta, local, e = theta32.clone(), local32, [x.clone() for x in e32]
+        deferred = "deferred" in name
+        if deferred:
+            sl.set_ef_deferred(True)
+        reps = 5 if deferred else 3
         for _ in range(2):
             sl.outer_step(theta, local, e, pay)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
-        for _ in range(3):
+        for _ in range(reps):
             sl.outer_step(theta, local, e, pay)
+        if deferred:
+            sl.ef_flush()
         b.record(stream)
         torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / 3
+        ms = a.elapsed_time(b) / reps
         bpp = (12 * R + 8) * (0.5 if half else 1.0)
         out[name] = {"ms_per_step": ms, "state_bytes_per_param": bpp, "gbs": bpp * N / (ms * 1e-3) / 1e9,
                      "frac_of_measured_peak": bpp * N / (ms * 1e-3) / 1e9 / peak}

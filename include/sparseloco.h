@@ -160,7 +160,13 @@ sl_status sl_outer_step(sl_ctx* ctx, float* theta_sync, const float* const* thet
  * fp32 calls would write for these inputs -- and every store rounds once to the nearest bfloat16,
  * ties to even: e = bf16(u), or bf16(u - table[code]) at the selected positions;
  * theta = bf16(fma(-alpha / D, sum, theta)) where some worker selected the element, else unchanged.
- * Plain kernels (no tile copies, no fusion, no deferral); any k up to 2048 and quant_bits 1..4.
+ * At 2 bits and k <= 256 the quantiser statistics and the fused packing / update kernel are the tuned ones
+ * of the fp32 path (with widening loads and rounding stores), the deferred subtraction is available
+ * (sl_set_ef_deferred; the waiting values stay fp32 in the workspace and are rounded when they reach e;
+ * sl_ef_flush_bf16 for explicit buffers) and so are the wire codec, sl_validate_payload and sl_read_stats;
+ * the selection runs in a warp-per-unit kernel with plain loads (no tile copies).  Other widths and
+ * larger k run in the plain kernels.  Not available: sl_outer_step_host, sl_aggregate_apply_coded, the
+ * comparison methods, quant_bits = 32.
  * Errors as for the fp32 calls; UNSUPPORTED when the context is not a bf16_storage one (and the
  * fp32 calls return UNSUPPORTED for a context that is). */
 sl_status sl_compress_bf16(sl_ctx* ctx, const uint16_t* theta_sync, const uint16_t* theta_local, uint16_t* e,
@@ -169,6 +175,7 @@ sl_status sl_aggregate_apply_bf16(sl_ctx* ctx, const uint8_t* const* payloads, u
                                   void* cuda_stream);
 sl_status sl_outer_step_bf16(sl_ctx* ctx, uint16_t* theta_sync, const uint16_t* const* theta_local,
                              uint16_t* const* e, uint8_t* const* payloads, void* cuda_stream);
+sl_status sl_ef_flush_bf16(sl_ctx* ctx, uint16_t* const* e, int32_t keep_pending, void* cuda_stream);
 
 /* Dense baseline on the same buffers: DiLoCo's outer step with Nesterov outer momentum (Eq. 1),
  *     Dbar = (1/R) sum_r (theta - theta_r);  m = beta_outer m + Dbar;

@@ -20,7 +20,7 @@ EXPORTS = (
     "sl_flat_elems", "sl_workspace_bytes", "sl_set_workspace", "sl_compress", "sl_aggregate_apply",
     "sl_outer_step", "sl_outer_step_host", "sl_validate_payload", "sl_read_stats", "sl_strerror",
     "sl_last_cuda_error", "sl_diloco_step", "sl_coded_payload_capacity", "sl_encode_payload", "sl_decode_payload", "sl_set_tile_copies", "sl_device_status", "sl_static_scratch_bytes", "sl_compress_tensor_static", "sl_set_ef_deferred", "sl_ef_pending", "sl_ef_flush", "sl_profile_enable", "sl_profile_read", "sl_profile_name", "sl_lom_step", "sl_diloco_topk_step", "sl_lom_topk_step", "sl_streaming_due",
-    "sl_compress_bf16", "sl_aggregate_apply_bf16", "sl_outer_step_bf16", "sl_aggregate_apply_coded",
+    "sl_compress_bf16", "sl_aggregate_apply_bf16", "sl_outer_step_bf16", "sl_aggregate_apply_coded", "sl_ef_flush_bf16",
 )
 PROFILE_SLOTS = 9
 
@@ -67,6 +67,7 @@ def _load():
     L.sl_aggregate_apply.argtypes = [P, P, P, P]
     L.sl_outer_step.argtypes = [P, P, P, P, P, P]
     L.sl_compress_bf16.argtypes = [P, P, P, P, P, P]
+    L.sl_ef_flush_bf16.argtypes = [P, P, C.c_int32, P]
     L.sl_aggregate_apply_coded.argtypes = [P, P, P, P, P]
     L.sl_aggregate_apply_bf16.argtypes = [P, P, P, P]
     L.sl_outer_step_bf16.argtypes = [P, P, P, P, P, P]
@@ -324,7 +325,7 @@ class SparseLoCo:
         sizes = (C.c_size_t * len(coded))()
         for r, p in enumerate(coded):
             sizes[r] = 0 if p is None else int(coded_bytes[r] if coded_bytes is not None and coded_bytes[r] else p.numel())
-        _check(_L.sl_aggregate_apply_coded(self._h, arr, sizes, _dev_ptr(theta_sync, torch.float32), _stream()))
+        _check(_L.sl_aggregate_apply_coded(self._h, arr, sizes, _dev_ptr(theta_sync, self.dtype), _stream()))
 
     def set_tile_copies(self, use_tensor_maps: bool) -> None:
         _check(_L.sl_set_tile_copies(self._h, int(use_tensor_maps)))
@@ -342,8 +343,9 @@ class SparseLoCo:
         return bool(v.value)
 
     def ef_flush(self, e: Optional[List[torch.Tensor]] = None, keep_pending: bool = False) -> None:
-        ea = _ptr_array([_dev_ptr(t, torch.float32) if t is not None else None for t in e]) if e is not None else None
-        _check(_L.sl_ef_flush(self._h, ea, int(keep_pending), _stream()))
+        ea = _ptr_array([_dev_ptr(t, self.dtype) if t is not None else None for t in e]) if e is not None else None
+        fn = _L.sl_ef_flush_bf16 if self.dtype == torch.bfloat16 else _L.sl_ef_flush
+        _check(fn(self._h, ea, int(keep_pending), _stream()))
 
     def profile_enable(self, on: bool = True) -> None:
         _check(_L.sl_profile_enable(self._h, int(on)))

@@ -76,12 +76,18 @@ __device__ __forceinline__ void async_copy16(void* smem_dst, const void* gmem_sr
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void async_copy8(void* smem_dst, const void* gmem_src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void async_copy_wait_all() {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
 }
 
 // PPL = slot pairs per lane: ceil(k / 64) rounded up to 1, 2 or 4
-template <int PPL, int FUSE>
+// HALF (FUSE 0-2): theta and the error buffers are bfloat16 arrays; they are widened on the way in and what is
+// stored is rounded once to nearest-even, the arithmetic in between is the fp32 arithmetic of the fp32 form.
+template <int PPL, int FUSE, bool HALF = false>
 __global__ void __launch_bounds__(kApplyThreads, kApplyCtasPerSm)
 decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, float scale,
                         PayloadPtrs pl, float* __restrict__ theta_sync, FuseArgs fa, WorkerPtrs ptrs) {
@@ -118,11 +124,19 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     __syncthreads();
 
     // thread t owns in-chunk indices 512 i + 4 t + j: block row 8 i + t / 16, column 4 (t % 16)
+    bf16_bits* const theta_h = reinterpret_cast<bf16_bits*>(theta_sync);  // HALF: the same array seen as bfloat16
+    uint2* const stage_h = reinterpret_cast<uint2*>(stage);                 // HALF: four bfloat16 per vector
     auto prefetch_theta = [&](const ChunkDesc& d) {
         const int prs = d.row_stride ? d.row_stride : kTile;
-        const float* src = theta_sync + d.base + (long long)(tid >> 4) * prs + 4 * (tid & 15);
+        if (HALF) {
+            const bf16_bits* src = theta_h + d.base + (long long)(tid >> 4) * prs + 4 * (tid & 15);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) async_copy16(&stage[128 * i + tid], src + (long long)i * 8 * prs);
+            for (int i = 0; i < 8; ++i) async_copy8(&stage_h[128 * i + tid], src + (long long)i * 8 * prs);
+        } else {
+            const float* src = theta_sync + d.base + (long long)(tid >> 4) * prs + 4 * (tid & 15);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) async_copy16(&stage[128 * i + tid], src + (long long)i * 8 * prs);
+        }
     };
     ChunkDesc cd_next;
     if (g_first < n_chunks) {
@@ -142,7 +156,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
         async_copy_wait_all();  // (this thread's copies; nothing is outstanding after a short chunk)
         if (full) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a[i] = stage[128 * i + tid];
+            for (int i = 0; i < 8; ++i) a[i] = HALF ? bf16_widen4(stage_h[128 * i + tid]) : stage[128 * i + tid];
         }
         if (next_of(g) < n_chunks) {  // the block is free again (this thread's part of it): the next chunk's theta
             cd_next = chunks[next_of(g)];
@@ -323,7 +337,11 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     const float l1 = RAW ? val[q][j].y : c1 == 0 ? lut.x : c1 == 1 ? lut.y : c1 == 2 ? lut.z : lut.w;
                     if (PACK) {
                         const float f0 = __fsub_rn(val[q][j].x, l0), f1 = __fsub_rn(val[q][j].y, l1);
-                        if (FUSE == 1) {
+                        if (FUSE == 1 && HALF) {
+                            bf16_bits* eh = reinterpret_cast<bf16_bits*>(ptrs.e[r]) + cd.base;
+                            if (ok0 && p0 < (unsigned)cd.len) eh[chunk_elem_offset(cd.row_stride, (int)p0)] = (bf16_bits)bf16_narrow(f0);
+                            if (ok1 && p1 < (unsigned)cd.len) eh[chunk_elem_offset(cd.row_stride, (int)p1)] = (bf16_bits)bf16_narrow(f1);
+                        } else if (FUSE == 1) {
                             if (ok0 && p0 < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p0)] = f0;
                             if (ok1 && p1 < (unsigned)cd.len) ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p1)] = f1;
                         } else if (ok0) {
@@ -420,13 +438,21 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     o.y = __fmaf_rn(scale, sv.y, a[i].y);
                     o.z = __fmaf_rn(scale, sv.z, a[i].z);
                     o.w = __fmaf_rn(scale, sv.w, a[i].w);
-                    *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
+                    if (HALF)  // (an element that received nothing keeps its bits: fma(scale, +0, x) = x, and x is a bfloat16)
+                        bf16_store4(theta_h + cd.base + (long long)(tid >> 4) * rs + 4 * (tid & 15) + i * vec_step, o);
+                    else
+                        *reinterpret_cast<float4*>(th_vec + i * vec_step) = o;
                     *reinterpret_cast<float4*>(av) = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
         } else {
             for (int p = tid; p < cd.len; p += kApplyThreads) {  // (nothing was added at or beyond the chunk's length)
-                th[p] = __fmaf_rn(scale, acc[p], th[p]);
+                if (HALF) {
+                    bf16_bits* thh = theta_h + cd.base;
+                    thh[p] = (bf16_bits)bf16_narrow(__fmaf_rn(scale, acc[p], bf16_widen(thh[p])));
+                } else {
+                    th[p] = __fmaf_rn(scale, acc[p], th[p]);
+                }
                 acc[p] = 0.0f;
             }
         }

@@ -1,7 +1,6 @@
 // bfloat16 storage of theta, theta_r and e: the selection kernel and the store helpers of that mode.
 // Part of libsparseloco (one translation unit: included by sparseloco.cu).
 #pragma once
-#include <cuda_bf16.h>
 #include "common.cuh"
 #include "ef_select.cuh"
 
@@ -20,22 +19,6 @@
 // ================================================================================================
 namespace {
 
-typedef unsigned short bf16_bits;
-
-__device__ __forceinline__ float bf16_widen(unsigned b) { return __uint_as_float(b << 16); }
-__device__ __forceinline__ unsigned bf16_narrow(float x) { return (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
-
-__device__ __forceinline__ float4 bf16_load4(const bf16_bits* p) {
-    const uint2 w = *reinterpret_cast<const uint2*>(p);
-    return make_float4(bf16_widen(w.x & 0xFFFFu), bf16_widen(w.x >> 16), bf16_widen(w.y & 0xFFFFu), bf16_widen(w.y >> 16));
-}
-__device__ __forceinline__ void bf16_store4(bf16_bits* p, const float4& x) {
-    uint2 w;
-    w.x = bf16_narrow(x.x) | (bf16_narrow(x.y) << 16);
-    w.y = bf16_narrow(x.z) | (bf16_narrow(x.w) << 16);
-    *reinterpret_cast<uint2*>(p) = w;
-}
-
 constexpr int kHalfSelWarps = 12;  // what shared memory (16 KB of u per warp) and the register file allow
 constexpr int kHalfSelThreads = 32 * kHalfSelWarps;
 struct HalfSelSmem {
@@ -46,7 +29,9 @@ struct HalfSelSmem {
 
 // One warp per (chunk, worker) unit, units taken chunk-major so that the workers of a chunk follow one
 // another (theta's block is re-read from L2).  The WorkerPtrs / theta pointers address bfloat16 arrays.
-template <bool EF, int WIDE>
+// PENDING: the corrected values of the previous step still wait in the staging arrays (deferred subtraction):
+// they are rounded into the error buffer at their positions before the unit's e is read.
+template <bool EF, int WIDE, bool PENDING = false>
 __global__ void __launch_bounds__(kHalfSelThreads, 1)
 ef_select_bf16_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, float beta,
                       const bf16_bits* __restrict__ theta_sync, WorkerPtrs ptrs, Workspace ws) {
@@ -65,6 +50,14 @@ ef_select_bf16_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, 
         const bf16_bits* __restrict__ tlp = reinterpret_cast<const bf16_bits*>(ptrs.theta_local[r]) + cd.base;
         bf16_bits* __restrict__ er = EF ? reinterpret_cast<bf16_bits*>(ptrs.e[r]) + cd.base : nullptr;
         *reinterpret_cast<uint4*>(&bitmap[4 * lane]) = make_uint4(0u, 0u, 0u, 0u);
+        const long long slot_base = ((long long)r * n_chunks + g) * kp;
+        if (PENDING && EF) {  // (the lanes' plain loads below read what is patched here)
+            for (int j = lane; j < keff; j += 32) {
+                const unsigned p = ws.idx[slot_base + j];
+                if (p < (unsigned)cd.len) er[chunk_elem_offset(cd.row_stride, (int)p)] = (bf16_bits)bf16_narrow(ws.val[slot_base + j]);
+            }
+            __syncwarp();
+        }
         float u[128];
         if (cd.len == kChunk) {
             // a full chunk: the loads of 8 vectors per array are issued before any of them is used (the stores
@@ -145,7 +138,6 @@ ef_select_bf16_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, 
         USource src;
         src.ptr = reinterpret_cast<const unsigned*>(scratch);
         src.rs = kTile;
-        const long long slot_base = ((long long)r * n_chunks + g) * kp;
         select_unit<false, WIDE>(u, src, cd.len, keff, bitmap, sm.cand[warp], ws.idx + slot_base, ws.val + slot_base);
         __syncwarp();  // the block, the map and the list are free again
     }

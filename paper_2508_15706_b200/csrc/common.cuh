@@ -1,6 +1,7 @@
 // Constants, the chunk table and workspace layouts, small helpers shared by all kernels.
 // Part of libsparseloco (one translation unit: included by sparseloco.cu).
 #pragma once
+#include <cuda_bf16.h>
 
 namespace {
 
@@ -64,6 +65,22 @@ __host__ __device__ constexpr int record_index_bytes(int k) { return (12 * k + 7
 __host__ __device__ constexpr int record_stride(int k) {
     return (record_index_bytes(k) + (2 * k + 7) / 8 + 15) / 16 * 16;
 }
+
+// bfloat16 storage (the upper half of an fp32): widening is exact, narrowing rounds to nearest-even.
+typedef unsigned short bf16_bits;
+__device__ __forceinline__ float bf16_widen(unsigned b) { return __uint_as_float(b << 16); }
+__device__ __forceinline__ unsigned bf16_narrow(float x) { return (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float4 bf16_widen4(const uint2& w) {
+    return make_float4(bf16_widen(w.x & 0xFFFFu), bf16_widen(w.x >> 16), bf16_widen(w.y & 0xFFFFu), bf16_widen(w.y >> 16));
+}
+__device__ __forceinline__ uint2 bf16_narrow4(const float4& x) {
+    uint2 w;
+    w.x = bf16_narrow(x.x) | (bf16_narrow(x.y) << 16);
+    w.y = bf16_narrow(x.z) | (bf16_narrow(x.w) << 16);
+    return w;
+}
+__device__ __forceinline__ float4 bf16_load4(const bf16_bits* p) { return bf16_widen4(*reinterpret_cast<const uint2*>(p)); }
+__device__ __forceinline__ void bf16_store4(bf16_bits* p, const float4& x) { *reinterpret_cast<uint2*>(p) = bf16_narrow4(x); }
 
 // Element offset (relative to ChunkDesc::base) of in-chunk index p.
 __device__ __forceinline__ long long chunk_elem_offset(int row_stride, int p) {

@@ -13,7 +13,8 @@ namespace {
 // ------------------------------------------------------------------------------------------------
 // MODE 0: records only (error feedback frozen).  MODE 1: e[index] = value - table[code].
 // MODE 2: the corrected value replaces the staged value instead (deferred subtraction).
-template <int MODE>
+// HALF: the error buffers are bfloat16 arrays (MODE 1 rounds the corrected value to nearest-even on the store).
+template <int MODE, bool HALF = false>
 __global__ void __launch_bounds__(128)
 pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int n_tensors,
                 int k, int kp, Workspace ws, WorkerPtrs ptrs) {
@@ -42,8 +43,10 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
         const int cbit = code_word0 * 8 + 2 * s;
         atomicOr(&rec[warp][cbit >> 5], (unsigned)c << (cbit & 31));
         if (MODE == 1 && p < (unsigned)cd.len) {
-            float* er = ptrs.e[r] + cd.base + chunk_elem_offset(cd.row_stride, (int)p);
-            *er = __fsub_rn(v, st.lut[c]);
+            const long long at = cd.base + chunk_elem_offset(cd.row_stride, (int)p);
+            const float fix = __fsub_rn(v, st.lut[c]);
+            if (HALF) reinterpret_cast<bf16_bits*>(ptrs.e[r])[at] = (bf16_bits)bf16_narrow(fix);
+            else ptrs.e[r][at] = fix;
         }
         if (MODE == 2) ws.val[slot_base + s] = __fsub_rn(v, st.lut[c]);
     }
@@ -57,7 +60,7 @@ pack_fix_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
 // subtraction made good).  One warp per (worker, chunk).  ZERO: writes +0 at the staged positions
 // instead (Top-k without a quantiser sends the selected values exactly, so what stays behind there,
 // u - Top-k(u), is zero: Alg. 2-4 of the appendix on DiLoCo variants).
-template <bool ZERO>
+template <bool ZERO, bool HALF = false>
 __global__ void __launch_bounds__(128)
 ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, int kp, Workspace ws,
                 WorkerPtrs ptrs) {
@@ -72,8 +75,12 @@ ef_flush_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_
     const long long slot_base = ((long long)r * n_chunks + g) * kp;
     for (int s = lane; s < keff; s += 32) {
         const unsigned p = ws.idx[slot_base + s];
-        if (p < (unsigned)cd.len)
-            ptrs.e[r][cd.base + chunk_elem_offset(cd.row_stride, (int)p)] = ZERO ? 0.0f : ws.val[slot_base + s];
+        if (p < (unsigned)cd.len) {
+            const long long at = cd.base + chunk_elem_offset(cd.row_stride, (int)p);
+            const float v = ZERO ? 0.0f : ws.val[slot_base + s];
+            if (HALF) reinterpret_cast<bf16_bits*>(ptrs.e[r])[at] = (bf16_bits)bf16_narrow(v);
+            else ptrs.e[r][at] = v;
+        }
     }
 }
 

@@ -131,12 +131,12 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // general-width quantiser (quant_bits 1, 3, 4): its per-unit bin partials and per-tensor tables follow
 // the arrays of the 2-bit path in the workspace
 // (also the 2-bit quantiser at k > 256, which the fused kernels are not laid out for)
-// (and everything under bfloat16 storage)
 inline bool half_store(const sl_ctx* c) { return c->cfg.bf16_storage != 0; }
 inline bool wide_quant(const sl_ctx* c) {
-    return c->cfg.quant_bits != 32 && (c->cfg.quant_bits != 2 || c->cfg.k > kFastMaxK || half_store(c));
+    return c->cfg.quant_bits != 32 && (c->cfg.quant_bits != 2 || c->cfg.k > kFastMaxK);
 }
-inline bool fast_2bit(const sl_ctx* c) { return c->cfg.quant_bits == 2 && c->cfg.k <= kFastMaxK && !half_store(c); }
+// the paper's setting (2 bits, k <= 256): the tuned kernels, the deferred subtraction, the wire codec; fp32 or bfloat16 arrays
+inline bool fast_2bit(const sl_ctx* c) { return c->cfg.quant_bits == 2 && c->cfg.k <= kFastMaxK; }
 size_t wide_bytes_for(const sl_ctx* c, int workers) {
     if (!wide_quant(c)) return 0;
     const size_t WG = (size_t)workers * (size_t)c->n_chunks, nb = (size_t)1 << c->qbits;
@@ -244,8 +244,12 @@ sl_status order_after_map_uploads(sl_ctx* c, cudaStream_t st) {
 sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
     const int R = c->cfg.R;
     const Workspace ws = carve(c, R);
-    ef_flush_kernel<false><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
-                                                                           ws, ptrs);
+    if (half_store(c))
+        ef_flush_kernel<false, true><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k,
+                                                                                     c->kp, ws, ptrs);
+    else
+        ef_flush_kernel<false><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, c->kp,
+                                                                               ws, ptrs);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
@@ -282,7 +286,7 @@ sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const W
     const long long G = c->n_chunks;
     const int k = c->cfg.k, kp = c->kp;
     if (half_store(c)) {  // bfloat16 arrays: the warp-per-unit kernel with plain loads
-        if (consume || delta) return SL_ERR_UNSUPPORTED;
+        if (delta || (consume && k > kFastMaxK)) return SL_ERR_UNSUPPORTED;
         const long long units = G * workers;
         const long long want = (units + kHalfSelWarps - 1) / kHalfSelWarps;
         const unsigned grid = (unsigned)(want < c->n_sms ? (want < 1 ? 1 : want) : c->n_sms);
@@ -299,7 +303,14 @@ sl_status launch_select(sl_ctx* c, int workers, const float* theta_sync, const W
             ef_select_bf16_kernel<EFV, 0><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(                     \
                 c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);                                        \
     } while (0)
-        if (ef) SL_LAUNCH_HALF(true);
+        if (ef && consume) {
+            if (k > kSelNarrowMaxK)
+                ef_select_bf16_kernel<true, 1, true><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(
+                    c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);
+            else
+                ef_select_bf16_kernel<true, 0, true><<<grid, kHalfSelThreads, sizeof(HalfSelSmem), st>>>(
+                    c->d_chunks, G, workers, k, kp, c->cfg.beta, ts, ptrs, ws);
+        } else if (ef) SL_LAUNCH_HALF(true);
         else SL_LAUNCH_HALF(false);
 #undef SL_LAUNCH_HALF
         SL_CUDA(cudaGetLastError());
@@ -444,6 +455,8 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
         pack_fix_kernel<0><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     else if (defer)
         pack_fix_kernel<2><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
+    else if (half_store(c))
+        pack_fix_kernel<1, true><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     else
         pack_fix_kernel<1><<<pb, 128, 0, st>>>(c->d_chunks, G, workers, T, k, kp, ws, ptrs);
     prof_mark(c, 7, st);
@@ -504,6 +517,23 @@ sl_status launch_apply(sl_ctx* c, const PayloadPtrs& pl, int present, float* the
     const long long fit = (227ll * 1024) / ((long long)smem + 1024);
     const long long resident = (long long)c->n_sms * (fit < kApplyCtasPerSm ? (fit < 1 ? 1 : fit) : kApplyCtasPerSm);
     const unsigned grid = (unsigned)(c->n_chunks < resident ? c->n_chunks : resident);
+#define SL_APPLY_H(PPLV)                                                                                        \
+    do {                                                                                                        \
+        auto kern = fuse == 0 ? decode_avg_apply_kernel<PPLV, 0, true>                                          \
+                  : fuse == 1 ? decode_avg_apply_kernel<PPLV, 1, true> : decode_avg_apply_kernel<PPLV, 2, true>; \
+        kern<<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp); \
+    } while (0)
+    if (half_store(c)) {
+        if (fuse > 2) return SL_ERR_UNSUPPORTED;
+        if (ppl <= 1) SL_APPLY_H(1);
+        else if (ppl <= 2) SL_APPLY_H(2);
+        else SL_APPLY_H(4);
+        prof_mark(c, 8, st);
+        if (c->prof_on && c->prof_steps < kProfMaxSeq) c->prof_steps++;
+        SL_CUDA(cudaGetLastError());
+        return SL_OK;
+    }
+#undef SL_APPLY_H
 #define SL_APPLY(PPLV)                                                                                          \
     do {                                                                                                        \
         auto kern = fuse == 0 ? decode_avg_apply_kernel<PPLV, 0>                                                \
@@ -749,6 +779,12 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
                                  (int)sizeof(HalfSelSmem))
     SL_HALF_ATTR(true, 0); SL_HALF_ATTR(false, 0); SL_HALF_ATTR(true, 1); SL_HALF_ATTR(false, 1);
     SL_HALF_ATTR(true, 2); SL_HALF_ATTR(false, 2);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_select_bf16_kernel<true, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(HalfSelSmem));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ef_select_bf16_kernel<true, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(HalfSelSmem));
 #undef SL_HALF_ATTR
     per_sm = 1;
     {   // the apply kernel's shared memory grows with k (and, for coded payloads, with R): the limit is a property of
@@ -761,6 +797,13 @@ sl_status sl_create(const sl_config* cfg, const sl_tensor_desc* tensors, int32_t
         SL_APPLY_ATTR(2, 0); SL_APPLY_ATTR(2, 1); SL_APPLY_ATTR(2, 2); SL_APPLY_ATTR(2, 3); SL_APPLY_ATTR(2, 4);
         SL_APPLY_ATTR(4, 0); SL_APPLY_ATTR(4, 1); SL_APPLY_ATTR(4, 2); SL_APPLY_ATTR(4, 3); SL_APPLY_ATTR(4, 4);
         SL_APPLY_ATTR(1, 5); SL_APPLY_ATTR(2, 5); SL_APPLY_ATTR(4, 5);
+#define SL_APPLY_ATTR_H(PPLV, FUSEV)                                                                                   \
+    if (e == cudaSuccess)                                                                                              \
+        e = cudaFuncSetAttribute(decode_avg_apply_kernel<PPLV, FUSEV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, asz)
+        SL_APPLY_ATTR_H(1, 0); SL_APPLY_ATTR_H(1, 1); SL_APPLY_ATTR_H(1, 2);
+        SL_APPLY_ATTR_H(2, 0); SL_APPLY_ATTR_H(2, 1); SL_APPLY_ATTR_H(2, 2);
+        SL_APPLY_ATTR_H(4, 0); SL_APPLY_ATTR_H(4, 1); SL_APPLY_ATTR_H(4, 2);
+#undef SL_APPLY_ATTR_H
 #undef SL_APPLY_ATTR
     }
     c->n_sms = n_sms;
@@ -860,6 +903,7 @@ sl_status do_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
 sl_status do_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream);
 sl_status do_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_local, float* const* e,
                         uint8_t* const* payloads, void* stream);
+sl_status do_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* stream);
 }  // namespace
 
 // The fp32 entry points refuse a context made for bfloat16 storage and the other way round: the element
@@ -1308,7 +1352,7 @@ sl_status sl_decode_payload(sl_ctx* c, const uint8_t* coded, size_t coded_bytes,
 sl_status sl_aggregate_apply_coded(sl_ctx* c, const uint8_t* const* coded, const size_t* coded_bytes, float* theta_sync,
                                    void* stream) {
     if (!c || !coded || !theta_sync) return SL_ERR_INVALID_ARG;
-    if (!fast_2bit(c)) return SL_ERR_UNSUPPORTED;  // a format of the 2-bit payload only
+    if (!fast_2bit(c) || half_store(c)) return SL_ERR_UNSUPPORTED;  // the 2-bit payload, fp32 arrays
     if (!c->ixc_capacity) return SL_ERR_TOO_LARGE;
     if (misaligned(theta_sync)) return SL_ERR_ALIGNMENT;
     PayloadPtrs pl;
@@ -1361,7 +1405,18 @@ sl_status sl_ef_pending(const sl_ctx* c, int32_t* pending) {
     return SL_OK;
 }
 
+sl_status sl_ef_flush_bf16(sl_ctx* c, uint16_t* const* e, int32_t keep_pending, void* stream) {
+    if (c && !half_store(c)) return SL_ERR_UNSUPPORTED;
+    return do_ef_flush(c, reinterpret_cast<float* const*>(e), keep_pending, stream);
+}
+
 sl_status sl_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* stream) {
+    if (c && half_store(c) && e) return SL_ERR_UNSUPPORTED;  // (with e = NULL the call is type-free)
+    return do_ef_flush(c, e, keep_pending, stream);
+}
+
+namespace {
+sl_status do_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* stream) {
     if (!c) return SL_ERR_INVALID_ARG;
     if (!c->pending) return SL_OK;
     WorkerPtrs ptrs;
@@ -1379,6 +1434,7 @@ sl_status sl_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* st
     if (!keep_pending) c->pending = false;
     return SL_OK;
 }
+}  // namespace
 
 sl_status sl_streaming_due(int32_t H, int32_t P, int64_t inner_step, int32_t* fragment) {
     if (!fragment || H < 1 || P < 1 || P > H || inner_step < 1) return SL_ERR_INVALID_ARG;

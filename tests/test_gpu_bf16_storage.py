@@ -29,8 +29,10 @@ def _widen(t: torch.Tensor) -> np.ndarray:
     return t.to(torch.float32).cpu().numpy()
 
 
-@pytest.mark.parametrize("bits,k,R", [(2, 64, 3), (2, 41, 2), (4, 64, 2), (1, 200, 2), (2, 600, 2)])
-def test_outer_step_bf16_against_oracle(bits, k, R):
+@pytest.mark.parametrize("bits,k,R,deferred", [(2, 64, 3, False), (2, 64, 3, True), (2, 41, 2, False), (2, 200, 5, True),
+                                               (2, 1, 1, True), (4, 64, 2, False), (1, 200, 2, False), (2, 600, 2, False),
+                                               (3, 300, 1, False)])
+def test_outer_step_bf16_against_oracle(bits, k, R, deferred):
     from paper_2508_15706_b200 import binding as B
     O.set_threads(8)
     dev = torch.device("cuda", torch.cuda.current_device())
@@ -41,21 +43,30 @@ def test_outer_step_bf16_against_oracle(bits, k, R):
     cfg = O.Config(k=k, R=R, beta=wl.beta, outer_lr=wl.outer_lr, quant_bits=bits, storage_bf16=1)
     tab = O.Table(shapes, offs)
     assert sl.payload_bytes() == O.payload_bytes(cfg, tab)
+    if deferred:   # the corrected values wait (as fp32) in the workspace and are rounded when they reach e
+        sl.set_ef_deferred(True)
     theta = _padded(I.theta_sync(wl, dev))
     e = [_padded(I.initial_error(wl, r, dev, scale=0.5)) for r in range(R)]
     pay = [torch.full((sl.payload_bytes() + 64,), 0xC5, dtype=torch.uint8, device=dev) for _ in range(R)]
     th_o = _widen(theta[:n])
     e_o = [_widen(x[:n]) for x in e]
-    for step in range(2):
+    for step in range(3):
         local = [_padded(I.theta_local(wl, theta[:n].to(torch.float32), r, step)) for r in range(R)]
         lo_o = [_widen(x[:n]) for x in local]
         sl.outer_step(theta, local, e, pay)
         torch.cuda.synchronize()
+        assert sl.device_status() == 0
         want = O.outer_step(cfg, tab, th_o, lo_o, e_o)
+        true_e = e
+        if deferred:   # the error as the method defines it: the waiting values written into copies
+            assert sl.ef_pending()
+            true_e = [x.clone() for x in e]
+            sl.ef_flush(true_e, keep_pending=True)
+            torch.cuda.synchronize()
         for r in range(R):
             assert np.array_equal(pay[r][:-64].cpu().numpy(), want[r]), f"payload of worker {r}, step {step}"
             assert bool((pay[r][-64:] == 0xC5).all())
-            got_e = _widen(e[r][:n])
+            got_e = _widen(true_e[r][:n])
             assert np.array_equal(got_e.view(np.uint32), e_o[r].view(np.uint32)), f"e of worker {r}, step {step}"
             assert bool((e[r][n:] == 1.5).all()) and bool((local[r][n:] == 1.5).all())
         got = _widen(theta[:n])
@@ -66,6 +77,13 @@ def test_outer_step_bf16_against_oracle(bits, k, R):
             a, b = int(got.view(np.uint32)[i]) >> 16, int(th_o.view(np.uint32)[i]) >> 16
             assert abs(a - b) == 1, (i, got[i], th_o[i])
         th_o = got.copy()  # both sides continue from the same parameters
+    if deferred:
+        sl.ef_flush()
+        torch.cuda.synchronize()
+        assert not sl.ef_pending()
+        for r in range(R):
+            assert np.array_equal(_widen(e[r][:n]).view(np.uint32), e_o[r].view(np.uint32))
+            assert bool((e[r][n:] == 1.5).all())
 
 
 def test_halves_through_their_own_entry_points_and_type_checks():
@@ -121,6 +139,17 @@ def test_halves_through_their_own_entry_points_and_type_checks():
     with pytest.raises(B.SlError) as ei:
         B.SparseLoCo(shapes, offs, k=k, R=R, bf16_storage=True, quant_bits=32)
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
-    with pytest.raises(B.SlError) as ei:
-        sl.set_ef_deferred(True)
+    with pytest.raises(B.SlError) as ei:     # the fused update from coded payloads works on fp32 arrays
+        sl.aggregate_apply_coded([p, None, None], theta)
     assert ei.value.status == B.SL_ERR_UNSUPPORTED
+    # the wire codec and the validator are about payloads, not about storage
+    cap = sl.coded_payload_capacity()
+    coded = torch.zeros(cap, dtype=torch.uint8, device=dev)
+    size = torch.zeros(1, dtype=torch.int64, device=dev)
+    sl.encode_payload(pays[0], coded, size)
+    back = torch.zeros_like(pays[0])
+    sl.decode_payload(coded, back, int(size.item()))
+    status = torch.full((1,), -1, dtype=torch.int32, device=dev)
+    sl.validate_payload(back, status)
+    torch.cuda.synchronize()
+    assert torch.equal(back, pays[0]) and status.item() == 0
