@@ -1,4 +1,4 @@
-// Decode + average + outer update (optionally fused with the packing step), one warp per chunk.
+// Decode + average + outer update (optionally fused with the packing step, or with the decoding of coded payloads).
 // Part of libsparseloco (one translation unit: included by sparseloco.cu).
 #pragma once
 #include "common.cuh"

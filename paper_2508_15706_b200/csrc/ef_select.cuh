@@ -34,7 +34,9 @@ namespace {
 //  F. selected candidates set their bit in a 4096-bit map; its prefix popcount is the slot of each
 //     (ascending in-chunk index) and the holder writes (index, value) to the staging arrays.
 // All-zero chunks, thresholds of zero and more candidates than the list holds take an exact bitwise
-// search over all 4096 keys instead (select_slow).
+// search over all 4096 keys instead (select_slow).  Beyond keff = 256 (instantiation WIDE = 2) a threshold
+// over group maxima no longer thins the field and select_dense takes over: a key interval around the cut
+// narrowed on the registers, everything above it marked directly, the elements inside it listed and ranked.
 //
 // Chunks that cannot travel as tensor-map blocks (short tails, tables whose blocks do not start on a
 // 64-element boundary, tile copies switched off) are read and written with plain loads and stores by

@@ -15,7 +15,9 @@
 //   apply.cuh        decode_avg_apply_kernel  decode R payloads, sum, theta -= alpha/D * sum
 //                                             (Eq. 2 lines 3-4)
 // Beside the path: index_codec.cuh (entropy-coded indices for the wire), dense.cuh (DiLoCo's dense
-// outer step, Eq. 1), misc.cuh (payload validation).
+// outer step, Eq. 1, and the local-momentum baselines), misc.cuh (payload validation), quant_wide.cuh
+// (quantiser widths 1, 3, 4 and k beyond 256: plain kernels), bf16_storage.cuh (the selection kernel
+// for bfloat16 arrays).
 //
 // Everything is HBM-bound streaming except the per-chunk selection, which works on registers and
 // shared memory.  No tensor cores: nothing here is a dense contraction.
