@@ -313,10 +313,12 @@ def run_ours(args) -> dict:
                                                "scattered pass in every step"}
         sl.set_ef_deferred(True)
     if rank == 0 and world == 1 and not args.no_dense:
-        # the two halves of the step through their own entry points (sl_compress always writes
-        # the error correction in place; one worker per call)
+        # the two halves of the step through their own entry points, one worker per sl_compress call: first with
+        # the error correction written in place, then (one worker, called again and again as a rank of the
+        # worker-per-GPU deployment does) with it deferred
         if deferred:
             sl.ef_flush()
+        sl.set_ef_deferred(False)
         p0, p1, p2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         sl.compress(theta, locals_r[0], e[0], payloads[0])
         p0.record(stream)
@@ -328,7 +330,20 @@ def run_ours(args) -> dict:
         p2.record(stream)
         torch.cuda.synchronize()
         cms, ams = p0.elapsed_time(p1) / wl.R, p1.elapsed_time(p2) / 3
+        sl.set_ef_deferred(True)
+        for _ in range(2):
+            sl.compress(theta, locals_r[0], e[0], payloads[0])
+        p3, p4 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p3.record(stream)
+        for _ in range(8):
+            sl.compress(theta, locals_r[0], e[0], payloads[0])
+        p4.record(stream)
+        sl.ef_flush()
+        torch.cuda.synchronize()
+        if not deferred:
+            sl.set_ef_deferred(False)
         result["parts"] = {
+            "sl_compress_deferred_ms_per_worker": p3.elapsed_time(p4) / 8,
             "sl_compress_ms_per_worker": cms,
             "sl_compress_gbs": (16 + 2 * record_stride(k) / 4096.0) * N / (cms * 1e-3) / 1e9,
             "sl_aggregate_apply_ms": ams,
@@ -636,6 +651,7 @@ def run_worker_per_gpu(args) -> dict:
     coded = args.wire == "coded"
     ws = WorkerStep(sl, sl.payload_bytes(), world, rank, dev, coded=coded,
                     coded_capacity=sl.coded_payload_capacity() if coded else 0)
+    sl.set_ef_deferred(True)  # this rank's corrected values wait for its next sl_compress; one flush at the end, timed
     for _ in range(args.warmup):
         ws.step(theta, local, e)
     torch.cuda.synchronize()
@@ -651,6 +667,7 @@ def run_worker_per_gpu(args) -> dict:
     ev0.record(stream)
     for _ in range(args.steps):
         ws.step(theta, local, e)
+    sl.ef_flush()
     ev1.record(stream)
     torch.cuda.synchronize()
     t1 = time.time()

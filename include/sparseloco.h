@@ -297,9 +297,12 @@ sl_status sl_device_status(sl_ctx* ctx, void* cuda_stream);
  *   DEVICE pointers; NULL = the buffers of the last step), which then hold the true error.  With
  *   keep_pending != 0 the values keep waiting (use it to materialise a copy, e.g. for a checkpoint),
  *   and NULL entries of e skip that worker (one spare buffer then serves all workers in turn).
- * A step that cannot substitute them (error feedback frozen, deferral switched off, sl_compress(),
- * sl_outer_step_host()) writes them into the buffers of the last step first.  Only sl_outer_step()
- * defers. */
+ * sl_compress() defers in the same way for its one worker (the deployment with one worker per GPU: the
+ * values of that worker wait for its next sl_compress(), which must be given the same e).
+ * A step that cannot substitute them (error feedback frozen, deferral switched off, other buffers or
+ * another number of workers than the call that left them, sl_outer_step_host()) writes them into the
+ * buffers of the call that left them first.  sl_ef_flush()'s array then has as many entries as that
+ * call had workers. */
 sl_status sl_set_ef_deferred(sl_ctx* ctx, int32_t on);
 sl_status sl_ef_pending(const sl_ctx* ctx, int32_t* pending);
 sl_status sl_ef_flush(sl_ctx* ctx, float* const* e, int32_t keep_pending, void* cuda_stream);

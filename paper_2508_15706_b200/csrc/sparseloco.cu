@@ -85,6 +85,7 @@ struct sl_ctx {
     bool deferred;              // deferred error-feedback subtraction (sl_set_ef_deferred)
     bool pending;               // corrected values of the last step still wait in the workspace
     float* pending_e[kMaxR];    // the error buffers they belong to
+    int pending_workers;        // how many workers' values wait (R after sl_outer_step, 1 after sl_compress)
     void* ws_ptr;
     size_t ws_bytes;
     int last_workers;  // worker count the workspace was last laid out for
@@ -244,7 +245,7 @@ sl_status order_after_map_uploads(sl_ctx* c, cudaStream_t st) {
 }
 
 sl_status launch_flush(sl_ctx* c, const WorkerPtrs& ptrs, cudaStream_t st) {
-    const int R = c->cfg.R;
+    const int R = c->pending_workers;  // (the staging arrays are laid out for the call that left the values)
     const Workspace ws = carve(c, R);
     if (half_store(c))
         ef_flush_kernel<false, true><<<blocks_for(c->n_chunks * R, 4), 128, 0, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k,
@@ -273,7 +274,7 @@ sl_status flush_pending(sl_ctx* c, cudaStream_t st) {
     if (!c->pending) return SL_OK;
     WorkerPtrs fp;
     memset(&fp, 0, sizeof(fp));
-    for (int r = 0; r < c->cfg.R; ++r) fp.e[r] = c->pending_e[r];
+    for (int r = 0; r < c->pending_workers; ++r) fp.e[r] = c->pending_e[r];
     sl_status s = launch_flush(c, fp, st);
     if (s == SL_OK) c->pending = false;
     return s;
@@ -396,10 +397,12 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     const bool ef = c->cfg.ef_enabled != 0;
     bool consume = false;  // this step substitutes the waiting values while it streams e
     if (c->pending) {
-        if (ef && defer) {
+        bool same = c->pending_workers == workers;  // the values of exactly these buffers, in the same layout
+        for (int r = 0; r < workers && same; ++r) same = ptrs.e[r] == c->pending_e[r];
+        if (ef && defer && same) {
             consume = true;
             c->pending = false;
-        } else {  // nothing will read them in flight (frozen step): write them out first
+        } else {  // nothing will read them in flight (frozen step, other buffers): write them out first
             sl_status s = flush_pending(c, st);
             if (s != SL_OK) return s;
         }
@@ -465,6 +468,7 @@ sl_status launch_compress(sl_ctx* c, int workers, const float* theta_sync, const
     SL_CUDA(cudaGetLastError());
     if (ef && defer) {
         c->pending = true;
+        c->pending_workers = workers;
         for (int r = 0; r < workers; ++r) c->pending_e[r] = ptrs.e[r];
     }
     return SL_OK;
@@ -956,7 +960,9 @@ sl_status do_compress(sl_ctx* c, const float* theta_sync, const float* theta_loc
     ptrs.theta_local[0] = theta_local;
     ptrs.e[0] = e;
     ptrs.payload[0] = payload;
-    return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream), false);
+    // with deferral on, this worker's corrected values wait in the workspace for its next sl_compress
+    const bool defer = c->deferred && c->cfg.ef_enabled && fast_2bit(c);
+    return launch_compress(c, 1, theta_sync, ptrs, static_cast<cudaStream_t>(stream), defer);
 }
 
 sl_status do_aggregate_apply(sl_ctx* c, const uint8_t* const* payloads, float* theta_sync, void* stream) {
@@ -1047,7 +1053,7 @@ sl_status do_outer_step(sl_ctx* c, float* theta_sync, const float* const* theta_
         return launch_apply(c, pl, R, theta_sync, st);
     }
     const bool defer = c->deferred && c->cfg.ef_enabled;
-    if (c->pending && defer) {  // the waiting values can only be substituted into the buffers they came from
+    if (c->pending && defer && c->pending_workers == R) {  // they can only be substituted into the buffers they came from
         for (int r = 0; r < R; ++r)
             if (e[r] != c->pending_e[r]) return SL_ERR_INVALID_ARG;
     }
@@ -1423,7 +1429,7 @@ sl_status do_ef_flush(sl_ctx* c, float* const* e, int32_t keep_pending, void* st
     if (!c->pending) return SL_OK;
     WorkerPtrs ptrs;
     memset(&ptrs, 0, sizeof(ptrs));
-    for (int r = 0; r < c->cfg.R; ++r) {
+    for (int r = 0; r < c->pending_workers; ++r) {
         float* dst = e ? e[r] : c->pending_e[r];
         if (!dst && !keep_pending) return SL_ERR_INVALID_ARG;  // a worker may be skipped only if its values stay
         if (misaligned(dst)) return SL_ERR_ALIGNMENT;

@@ -529,3 +529,39 @@ def test_two_live_contexts_with_different_k():
         sl.aggregate_apply_coded([coded, None], theta, [int(size.item()), 0])
         torch.cuda.synchronize()
         assert sl.device_status() == 0
+
+
+def test_deferred_subtraction_in_sl_compress():
+    """The deployment with one worker per GPU calls sl_compress for its own worker only.  With deferral on,
+    that worker's corrected values wait in the workspace for its next sl_compress: payloads must be the
+    oracle's at every step, the true error (the waiting values written into a copy) too, and a call that
+    cannot use them (sl_outer_step with all workers) must first put them where they belong."""
+    import oracle as O
+    wl = I.Workload("compress_deferred", SMALL, R=2, k=41, recipe="student_t4", seed=91)
+    c = _case(wl, e_scale=0.5)
+    c.sl.set_ef_deferred(True)
+    tab = O.Table(c.shapes, c.offs)
+    cfg = O.Config(k=41, R=2, beta=wl.beta, outer_lr=wl.outer_lr)
+    theta_o = c.theta.cpu().numpy()
+    e_o = c.e[0].cpu().numpy().copy()
+    for step in range(3):
+        c.fill_local(step)
+        c.sl.compress(c.theta, c.local_of(0), c.e[0], c.payloads[0])
+        torch.cuda.synchronize()
+        assert c.sl.ef_pending() and c.guards_intact()
+        out = O.compress(cfg, tab, theta_o, c.local_of(0).cpu().numpy(), e_o)
+        assert np.array_equal(c.payloads[0].cpu().numpy(), out.payload), step
+        copy = c.e[0].clone()
+        c.sl.ef_flush([copy], keep_pending=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(copy.cpu().numpy().view(np.uint32), e_o.view(np.uint32)), step
+        assert not np.array_equal(c.e[0].cpu().numpy().view(np.uint32), e_o.view(np.uint32))  # (they do wait)
+    # a full outer step next: the single worker's values are written out before anything else happens
+    c.fill_local(3)
+    snap = c.snapshot(range(len(SMALL)))
+    assert np.array_equal(snap[0]["e"][1], c.e[1][c.offs[0]:c.offs[0] + SMALL[0].numel].cpu().numpy())
+    c.step()
+    for j in snap:   # the snapshot was taken with the values still waiting: give the oracle the true error
+        t, off = SMALL[j], c.offs[j]
+        snap[j]["e"][0] = e_o[off:off + t.numel].copy()
+    c.check(snap)
