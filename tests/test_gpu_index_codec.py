@@ -141,7 +141,7 @@ def test_damaged_coded_payloads_stay_inside_the_buffer():
     assert st == 4
 
 
-@pytest.mark.parametrize("k,R", [(1, 2), (8, 3), (41, 3), (64, 16), (123, 5), (256, 3), (64, 40)])
+@pytest.mark.parametrize("k,R", [(1, 2), (8, 3), (41, 3), (64, 16), (123, 5), (256, 3), (64, 40), (200, 64), (1, 1)])
 def test_aggregate_apply_straight_from_coded_payloads(k, R):
     """sl_aggregate_apply_coded (the decoding fused into the update kernel; Eq. 2 lines 3-4) must leave the
     bits that sl_decode_payload for every worker + sl_aggregate_apply leave, with an absent worker and with
