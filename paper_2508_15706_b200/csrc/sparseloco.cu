@@ -1321,8 +1321,10 @@ sl_status sl_encode_payload(sl_ctx* c, const uint8_t* payload, uint8_t* coded, u
     DeviceGuard g(c->device);
     if (!g.ok) return cuda_fail(cudaErrorInvalidDevice, "set device");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // scratch: two 32-bit words per chunk in the partial-sum area of the workspace (unused between
-    // compressions; the values a deferred subtraction keeps waiting live elsewhere)
+    // scratch: two 32-bit words per chunk in the partial-sum area of the workspace as laid out for R workers
+    // (unused between compressions).  The values a deferred subtraction keeps waiting live in the staging
+    // arrays, which end before that area both in the layout for R workers and in the one sl_compress uses
+    // for its single worker (R x G x kp x 6 bytes against G x kp x 6).
     unsigned* lens = reinterpret_cast<unsigned*>(carve(c, c->cfg.R).psum);
     unsigned* offs = lens + c->n_chunks;
     const long long G = c->n_chunks;

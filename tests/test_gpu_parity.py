@@ -544,11 +544,15 @@ def test_deferred_subtraction_in_sl_compress():
     cfg = O.Config(k=41, R=2, beta=wl.beta, outer_lr=wl.outer_lr)
     theta_o = c.theta.cpu().numpy()
     e_o = c.e[0].cpu().numpy().copy()
+    coded = torch.zeros(c.sl.coded_payload_capacity(), dtype=torch.uint8, device=c.dev)
+    size = torch.zeros(1, dtype=torch.int64, device=c.dev)
     for step in range(3):
         c.fill_local(step)
         c.sl.compress(c.theta, c.local_of(0), c.e[0], c.payloads[0])
         torch.cuda.synchronize()
         assert c.sl.ef_pending() and c.guards_intact()
+        # the wire codec borrows scratch from the workspace in which the values wait: it must not disturb them
+        c.sl.encode_payload(c.payloads[0], coded, size)
         out = O.compress(cfg, tab, theta_o, c.local_of(0).cpu().numpy(), e_o)
         assert np.array_equal(c.payloads[0].cpu().numpy(), out.payload), step
         copy = c.e[0].clone()
