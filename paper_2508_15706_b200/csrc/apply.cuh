@@ -172,88 +172,11 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                         my_pos = sbits;
                     }
                 }
-                const unsigned* __restrict__ stream = reinterpret_cast<const unsigned*>(pl.p[tid] + fa.stream_off);
-                const unsigned long long wtot = sbits >> 5;
-                // a 64-bit window over the stream, refilled a word at a time (consecutive words: mostly L1 hits;
-                // words past the stated size read as zeros)
-                unsigned long long win = 0, wnext = my_pos >> 5;
-                int have = 0;
-                auto refill = [&]() {  // at least 32 valid bits
-                    while (have < 32) {
-                        const unsigned x = wnext < wtot ? __ldg(stream + wnext) : 0u;
-                        win |= (unsigned long long)x << have;
-                        have += 32;
-                        ++wnext;
-                    }
-                };
-                refill();
-                {
-                    const int skip = (int)(my_pos & 31ull);
-                    win >>= skip;
-                    have -= skip;
-                }
-                const IxcCode code = ixc_code(cd.len, keff);
-                unsigned consumed = 0;
-                int prev = -1;
+                IxcReader rd;
+                ixc_reader_open(rd, reinterpret_cast<const unsigned*>(pl.p[tid] + fa.stream_off), sbits, my_pos);
                 uint16_t* out = sidx + (size_t)tid * fa.kp;
-                const int nb = code.M > 1u ? (int)code.b - 1 : 0;  // remainder bits before the optional last one
-                for (int s = 0; s < keff; ++s) {
-                    if (have < 32) {  // (at most 32 bits are taken per round below, so one word restores the 32)
-                        const unsigned x = wnext < wtot ? __ldg(stream + wnext) : 0u;
-                        win |= (unsigned long long)x << have;
-                        have += 32;
-                        ++wnext;
-                    }
-                    const unsigned lo32 = (unsigned)win, inv = ~lo32;
-                    const int ones = __ffs(inv) - 1;  // -1 when all 32 bits are ones
-                    unsigned gap;
-                    int used;
-                    if (ones >= 0 && ones <= 19) {
-                        // the whole code lies in these 32 bits (at most 20 + 11 + 1): no branches from here on
-                        const unsigned w2 = lo32 >> (ones + 1);
-                        const unsigned r1 = nb ? __brev(w2) >> (32 - nb) : 0u;
-                        const bool longer = code.M > 1u && r1 >= code.cut;  // truncated binary: one more bit
-                        const unsigned r = longer ? ((r1 << 1) | ((w2 >> nb) & 1u)) - code.cut : r1;
-                        gap = (unsigned)ones * code.M + r;
-                        used = ones + 1 + nb + (longer ? 1 : 0);
-                        win >>= used;
-                        have -= used;
-                    } else {  // a long run of one-bits: bit by bit through the window (rare; bounded)
-                        unsigned q = 0, iv = inv;
-                        used = 0;
-                        while (iv == 0u && q < 4096u) {
-                            q += 32;
-                            win >>= 32;
-                            have -= 32;
-                            used += 32;
-                            refill();
-                            iv = ~(unsigned)win;
-                        }
-                        const int o2 = iv ? __ffs(iv) - 1 : 0;
-                        q += o2;
-                        win >>= o2 + 1;
-                        have -= o2 + 1;
-                        used += o2 + 1;
-                        unsigned r = 0;
-                        if (code.M > 1u) {
-                            refill();
-                            if (nb) r = __brev((unsigned)win) >> (32 - nb);
-                            win >>= nb;
-                            have -= nb;
-                            used += nb;
-                            if (r >= code.cut) {
-                                r = ((r << 1) | ((unsigned)win & 1u)) - code.cut;
-                                win >>= 1;
-                                have -= 1;
-                                used += 1;
-                            }
-                        }
-                        gap = q * code.M + r;
-                    }
-                    consumed += (unsigned)used;
-                    prev = prev + 1 + (int)gap;
-                    out[s] = (uint16_t)((unsigned)prev & 0xFFFu);
-                }
+                const unsigned consumed =
+                    ixc_decode_chunk(rd, ixc_code(cd.len, keff), keff, [&](int s, unsigned idx) { out[s] = (uint16_t)idx; });
                 my_pos += consumed;
                 if (my_pos > sbits) {
                     my_bad = true;

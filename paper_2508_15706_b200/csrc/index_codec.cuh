@@ -161,6 +161,102 @@ ixc_write_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n
     if (fill) atomicOr(&stream[word], (unsigned)acc);
 }
 
+// Reading a worker's index stream: a 64-bit window over the 32-bit words, refilled a word at a time through
+// the read-only path (consecutive words: mostly L1 hits).  `stream_bits` (a multiple of 32) = the bits the
+// caller's buffer holds: words past it read as zeros, so no access ever leaves the buffer.
+struct IxcReader {
+    const unsigned* stream;
+    unsigned long long wtot, wnext, win;
+    int have;  // valid bits in `win`, lowest first
+};
+__device__ __forceinline__ void ixc_refill(IxcReader& rd) {  // at least 32 valid bits afterwards
+    while (rd.have < 32) {
+        const unsigned x = rd.wnext < rd.wtot ? __ldg(rd.stream + rd.wnext) : 0u;
+        rd.win |= (unsigned long long)x << rd.have;
+        rd.have += 32;
+        ++rd.wnext;
+    }
+}
+__device__ __forceinline__ void ixc_reader_open(IxcReader& rd, const unsigned* stream, unsigned long long stream_bits,
+                                                unsigned long long bit_pos) {
+    rd.stream = stream;
+    rd.wtot = stream_bits >> 5;
+    rd.wnext = bit_pos >> 5;
+    rd.win = 0;
+    rd.have = 0;
+    ixc_refill(rd);
+    const int skip = (int)(bit_pos & 31ull);
+    rd.win >>= skip;
+    rd.have -= skip;
+}
+// Decodes the m gap codes of one chunk; emit(s, index) receives the ascending indices (12 bits kept).
+// Returns the bits consumed.  A damaged stream cannot run away: a run of one-bits is cut at 4096 and bits
+// beyond the buffer are zeros, so every code ends.
+template <typename Emit>
+__device__ __forceinline__ unsigned ixc_decode_chunk(IxcReader& rd, const IxcCode code, int m, Emit emit) {
+    const int nb = code.M > 1u ? (int)code.b - 1 : 0;  // remainder bits before the optional last one
+    unsigned consumed = 0;
+    int prev = -1;
+    for (int s = 0; s < m; ++s) {
+        if (rd.have < 32) {  // (at most 32 bits are taken per round below, so one word restores the 32)
+            const unsigned x = rd.wnext < rd.wtot ? __ldg(rd.stream + rd.wnext) : 0u;
+            rd.win |= (unsigned long long)x << rd.have;
+            rd.have += 32;
+            ++rd.wnext;
+        }
+        const unsigned lo32 = (unsigned)rd.win, inv = ~lo32;
+        const int ones = __ffs(inv) - 1;  // -1 when all 32 bits are ones
+        unsigned gap;
+        int used;
+        if (ones >= 0 && ones <= 19) {
+            // the whole code lies in these 32 bits (at most 20 + 11 + 1): no branches from here on
+            const unsigned w2 = lo32 >> (ones + 1);
+            const unsigned r1 = nb ? __brev(w2) >> (32 - nb) : 0u;
+            const bool longer = code.M > 1u && r1 >= code.cut;  // truncated binary: one more bit
+            const unsigned r = longer ? ((r1 << 1) | ((w2 >> nb) & 1u)) - code.cut : r1;
+            gap = (unsigned)ones * code.M + r;
+            used = ones + 1 + nb + (longer ? 1 : 0);
+            rd.win >>= used;
+            rd.have -= used;
+        } else {  // a long run of one-bits: through the window 32 bits at a time (rare; bounded)
+            unsigned q = 0, iv = inv;
+            used = 0;
+            while (iv == 0u && q < 4096u) {
+                q += 32;
+                rd.win >>= 32;
+                rd.have -= 32;
+                used += 32;
+                ixc_refill(rd);
+                iv = ~(unsigned)rd.win;
+            }
+            const int o2 = iv ? __ffs(iv) - 1 : 0;
+            q += o2;
+            rd.win >>= o2 + 1;
+            rd.have -= o2 + 1;
+            used += o2 + 1;
+            unsigned r = 0;
+            if (code.M > 1u) {  // truncated binary, most significant bit first
+                ixc_refill(rd);
+                if (nb) r = __brev((unsigned)rd.win) >> (32 - nb);
+                rd.win >>= nb;
+                rd.have -= nb;
+                used += nb;
+                if (r >= code.cut) {
+                    r = ((r << 1) | ((unsigned)rd.win & 1u)) - code.cut;
+                    rd.win >>= 1;
+                    rd.have -= 1;
+                    used += 1;
+                }
+            }
+            gap = q * code.M + r;
+        }
+        consumed += (unsigned)used;
+        prev = prev + 1 + (int)gap;
+        emit(s, (unsigned)prev & 0xFFFu);
+    }
+    return consumed;
+}
+
 // K4: coded payload -> 12-bit records.  One thread per group of 16 chunks (one directory entry).
 // `stream_bits` = bits of the index stream that the caller's buffer holds: a read position taken from
 // the directory is clamped to it and a bit past it reads as 0, so a corrupted directory or stream
@@ -175,49 +271,32 @@ ixc_decode_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
         reinterpret_cast<unsigned*>(payload)[grp] = reinterpret_cast<const unsigned*>(coded)[grp];
     const long long g0 = grp * kIxcGroup;
     if (g0 >= n_chunks) return;
-    const unsigned* stream = reinterpret_cast<const unsigned*>(coded + stream_off);
     const unsigned* dir = reinterpret_cast<const unsigned*>(coded + dir_off);
     unsigned long long pos = dir[grp];
     bool bad = pos > stream_bits;
     if (g0 + kIxcGroup < n_chunks) bad |= dir[grp + 1] < pos;
     if (pos > stream_bits) pos = stream_bits;
     const int cb = (2 * k + 7) / 8, ib = (12 * k + 7) / 8, stride = record_stride(k);
-    auto get1 = [&]() -> unsigned {
-        if (pos >= stream_bits) {
-            bad = true;
-            return 0u;
-        }
-        const unsigned bit = (stream[pos >> 5] >> (pos & 31)) & 1u;
-        ++pos;
-        return bit;
-    };
+    IxcReader rd;
+    ixc_reader_open(rd, reinterpret_cast<const unsigned*>(coded + stream_off), stream_bits, pos);
     for (long long g = g0; g < g0 + kIxcGroup && g < n_chunks; ++g) {
         const ChunkDesc cd = chunks[g];
         const int m = min(k, cd.len);
-        const IxcCode c = ixc_code(cd.len, m);
         uint8_t* recb = payload + cd.rec_off;
         unsigned* rec = reinterpret_cast<unsigned*>(recb);
         // the record is this thread's alone: index words are assembled in a register and stored
         unsigned long long acc = 0;
         unsigned fill = 0;
-        int w = 0, prev = -1;
-        for (int s = 0; s < m; ++s) {
-            unsigned q = 0;
-            while (get1() && q < 4096u) ++q;  // a corrupted stream cannot run away
-            unsigned r = 0;
-            if (c.M > 1) {
-                for (unsigned i = 0; i + 1 < c.b; ++i) r = (r << 1) | get1();
-                if (r >= c.cut) r = ((r << 1) | get1()) - c.cut;
-            }
-            prev = prev + 1 + (int)(q * c.M + r);
-            acc |= (unsigned long long)((unsigned)prev & 0xFFFu) << fill;
+        int w = 0;
+        pos += ixc_decode_chunk(rd, ixc_code(cd.len, m), m, [&](int, unsigned idx) {
+            acc |= (unsigned long long)idx << fill;
             fill += 12;
             if (fill >= 32) {
                 rec[w++] = (unsigned)acc;
                 acc >>= 32;
                 fill -= 32;
             }
-        }
+        });
         // rest of the index block, the code block, the padding: byte-wise after the whole words
         int byte = 4 * w;
         for (; byte < ib; ++byte, acc >>= 8) recb[byte] = (uint8_t)(acc & 0xFFu);
@@ -225,6 +304,7 @@ ixc_decode_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int 
         for (int i = 0; i < cb; ++i) recb[ib + i] = csrc[i];
         for (byte = ib + cb; byte < stride; ++byte) recb[byte] = 0;
     }
+    if (pos > stream_bits) bad = true;  // the codes ran past what the buffer holds
     if (bad) atomicExch(status, (int)SL_ERR_BAD_PAYLOAD);
 }
 
