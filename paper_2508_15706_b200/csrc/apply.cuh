@@ -37,9 +37,12 @@ namespace {
 // FUSE 5: the payloads are in the entropy-coded wire form (index_codec.cuh) and are decoded here instead of
 // being expanded to records first.  A chunk's position in a worker's index stream is known only after
 // the chunks before it in its group of 16 (one directory entry per group), so a CTA takes whole groups
-// and walks their chunks in order; thread r keeps worker r's read position and decodes the chunk's gaps
-// through a 64-bit register window over the stream into a shared index list, and the rest of the kernel
-// reads the list and the code blocks.  Reads of a
+// and walks their chunks in order.  The CTA has two extra warps for this: decoder thread r keeps worker r's
+// read position and decodes the chunk's gaps through a 64-bit register window over the stream into one of
+// two shared index lists, one chunk ahead of the four warps that run the update proper, which read the
+// list and the code blocks.  The two groups meet through two counters in shared memory (chunks decoded,
+// chunks whose list has been read) with bounded polls -- SL_ERR_TIMEOUT and an orderly exit of both groups if
+// one ever runs out -- and each group keeps to a named barrier of its own size.  Reads of a
 // stream are confined to the size its buffer is said to have; a stream that runs out reads as zeros
 // and is recorded as SL_ERR_BAD_PAYLOAD.
 //
@@ -65,6 +68,7 @@ constexpr int kApplyThreads = 32 * kApplyWarps;
 constexpr int kApplyCtasPerSm = 6;   // what the shared memory of a CTA (tile, records, staging block) lets an SM hold
 constexpr int kApplyBatch = 16;                  // workers decoded between two rounds of ordered additions
 constexpr int kApplyPerWarp = kApplyBatch / kApplyWarps;
+constexpr int kApplyDecoders = 64;                  // FUSE 5: two more warps, one thread per worker, decode one chunk ahead
 constexpr int kApplyTile = kChunk + kApplyThreads;  // the sum tile + one dump slot per thread for entries that do not count
 
 __host__ __device__ constexpr size_t apply_smem_bytes(int k) {
@@ -88,7 +92,7 @@ __device__ __forceinline__ void async_copy_wait_all() {
 // HALF (FUSE 0-2): theta and the error buffers are bfloat16 arrays; they are widened on the way in and what is
 // stored is rounded once to nearest-even, the arithmetic in between is the fp32 arithmetic of the fp32 form.
 template <int PPL, int FUSE, bool HALF = false>
-__global__ void __launch_bounds__(kApplyThreads, kApplyCtasPerSm)
+__global__ void __launch_bounds__(FUSE == 5 ? kApplyThreads + kApplyDecoders : kApplyThreads, kApplyCtasPerSm)
 decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks, int n_workers, int k, float scale,
                         PayloadPtrs pl, float* __restrict__ theta_sync, FuseArgs fa, WorkerPtrs ptrs) {
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -107,11 +111,19 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     const unsigned dump = (unsigned)(kChunk + tid);  // where an entry that does not count adds its 0
     // per-worker strides of the staging arrays, in index pairs / value pairs (kp is a multiple of 8)
     const long long wstride = STAGED ? fa.n_chunks * (long long)fa.kp / 2 : 0;
-    // CODED: per worker kp decoded indices
-    uint16_t* sidx = reinterpret_cast<uint16_t*>(stage + kChunk / 4);
-    unsigned long long my_pos = 0;   // thread r: worker r's read position in its index stream
-    bool my_bad = false;
+    // CODED: two lists of kp decoded indices per worker, then the two counters and the abort flag
+    uint16_t* sidx_all = reinterpret_cast<uint16_t*>(stage + kChunk / 4);
+    const size_t sidx_len = CODED ? (size_t)n_workers * fa.kp : 0;
+    // [0] chunks decoded, [1] chunks whose lists have been read, [2] abort (set by whoever's wait ran out),
+    // [3] / [4] what the decoders / the update warps decided at their last meeting point (written by one thread
+    // before the group's barrier and read by all after it, so that a whole group stops at the same place)
+    int* sync_words = reinterpret_cast<int*>(sidx_all + 2 * ((sidx_len + 7) / 8 * 8));
     const int cb = (2 * k + 7) / 8;  // bytes of a chunk's code block in a coded payload
+    // the 128 threads of the update meet at a barrier of their own when decoder warps share the CTA
+    auto cta_sync = [&]() {
+        if (CODED) asm volatile("bar.sync 1, 128;" ::: "memory");
+        else __syncthreads();
+    };
     // the CTA's walk: chunk after chunk inside a group of kIxcGroup when CODED, else every gridDim-th chunk
     auto next_of = [&](long long g) -> long long {
         if (!CODED) return g + gridDim.x;
@@ -120,8 +132,68 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
     };
     const long long g_first = CODED ? (long long)blockIdx.x * kIxcGroup : (long long)blockIdx.x;
 
+    if (CODED) {
+        if (tid == 0) sync_words[0] = sync_words[1] = sync_words[2] = sync_words[3] = sync_words[4] = 0;
+        __syncthreads();  // (all 192 threads, once: the counters start at zero for both groups)
+    }
+    if (CODED && tid >= kApplyThreads) {
+        // ------------------------------------------------------------ decoder warps: one chunk ahead
+        const int d = tid - kApplyThreads;  // worker
+        const bool mine = d < n_workers && pl.p[d] != nullptr;
+        const unsigned long long sbits = mine ? fa.stream_bits[d] : 0ull;
+        unsigned long long my_pos = 0;  // worker d's read position in its index stream
+        bool my_bad = false;
+        int i = 0;
+        for (long long g = g_first; g < n_chunks; g = next_of(g), ++i) {
+            if (d == 0) {  // the list that chunk i goes into was last used by chunk i - 2
+                bool ok = false;
+                for (unsigned it = 0; it < (1u << 22); ++it) {
+                    int done;
+                    asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(done) : "r"((unsigned)__cvta_generic_to_shared(&sync_words[1])) : "memory");
+                    if (done >= i - 1) {
+                        ok = true;
+                        break;
+                    }
+                    if (*reinterpret_cast<volatile int*>(&sync_words[2])) break;
+                    __nanosleep(64);
+                }
+                if (!ok) {
+                    if (!*reinterpret_cast<volatile int*>(&sync_words[2])) atomicExch(fa.status, (int)SL_ERR_TIMEOUT);
+                    *reinterpret_cast<volatile int*>(&sync_words[2]) = 1;
+                    *reinterpret_cast<volatile int*>(&sync_words[3]) = 1;
+                }
+            }
+            asm volatile("bar.sync 2, 64;" ::: "memory");
+            if (*reinterpret_cast<volatile int*>(&sync_words[3])) break;  // (written by one thread before the barrier)
+            if (mine) {
+                const ChunkDesc dcd = chunks[g];
+                const int dk = min(k, dcd.len);
+                if (g % kIxcGroup == 0) {  // a new group: its directory entry
+                    my_pos = reinterpret_cast<const unsigned*>(pl.p[d] + fa.dir_off)[g / kIxcGroup];
+                    if (my_pos > sbits) {
+                        my_bad = true;
+                        my_pos = sbits;
+                    }
+                }
+                IxcReader rd;
+                ixc_reader_open(rd, reinterpret_cast<const unsigned*>(pl.p[d] + fa.stream_off), sbits, my_pos);
+                uint16_t* out = sidx_all + (size_t)(i & 1) * ((sidx_len + 7) / 8 * 8) + (size_t)d * fa.kp;
+                my_pos += ixc_decode_chunk(rd, ixc_code(dcd.len, dk), dk, [&](int s, unsigned idx) { out[s] = (uint16_t)idx; });
+                if (my_pos > sbits) {
+                    my_bad = true;
+                    my_pos = sbits;
+                }
+            }
+            asm volatile("bar.sync 2, 64;" ::: "memory");  // every worker's list of chunk i is written
+            if (d == 0)
+                asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(&sync_words[0])), "r"(i + 1) : "memory");
+        }
+        if (my_bad) atomicExch(fa.status, (int)SL_ERR_BAD_PAYLOAD);
+        return;
+    }
+
     for (int i = tid; i < kApplyTile / 4; i += kApplyThreads) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    __syncthreads();
+    cta_sync();
 
     // thread t owns in-chunk indices 512 i + 4 t + j: block row 8 i + t / 16, column 4 (t % 16)
     bf16_bits* const theta_h = reinterpret_cast<bf16_bits*>(theta_sync);  // HALF: the same array seen as bfloat16
@@ -144,7 +216,8 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
         if (cd_next.len == kChunk) prefetch_theta(cd_next);
     }
 
-    for (long long g = g_first; g < n_chunks; g = next_of(g)) {
+    int seq = 0;  // position of the chunk in this CTA's walk
+    for (long long g = g_first; g < n_chunks; g = next_of(g), ++seq) {
         const ChunkDesc cd = cd_next;
         const int keff = min(k, cd.len);
         const bool full = cd.len == kChunk;
@@ -163,28 +236,28 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
             if (cd_next.len == kChunk) prefetch_theta(cd_next);
         }
         if (CODED) {
-            if (tid < n_workers && pl.p[tid]) {
-                const unsigned long long sbits = fa.stream_bits[tid];
-                if (g == g_first || g % kIxcGroup == 0) {  // a new group: its directory entry
-                    my_pos = reinterpret_cast<const unsigned*>(pl.p[tid] + fa.dir_off)[g / kIxcGroup];
-                    if (my_pos > sbits) {
-                        my_bad = true;
-                        my_pos = sbits;
+            if (tid == 0) {  // the decoders have finished this chunk's lists
+                bool ok = false;
+                for (unsigned it = 0; it < (1u << 22); ++it) {
+                    int made;
+                    asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(made) : "r"((unsigned)__cvta_generic_to_shared(&sync_words[0])) : "memory");
+                    if (made > seq) {
+                        ok = true;
+                        break;
                     }
+                    if (*reinterpret_cast<volatile int*>(&sync_words[2])) break;
+                    __nanosleep(64);
                 }
-                IxcReader rd;
-                ixc_reader_open(rd, reinterpret_cast<const unsigned*>(pl.p[tid] + fa.stream_off), sbits, my_pos);
-                uint16_t* out = sidx + (size_t)tid * fa.kp;
-                const unsigned consumed =
-                    ixc_decode_chunk(rd, ixc_code(cd.len, keff), keff, [&](int s, unsigned idx) { out[s] = (uint16_t)idx; });
-                my_pos += consumed;
-                if (my_pos > sbits) {
-                    my_bad = true;
-                    my_pos = sbits;
+                if (!ok) {
+                    if (!*reinterpret_cast<volatile int*>(&sync_words[2])) atomicExch(fa.status, (int)SL_ERR_TIMEOUT);
+                    *reinterpret_cast<volatile int*>(&sync_words[2]) = 1;
+                    *reinterpret_cast<volatile int*>(&sync_words[4]) = 1;
                 }
             }
-            __syncthreads();  // the index lists of this chunk are complete
+            cta_sync();
+            if (*reinterpret_cast<volatile int*>(&sync_words[4])) break;  // (written by one thread before the barrier)
         }
+        const uint16_t* sidx = sidx_all + (size_t)(seq & 1) * ((sidx_len + 7) / 8 * 8);
         // which of this lane's slots exist in this chunk (the same for every worker)
         bool in0[PPL], in1[PPL];
 #pragma unroll
@@ -259,7 +332,9 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                     }
                 }
             }
-            __syncthreads();  // tables and zeroed records are in place
+            cta_sync();  // tables and zeroed records are in place
+            if (CODED && r0 + kApplyBatch >= n_workers && tid == 0)  // the lists of this chunk have been read (last batch)
+                asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(&sync_words[1])), "r"(seq + 1) : "memory");
 #pragma unroll
             for (int q = 0; q < WB; ++q) {
                 const int r = r0 + w0 + q;
@@ -329,7 +404,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
                         __syncwarp();
                     }
                 }
-                __syncthreads();
+                cta_sync();
             }
             if (PACK) {  // the records of the batch are complete (written before the barriers above): out they go
                 const int vpr = stride / 16;
@@ -405,7 +480,7 @@ decode_avg_apply_kernel(const ChunkDesc* __restrict__ chunks, long long n_chunks
         }
         // (the next chunk's first additions come after several CTA barriers: the cleared tile is seen by all)
     }
-    if (CODED && my_bad) atomicExch(fa.status, (int)SL_ERR_BAD_PAYLOAD);
+    async_copy_wait_all();  // (an early exit leaves the copies of the chunk to come in flight)
 }
 
 }  // namespace

@@ -576,7 +576,8 @@ sl_status launch_apply_coded(sl_ctx* c, const PayloadPtrs& pl, const size_t* cod
     for (int r = 0; r < R; ++r) fa.stream_bits[r] = pl.p[r] ? (unsigned long long)((coded_bytes[r] - c->ixc_stream_off) / 4 * 4) * 8ull : 0ull;
     WorkerPtrs wp;
     memset(&wp, 0, sizeof(wp));
-    const size_t smem = (apply_smem_bytes(c->cfg.k) + (size_t)R * c->kp * sizeof(uint16_t) + 15) / 16 * 16;
+    // + two index lists per worker (each rounded up to 8 entries) and the words the two groups of warps meet through
+    const size_t smem = apply_smem_bytes(c->cfg.k) + 2 * (((size_t)R * c->kp + 7) / 8 * 8) * sizeof(uint16_t) + 32;
     if (smem > 227u * 1024u) return SL_ERR_UNSUPPORTED;
     const long long groups = (c->n_chunks + kIxcGroup - 1) / kIxcGroup;
     const long long fit = (227ll * 1024) / ((long long)smem + 1024);
@@ -584,11 +585,11 @@ sl_status launch_apply_coded(sl_ctx* c, const PayloadPtrs& pl, const size_t* cod
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
     const int ppl = (c->cfg.k + 63) / 64;
     if (ppl <= 1)
-        decode_avg_apply_kernel<1, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
+        decode_avg_apply_kernel<1, 5><<<grid, kApplyThreads + kApplyDecoders, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
     else if (ppl <= 2)
-        decode_avg_apply_kernel<2, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
+        decode_avg_apply_kernel<2, 5><<<grid, kApplyThreads + kApplyDecoders, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
     else
-        decode_avg_apply_kernel<4, 5><<<grid, kApplyThreads, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
+        decode_avg_apply_kernel<4, 5><<<grid, kApplyThreads + kApplyDecoders, smem, st>>>(c->d_chunks, c->n_chunks, R, c->cfg.k, scale, pl, theta_sync, fa, wp);
     SL_CUDA(cudaGetLastError());
     return SL_OK;
 }
